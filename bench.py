@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the pivoted (PBP) fully-connected layer on B200.
+
+A step is one forward call of one layer: y = act(W x + b), batch 1, on the
+8192 x 8192 fp16 workload (tile 64, k of 128 tiles kept per block-row; k=128
+is density 1.0).  Prints ONE JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--k 128] [--impl reference]
+
+Device-timed `value` (us per layer) replays a CUDA graph of forward calls that
+rotate over enough independent copies of the layer that no call finds its
+weights in L2.  `e2e` is the same call made from host buffers through the
+Python binding (pinned host -> device copy, forward, device -> host read, sync).
+With several GPUs every rank runs an independent replica (no collective on the
+data path); the time is the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "pivoted_fc_us_per_layer_batch1"
+L2_BYTES = 126 * 1024 * 1024
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peak_gbs():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def algorithmic_bytes(lay, batch, n_tile_col):
+    """Bytes one forward call must move: kept tiles, index arrays, x, y, permutations, bias."""
+    esz = lay.tile_values.dtype.itemsize
+    Mb, Nb = lay.Mb, lay.Nb
+    b = lay.T * lay.B * lay.B * esz
+    b += 4 * (n_tile_col + Mb + 1)
+    b += lay.N * batch * esz + lay.M * batch * 4
+    b += 4 * (Nb * lay.B + Mb * lay.B)
+    b += 4 * lay.M if lay.bias is not None else 0
+    return b
+
+
+class ClockSampler:
+    """nvidia-smi polling in a child process; killed by PID when done."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        rows = []
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                ts = time.mktime(time.strptime(parts[0].split(".")[0], "%Y/%m/%d %H:%M:%S")) + \
+                    float("0." + parts[0].split(".")[1])
+                rows.append((ts, float(parts[1]), float(parts[2]), parts[4:8]))
+            except Exception:
+                continue
+        inside = [r for r in rows if t0 <= r[0] <= t1]
+        use = inside if len(inside) >= 3 else rows
+        if not use:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({n for r in use for n, v in zip(names, r[3]) if v.lower().startswith("active")})
+        return {"sm_mhz": statistics.median(r[1] for r in use), "sm_max_mhz": use[0][2], "reasons": reasons,
+                "samples": len(use), "window": "timed region" if use is inside else "whole run"}
+
+
+def cpu_baseline(lay, x, budget_s=12.0):
+    """The oracle as it stands, on this host: dense fp64 reconstruction, then matrix-vector products."""
+    from oracle import pp_oracle as po
+    cores = os.cpu_count() or 1
+    t0 = time.perf_counter()
+    W = po.reconstruct(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values)
+    t_rec = time.perf_counter() - t0
+    x64 = x.astype(np.float64)
+    po.dense_forward(W, lay.bias, x64, lay.act, threads=cores)
+    reps, t_acc = 0, 0.0
+    while t_acc < budget_s and reps < 30:
+        t0 = time.perf_counter()
+        po.dense_forward(W, lay.bias, x64, lay.act, threads=cores)
+        t_acc += time.perf_counter() - t0
+        reps += 1
+    return {"value": t_acc / reps * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
+            "sample": f"{reps} full dense fp64 matrix-vector products of the same layer "
+                      f"(dense reconstruction, {t_rec:.2f} s, done once and not counted)"}
+
+
+def run_reference(args, rank):
+    """Reference arm: the CPU oracle timed on the host cores, same workload, metric and unit."""
+    if rank != 0:
+        return
+    from oracle import pp_oracle as po
+    from paper_1712_01084_b200 import synth
+    wl = synth.config5(k=args.k, batch=1)
+    lay = wl.layers[0]
+    cores = os.cpu_count() or 1
+    W = po.reconstruct(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values)
+    x64 = wl.x.astype(np.float64)
+    t0 = time.perf_counter()
+    po.dense_forward(W, None, x64, lay.act, threads=cores)
+    t_full = time.perf_counter() - t0
+    # each step is a sample of output rows sized so that the whole run stays near two minutes
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    frac = min(1.0, budget / max(t_full, 1e-9))
+    n_rows = max(8, int(lay.M * frac))
+    rows = np.random.default_rng(0).choice(lay.M, n_rows, replace=False).astype(np.int32)
+    run = (lambda: po.dense_forward(W, None, x64, lay.act, threads=cores)) if n_rows >= lay.M else \
+          (lambda: po.dense_forward_rows(W, None, x64, lay.act, rows))
+    used = cores if n_rows >= lay.M else 1
+    for _ in range(args.warmup):
+        run()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run()
+    t = (time.perf_counter() - t0) / args.steps
+    us = t * 1e6 * (lay.M / min(n_rows, lay.M))
+    sample = f"{min(n_rows, lay.M)} of {lay.M} output rows per step, scaled to the full layer"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": us, "unit": "us", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": us / 1e3, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": 1, "M": lay.M, "N": lay.N, "B": lay.B, "tiles_per_block_row": args.k},
+        "cpu_baseline": {"value": us, "unit": "us", "cores": used, "kind": "oracle", "sample": sample},
+        "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def time_graph(pb, torch, replicas, x, y, act, steps, warmup, chunk=500):
+    """Device time of `steps` forward calls (rotating replicas) replayed from CUDA graphs."""
+    fn = pb.lib().pp_forward
+    xp, yp = ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(y.data_ptr())
+    handles = [r._h for r in replicas]
+    R = len(handles)
+
+    def enqueue(n, start, stream_ptr):
+        for s in range(n):
+            st = fn(handles[(start + s) % R], xp, yp, 1, act, stream_ptr)
+            if st != 0:
+                raise pb.PPError(st, "pp_forward")
+
+    stream = torch.cuda.Stream()
+    graphs = {}
+    with torch.cuda.stream(stream):
+        sp = ctypes.c_void_p(stream.cuda_stream)
+        enqueue(max(warmup, 3), 0, sp)              # untimed warm-up, plain launches
+        stream.synchronize()
+        chunk = min(chunk, steps)
+        chunk -= chunk % R if chunk > R else 0
+        chunk = max(chunk, 1)
+        for n in {chunk, steps % chunk} - {0}:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                enqueue(n, 0, ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+            graphs[n] = g
+        graphs[chunk].replay()                      # one untimed replay
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        return stream, graphs, chunk, e0, e1
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--k", type=int, default=128, help="kept tiles per block-row (of 128)")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the density sweep")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_1712_01084_b200 import binding as pb
+    from paper_1712_01084_b200 import synth
+
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    pb.lib()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    def build(k):
+        wl = synth.config5(k=k, batch=1)
+        lay = wl.layers[0]
+        L0 = pb.Layer.from_synth(lay)
+        pk_bytes = lay.T * lay.B * lay.B * 2
+        R = max(2, -(-2 * L2_BYTES // pk_bytes) + 1)
+        reps = [L0] + [L0.clone() for _ in range(R - 1)]
+        return wl, lay, reps
+
+    def time_config(k, steps, warmup, sample_clocks=False):
+        wl, lay, reps = build(k)
+        x = torch.from_numpy(wl.x).cuda()
+        y = torch.empty((1, lay.M), dtype=torch.float32, device="cuda")
+        stream, graphs, chunk, e0, e1 = time_graph(pb, torch, reps, x, y, lay.act, steps, warmup)
+        sampler = ClockSampler(local_rank) if sample_clocks else None
+        if sampler:
+            time.sleep(0.3)
+        barrier()
+        torch.cuda.synchronize()
+        w0 = time.time()
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _ in range(steps // chunk):
+                graphs[chunk].replay()
+            if steps % chunk:
+                graphs[steps % chunk].replay()
+            e1.record(stream)
+        torch.cuda.synchronize()
+        w1 = time.time()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        clocks = sampler.stop(w0, w1) if sampler else None
+        return wl, lay, reps, x, y, ms, clocks
+
+    wl, lay, reps, x, y, ms, clocks = time_config(args.k, args.steps, args.warmup, sample_clocks=True)
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    us_step = ms * 1e3 / args.steps                      # one step = one layer on every rank
+    value = us_step / world                              # whole job: `world` layers per step time
+
+    # end to end from host buffers through the public Python call
+    n_e2e = min(args.steps, 300)
+    xh = torch.from_numpy(wl.x).pin_memory()
+    yh = torch.empty((1, lay.M), dtype=torch.float32).pin_memory()
+    xd = torch.empty_like(x)
+    for i in range(5 + n_e2e):
+        if i == 5:
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+        xd.copy_(xh, non_blocking=True)
+        pb.pp_forward(reps[i % len(reps)], xd, lay.act, out=y)
+        yh.copy_(y, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+    e2e_us = (time.perf_counter() - t0) / n_e2e * 1e6
+    if world > 1:
+        t = torch.tensor([e2e_us], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_us = float(t.item())
+
+    pk = pb.Packed(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values, lay.bias)
+    abytes = algorithmic_bytes(lay, 1, pk.n_tile_col)
+    peak, peak_kind = measured_peak_gbs()
+    achieved = abytes / (us_step * 1e-6) / 1e9
+    out = {
+        "metric": METRIC, "value": value, "unit": "us", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": us_step / 1e3, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f16 weights, f32 accumulate", "data": "synthetic",
+        "config": {"workload": wl.name, "batch": 1, "M": lay.M, "N": lay.N, "B": lay.B,
+                   "tiles_per_block_row": args.k, "density": args.k / 128, "launch": "cuda_graph",
+                   "l2": f"inputs larger than L2: calls rotate over {len(reps)} independent copies of the "
+                         f"layer ({len(reps) * lay.T * lay.B * lay.B * 2 / 2**20:.0f} MiB of weights)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "gpu_launches": args.steps,
+        "e2e": {"value": e2e_us / world, "unit": "us", "h2d_bytes_per_step": int(wl.x.nbytes),
+                "d2h_bytes_per_step": int(lay.M * 4), "steps": n_e2e},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                     "algorithmic_bytes_per_launch": abytes, "kernel": "gemv_f16_kernel<64,1>", "traffic": None},
+        "clocks": clocks,
+    }
+
+    if rank == 0 and not args.no_sweep and world == 1:
+        sweep = {}
+        base = None
+        for k in (128, 64, 32, 16, 8):
+            if k == args.k:
+                us_k = us_step
+                lay_k, n_tc = lay, pk.n_tile_col
+            else:
+                for r in reps:
+                    r.close()
+                wl_k, lay_k, reps, _, _, ms_k, _ = time_config(k, min(args.steps, 5000), min(args.warmup, 50))
+                us_k = ms_k * 1e3 / min(args.steps, 5000)
+                pkk = pb.Packed(lay_k.M, lay_k.N, lay_k.B, lay_k.row_perm, lay_k.col_perm, lay_k.tile_list,
+                                lay_k.tile_values, None)
+                n_tc = pkk.n_tile_col
+            gbs = algorithmic_bytes(lay_k, 1, n_tc) / (us_k * 1e-6) / 1e9
+            if k == 128:
+                base = us_k
+            sweep[f"{k / 128:.4g}"] = {"us": round(us_k, 3), "GBps": round(gbs, 1),
+                                       "speedup_vs_dense": None if base is None else round(base / us_k, 3),
+                                       "linearity": None if base is None else round(base / us_k * k / 128, 3)}
+        out["density_sweep"] = sweep
+
+    if rank == 0 and world == 1 and not args.no_cpu:
+        wl0 = synth.config5(k=args.k, batch=1)
+        out["cpu_baseline"] = cpu_baseline(wl0.layers[0], wl0.x)
+
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,170 @@
+/*
+ * pp.h -- C interface of the pivoted (PBP) fully-connected inference library
+ * for NVIDIA B200 (sm_100a).
+ *
+ * A layer computes  y = act(W x + b)  where the pruned matrix is in the
+ * permutation-block-permutation form of Eq. 1,
+ *
+ *        W = P_row * W_piv * P_col ,
+ *
+ * W_piv holding only dense B x B tiles.  Evaluation follows Eq. 2 / Listing 1:
+ * gather x through the column index array, multiply the kept tiles, scatter
+ * through the row index array -- all inside one kernel per layer.
+ *
+ * Index arrays (Section 4.1.4): both map a PIVOTED index to an ORIGINAL index,
+ *        x_piv[j] = x[col_perm[j]]          (gather, Listing 1 step 4)
+ *        y[row_perm[i]] = y_piv[i]          (scatter, Listing 1 step 9)
+ * so W[row_perm[i]][col_perm[j]] = W_piv[i][j].  Sizes that are not multiples
+ * of B are padded in pivoted space: Mb = ceil(M/B), M_pad = Mb*B (same for N);
+ * row_perm / col_perm are bijections on [0,M_pad) / [0,N_pad); pivoted rows
+ * with row_perm[i] >= M are never stored and pivoted columns with
+ * col_perm[j] >= N read x as 0.
+ *
+ * Pointer kinds: "host" = ordinary CPU memory, "device" = memory of the
+ * current CUDA device.  All *_create calls copy what they are given; the caller
+ * keeps ownership of its arrays.  Handles own their device memory until the
+ * matching *_destroy.  The forward calls only ENQUEUE work on the given stream:
+ * they never synchronise and never allocate.  Calls that use the same handle
+ * must be ordered on one stream (a handle owns scratch memory that concurrent
+ * calls would share).  Every failure is a return code; nothing aborts or traps.
+ * There is no CPU fallback.
+ */
+#ifndef PP_H_
+#define PP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pp_layer pp_layer_t;
+typedef struct pp_chain pp_chain_t;
+typedef struct pp_packed pp_packed_t;
+
+typedef enum {
+    PP_OK = 0,
+    PP_ERR_INVALID_ARG = 1, /* NULL pointer, non-positive size, misaligned device pointer, batch < 1 */
+    PP_ERR_BAD_PERM = 2,    /* row_perm / col_perm is not a bijection on its padded range */
+    PP_ERR_BAD_TILE = 3,    /* tile outside the Mb x Nb grid, or listed twice */
+    PP_ERR_ALLOC = 4,       /* host or device allocation failed */
+    PP_ERR_CUDA = 5,        /* a CUDA runtime call failed (no device, launch error, ...) */
+    PP_ERR_UNSUPPORTED = 6, /* tile size / dtype / batch combination not implemented */
+    PP_ERR_TIMEOUT = 7      /* a bounded device-side wait gave up (status word set by the kernel) */
+} pp_status_t;
+
+typedef enum { PP_F32 = 0, PP_F16 = 1 } pp_dtype_t;
+typedef enum { PP_ACT_IDENTITY = 0, PP_ACT_RELU = 1 } pp_act_t;
+
+const char* pp_status_string(pp_status_t s);
+
+/* ------------------------------------------------------------------------- *
+ * Host-side packer ("network implementation time", Sections 2 and 4.1.1: the
+ * blocks may be ordered arbitrarily and mapped to the physical layout that
+ * suits the architecture).  Validates the layer, sorts the kept tiles by
+ * (block-row, block-col) and builds the block-row-compressed layout the
+ * kernels read:
+ *   - row_ptr[Mb+1]: first kept tile of each block-row (tile units);
+ *   - col_ptr[Mb+1] / tile_col[]: per-block-row tile-column index arrays, each
+ *     padded with -1 to a multiple of 4 entries (16 bytes);
+ *   - values: kept tiles of a block-row contiguous, re-ordered into 512-byte
+ *     "fragments" so that one 128-bit load per lane of a warp is fully
+ *     coalesced (fp32: lane = row, 4 consecutive columns; fp16: the register
+ *     layout of a 16x16 matrix-multiply operand);
+ *   - gather_idx[N_pad] = col_perm with entries >= N replaced by -1,
+ *     scatter_idx[M_pad] = row_perm with entries >= M replaced by -1,
+ *     bias_piv[M_pad] = bias[row_perm[i]] (0 for padded rows or bias == NULL);
+ *   - a work list cutting each block-row into parts of a few tiles.
+ * Host only; needs no GPU.
+ *
+ * M, N          logical output / input sizes (> 0)
+ * B             tile edge: 16, 32 or 64 (others: PP_ERR_UNSUPPORTED)
+ * row_perm      host, int32[M_pad]     col_perm   host, int32[N_pad]
+ * tile_list     host, int32[T][2] = (block_row, block_col), any order
+ * tile_values   host, [T][B][B] row-major inside a tile, W_piv coordinates,
+ *               element type wdtype (PP_F32: float, PP_F16: IEEE binary16 bits)
+ * bias          host, float[M] in ORIGINAL row order, or NULL
+ * ------------------------------------------------------------------------- */
+pp_status_t pp_pack_create(pp_packed_t** out, int M, int N, int B,
+                           const int32_t* row_perm, const int32_t* col_perm,
+                           const int32_t* tile_list, int64_t T,
+                           const void* tile_values, pp_dtype_t wdtype,
+                           const float* bias);
+pp_status_t pp_pack_destroy(pp_packed_t* p);
+
+/* Sizes of the packed arrays: out[0]=Mb, [1]=Nb, [2]=T, [3]=length of tile_col
+ * (padded), [4]=number of work items, [5]=bytes of packed values,
+ * [6]=max tiles in one work item, [7]=number of partial-sum slots. */
+pp_status_t pp_pack_info(const pp_packed_t* p, int64_t out[8]);
+
+/* Copy one packed array to host memory `dst` of capacity `bytes`.
+ * which: 0 row_ptr(int32[Mb+1]) 1 col_ptr(int32[Mb+1]) 2 tile_col(int32[])
+ *        3 gather_idx(int32[N_pad]) 4 scatter_idx(int32[M_pad]) 5 bias_piv(float[M_pad])
+ *        6 values (bytes) 7 work items (int32[n_items][8]) 8 inv_row_perm(int32[M_pad]) */
+pp_status_t pp_pack_get(const pp_packed_t* p, int which, void* dst, int64_t bytes);
+
+/* Inverse of the value re-ordering: writes the sorted tile list (int32[T][2])
+ * and the tiles in their original row-major form ([T][B][B], wdtype). */
+pp_status_t pp_pack_unpack(const pp_packed_t* p, int32_t* tile_list_out, void* tile_values_out);
+
+/* Cross-layer permutation fusion (Section 4.2.1): the row permutation of layer
+ * A followed by the column permutation of the next layer B is one static
+ * permutation.  q[j] = position, in A's pivoted output, of the value that B's
+ * pivoted column j reads:  q[j] = inv_row_perm_A[col_perm_B[j]], or -1 when
+ * col_perm_B[j] >= N_B (padding).  Requires N_B == M_A.  Host only.
+ * row_perm_A: int32[M_pad_A]; col_perm_B: int32[N_pad_B]; q_out: int32[N_pad_B]. */
+pp_status_t pp_fold_perm(const int32_t* row_perm_A, int M_A, int M_pad_A,
+                         const int32_t* col_perm_B, int N_B, int N_pad_B,
+                         int32_t* q_out);
+
+/* ------------------------------------------------------------------------- *
+ * Layer: pack (as above) and upload to the current CUDA device.
+ * Same arguments as pp_pack_create.  Errors: as pp_pack_create, plus
+ * PP_ERR_CUDA / PP_ERR_ALLOC when no device is usable or memory runs out.
+ * ------------------------------------------------------------------------- */
+pp_status_t pp_layer_create(pp_layer_t** out, int M, int N, int B,
+                            const int32_t* row_perm, const int32_t* col_perm,
+                            const int32_t* tile_list, int64_t T,
+                            const void* tile_values, pp_dtype_t wdtype,
+                            const float* bias);
+pp_status_t pp_layer_destroy(pp_layer_t* layer);
+
+/* Independent device copy of a layer (own weights, index arrays and scratch), e.g. to
+ * serve several streams at once or to rotate copies so that repeated timing runs do not
+ * find the weights in L2.  Errors: PP_ERR_INVALID_ARG, PP_ERR_ALLOC, PP_ERR_CUDA. */
+pp_status_t pp_layer_clone(pp_layer_t** out, const pp_layer_t* src);
+
+/* y = act(W x + b) (Eq. 2, Listing 1 with both permutations).
+ * x   device, [batch][N] row-major, element type = the layer's wdtype, 16-byte aligned
+ * y   device, [batch][M] row-major, float, must not alias x
+ * batch >= 1.  batch < 64 (and every fp32 layer) runs the streaming
+ * matrix-vector kernel in groups of up to 32 columns; fp16 layers with B = 64
+ * and batch >= 64 run the tensor-core tile kernel.
+ * cuda_stream: a cudaStream_t (NULL = default stream).  Enqueues only. */
+pp_status_t pp_forward(pp_layer_t* layer, const void* x, void* y, int batch,
+                       pp_act_t act, void* cuda_stream);
+
+/* ------------------------------------------------------------------------- *
+ * Chain of layers with folded permutations (Section 4.2.1): between two
+ * consecutive layers the activations stay in the producer's pivoted order and
+ * the consumer gathers through the folded map q (pp_fold_perm); only the first
+ * gather and the last scatter touch original order.  Layer l's output feeds
+ * layer l+1 rounded (to nearest even) to layer l+1's element type.
+ * layers[l+1].N must equal layers[l].M.  The chain references its layers: they
+ * must outlive it.  Intermediate buffers are sized for max_batch at create.
+ * x: device [batch][N_0] (dtype of layer 0); y: device float [batch][M_last]. */
+pp_status_t pp_chain_create(pp_chain_t** out, pp_layer_t* const* layers,
+                            const pp_act_t* acts, int n_layers, int max_batch);
+pp_status_t pp_chain_destroy(pp_chain_t* chain);
+pp_status_t pp_chain_forward(pp_chain_t* chain, const void* x, void* y, int batch,
+                             void* cuda_stream);
+
+/* Tuning knobs read at pack / create time (process-wide; for experiments).
+ * key 0: target kilobytes of tile values per work item (default 32)
+ * key 1: lower bound on the number of work items the splitter aims for (default 296) */
+pp_status_t pp_set_tuning(int key, int value);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PP_H_ */

@@ -1,0 +1,285 @@
+"""Python binding of libpp_b200.so: argument marshalling only.
+
+Function names mirror the C interface (``include/pp.h``).  Device buffers are
+PyTorch CUDA tensors; the binding passes their ``data_ptr()`` and the current
+stream's handle.  Nothing here computes: if the compiled library is missing the
+import fails with an error that says how to build it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpp_b200.so")
+
+PP_OK = 0
+PP_F32, PP_F16 = 0, 1
+PP_ACT_IDENTITY, PP_ACT_RELU = 0, 1
+
+STATUS_NAMES = {0: "PP_OK", 1: "PP_ERR_INVALID_ARG", 2: "PP_ERR_BAD_PERM", 3: "PP_ERR_BAD_TILE",
+                4: "PP_ERR_ALLOC", 5: "PP_ERR_CUDA", 6: "PP_ERR_UNSUPPORTED", 7: "PP_ERR_TIMEOUT"}
+
+
+class PPError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().pp_status_string(status).decode() if _lib is not None else ""
+        super().__init__(f"{where}: {STATUS_NAMES.get(status, status)} ({msg})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the C library (once).  No fallback: a missing library is an error."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} not found: build it with "
+                          f"`python -m paper_1712_01084_b200.build` (needs nvcc, targets sm_100a)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32p, i64p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)
+    ci, c64 = ctypes.c_int, ctypes.c_int64
+    fp = ctypes.POINTER(ctypes.c_float)
+    create_args = [ctypes.POINTER(vp), ci, ci, ci, i32p, i32p, i32p, c64, vp, ci, fp]
+    sig = {
+        "pp_status_string": (ctypes.c_char_p, [ci]),
+        "pp_pack_create": (ci, create_args),
+        "pp_pack_destroy": (ci, [vp]),
+        "pp_pack_info": (ci, [vp, i64p]),
+        "pp_pack_get": (ci, [vp, ci, vp, c64]),
+        "pp_pack_unpack": (ci, [vp, i32p, vp]),
+        "pp_fold_perm": (ci, [i32p, ci, ci, i32p, ci, ci, i32p]),
+        "pp_layer_create": (ci, create_args),
+        "pp_layer_destroy": (ci, [vp]),
+        "pp_layer_clone": (ci, [ctypes.POINTER(vp), vp]),
+        "pp_forward": (ci, [vp, vp, vp, ci, ci, vp]),
+        "pp_chain_create": (ci, [ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(ci), ci, ci]),
+        "pp_chain_destroy": (ci, [vp]),
+        "pp_chain_forward": (ci, [vp, vp, vp, ci, vp]),
+        "pp_set_tuning": (ci, [ci, ci]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(L, name)
+        fn.restype, fn.argtypes = res, args
+    _lib = L
+    return L
+
+
+def _check(st: int, where: str):
+    if st != PP_OK:
+        raise PPError(st, where)
+
+
+def _i32(a):
+    a = np.ascontiguousarray(a, dtype=np.int32)
+    return a, a.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+
+
+def _layer_args(M, N, B, row_perm, col_perm, tile_list, tile_values, bias):
+    rp, rpp = _i32(row_perm)
+    cp, cpp = _i32(col_perm)
+    tl, tlp = _i32(np.asarray(tile_list).reshape(-1, 2))
+    tv = np.ascontiguousarray(tile_values)
+    if tv.dtype == np.float16:
+        wd = PP_F16
+    elif tv.dtype == np.float32:
+        wd = PP_F32
+    else:
+        raise TypeError("tile_values must be float32 or float16")
+    T = tl.shape[0]
+    if tv.size != T * B * B:
+        raise ValueError("tile_values must hold T*B*B elements")
+    if rp.size != -(-M // B) * B or cp.size != -(-N // B) * B:
+        raise ValueError("row_perm/col_perm must cover the padded ranges")
+    b = None if bias is None else np.ascontiguousarray(bias, dtype=np.float32)
+    if b is not None and b.size != M:
+        raise ValueError("bias must have M entries")
+    bp = None if b is None else b.ctypes.data_as(ctypes.POINTER(ctypes.c_float))
+    keep = (rp, cp, tl, tv, b)
+    return keep, (int(M), int(N), int(B), rpp, cpp, tlp, T, tv.ctypes.data_as(ctypes.c_void_p), wd, bp)
+
+
+# ---------------------------------------------------------------- host packer
+class Packed:
+    """Host-side packed layer (pp_pack_create); needs no GPU."""
+
+    def __init__(self, M, N, B, row_perm, col_perm, tile_list, tile_values, bias=None):
+        keep, args = _layer_args(M, N, B, row_perm, col_perm, tile_list, tile_values, bias)
+        self._h = ctypes.c_void_p()
+        _check(lib().pp_pack_create(ctypes.byref(self._h), *args), "pp_pack_create")
+        self.M, self.N, self.B = int(M), int(N), int(B)
+        self.wdtype = np.asarray(tile_values).dtype
+        info = (ctypes.c_int64 * 8)()
+        _check(lib().pp_pack_info(self._h, info), "pp_pack_info")
+        (self.Mb, self.Nb, self.T, self.n_tile_col, self.n_items, self.value_bytes,
+         self.max_item_tiles, self.n_slots) = [int(v) for v in info]
+
+    def get(self, which: str) -> np.ndarray:
+        Mpad, Npad = self.Mb * self.B, self.Nb * self.B
+        spec = {"row_ptr": (0, np.int32, self.Mb + 1), "col_ptr": (1, np.int32, self.Mb + 1),
+                "tile_col": (2, np.int32, self.n_tile_col), "gather_idx": (3, np.int32, Npad),
+                "scatter_idx": (4, np.int32, Mpad), "bias_piv": (5, np.float32, Mpad),
+                "values": (6, np.uint8, self.value_bytes), "items": (7, np.int32, self.n_items * 8),
+                "inv_row_perm": (8, np.int32, Mpad)}[which]
+        out = np.empty(spec[2], dtype=spec[1])
+        _check(lib().pp_pack_get(self._h, spec[0], out.ctypes.data_as(ctypes.c_void_p), out.nbytes), "pp_pack_get")
+        return out.reshape(-1, 8) if which == "items" else out
+
+    def unpack(self):
+        tl = np.empty((self.T, 2), dtype=np.int32)
+        tv = np.empty((self.T, self.B, self.B), dtype=self.wdtype)
+        _check(lib().pp_pack_unpack(self._h, tl.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                                    tv.ctypes.data_as(ctypes.c_void_p)), "pp_pack_unpack")
+        return tl, tv
+
+    def close(self):
+        if self._h:
+            lib().pp_pack_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def pp_fold_perm(row_perm_A, M_A: int, col_perm_B, N_B: int) -> np.ndarray:
+    ra, rap = _i32(row_perm_A)
+    cb, cbp = _i32(col_perm_B)
+    q = np.empty(cb.size, dtype=np.int32)
+    _check(lib().pp_fold_perm(rap, int(M_A), ra.size, cbp, int(N_B), cb.size,
+                              q.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))), "pp_fold_perm")
+    return q
+
+
+def pp_set_tuning(key: int, value: int):
+    _check(lib().pp_set_tuning(int(key), int(value)), "pp_set_tuning")
+
+
+# ------------------------------------------------------------------ device API
+def _stream_ptr(stream=None):
+    import torch
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _require_cuda(t, name):
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA tensor")
+
+
+class Layer:
+    """Device-resident pivoted FC layer (pp_layer_create / pp_forward)."""
+
+    def __init__(self, M, N, B, row_perm, col_perm, tile_list, tile_values, bias=None):
+        keep, args = _layer_args(M, N, B, row_perm, col_perm, tile_list, tile_values, bias)
+        self._h = ctypes.c_void_p()
+        _check(lib().pp_layer_create(ctypes.byref(self._h), *args), "pp_layer_create")
+        self.M, self.N, self.B = int(M), int(N), int(B)
+        self.wdtype = np.asarray(tile_values).dtype
+
+    @classmethod
+    def from_synth(cls, lay):
+        return cls(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values, lay.bias)
+
+    def clone(self) -> "Layer":
+        other = object.__new__(Layer)
+        other._h = ctypes.c_void_p()
+        _check(lib().pp_layer_clone(ctypes.byref(other._h), self._h), "pp_layer_clone")
+        other.M, other.N, other.B, other.wdtype = self.M, self.N, self.B, self.wdtype
+        return other
+
+    def forward(self, x, act: int = PP_ACT_IDENTITY, out=None, stream=None):
+        return pp_forward(self, x, act, out=out, stream=stream)
+
+    def close(self):
+        if self._h:
+            lib().pp_layer_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def pp_layer_create(M, N, B, row_perm, col_perm, tile_list, tile_values, bias=None) -> Layer:
+    return Layer(M, N, B, row_perm, col_perm, tile_list, tile_values, bias)
+
+
+def _check_x(x, N, wdtype):
+    import torch
+    _require_cuda(x, "x")
+    want = torch.float16 if wdtype == np.float16 else torch.float32
+    if x.dtype != want:
+        raise TypeError(f"x must be {want}")
+    if x.dim() == 1:
+        x = x.unsqueeze(0)
+    if x.shape[-1] != N:
+        raise ValueError(f"x must be [batch][{N}]")
+    return x
+
+
+def pp_forward(layer: Layer, x, act: int = PP_ACT_IDENTITY, out=None, stream=None):
+    """y[batch][M] (float32, CUDA) = act(W x + b).  Enqueues on the current stream."""
+    import torch
+    x2 = _check_x(x, layer.N, layer.wdtype)
+    batch = x2.shape[0]
+    y = torch.empty((batch, layer.M), dtype=torch.float32, device=x.device) if out is None else out
+    _require_cuda(y, "out")
+    if y.dtype != torch.float32 or y.numel() != batch * layer.M:
+        raise ValueError("out must be float32 [batch][M]")
+    _check(lib().pp_forward(layer._h, ctypes.c_void_p(x2.data_ptr()), ctypes.c_void_p(y.data_ptr()),
+                            batch, int(act), _stream_ptr(stream)), "pp_forward")
+    return y
+
+
+class Chain:
+    """Stack of layers with folded permutations (pp_chain_create / pp_chain_forward)."""
+
+    def __init__(self, layers: Sequence[Layer], acts: Sequence[int], max_batch: int = 8):
+        self.layers = list(layers)          # keep the layers alive
+        n = len(self.layers)
+        arr = (ctypes.c_void_p * n)(*[l._h for l in self.layers])
+        acts_arr = (ctypes.c_int * n)(*[int(a) for a in acts])
+        self._h = ctypes.c_void_p()
+        _check(lib().pp_chain_create(ctypes.byref(self._h), arr, acts_arr, n, int(max_batch)), "pp_chain_create")
+        self.max_batch = int(max_batch)
+
+    def forward(self, x, out=None, stream=None):
+        return pp_chain_forward(self, x, out=out, stream=stream)
+
+    def close(self):
+        if self._h:
+            lib().pp_chain_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def pp_chain_create(layers, acts, max_batch: int = 8) -> Chain:
+    return Chain(layers, acts, max_batch)
+
+
+def pp_chain_forward(chain: Chain, x, out=None, stream=None):
+    import torch
+    first, last = chain.layers[0], chain.layers[-1]
+    x2 = _check_x(x, first.N, first.wdtype)
+    batch = x2.shape[0]
+    y = torch.empty((batch, last.M), dtype=torch.float32, device=x.device) if out is None else out
+    _require_cuda(y, "out")
+    _check(lib().pp_chain_forward(chain._h, ctypes.c_void_p(x2.data_ptr()), ctypes.c_void_p(y.data_ptr()),
+                                  batch, _stream_ptr(stream)), "pp_chain_forward")
+    return y

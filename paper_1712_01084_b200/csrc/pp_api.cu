@@ -1,0 +1,238 @@
+// C entry points that own device memory: layers, forward calls, folded chains.
+#include <cuda_runtime.h>
+
+#include <new>
+#include <vector>
+
+#include "pp_gemv.cuh"
+#include "pp_internal.h"
+
+struct pp_layer {
+    pp_packed* pk = nullptr;       // host copy (index arrays are needed again when chains are folded)
+    void* d_values = nullptr;
+    pp::WorkItem* d_items = nullptr;
+    int32_t* d_tile_col = nullptr;
+    int32_t* d_gather = nullptr;
+    int32_t* d_scatter = nullptr;
+    float* d_bias = nullptr;
+    float* d_partials = nullptr;
+    int* d_counters = nullptr;
+    int n_items = 0;
+    int max_item_tiles = 0;
+};
+
+struct pp_chain {
+    std::vector<pp_layer*> layers;
+    std::vector<pp_act_t> acts;
+    std::vector<int32_t*> d_q;     // folded gather map of layer l (l >= 1); entry 0 unused
+    std::vector<void*> d_inter;    // output of layer l in pivoted order, element type of layer l+1
+    int max_batch = 0;
+};
+
+namespace {
+
+template <typename T>
+bool upload(T** dst, const void* src, size_t bytes) {
+    *dst = nullptr;
+    if (cudaMalloc(reinterpret_cast<void**>(dst), bytes ? bytes : 16) != cudaSuccess) return false;
+    if (bytes && cudaMemcpy(*dst, src, bytes, cudaMemcpyHostToDevice) != cudaSuccess) return false;
+    return true;
+}
+
+void free_layer(pp_layer* L) {
+    if (!L) return;
+    cudaFree(L->d_values); cudaFree(L->d_items); cudaFree(L->d_tile_col); cudaFree(L->d_gather);
+    cudaFree(L->d_scatter); cudaFree(L->d_bias); cudaFree(L->d_partials); cudaFree(L->d_counters);
+    pp_pack_destroy(L->pk);
+    delete L;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Enqueue one layer in groups of batch columns.
+pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_elt, void* y, int ldy,
+                      int out_mode, int batch, pp_act_t act, cudaStream_t stream) {
+    const pp_packed* pk = L->pk;
+    pp::GemvArgs a{};
+    a.values = L->d_values; a.items = L->d_items; a.tile_col = L->d_tile_col;
+    a.gather_idx = gather; a.scatter_idx = L->d_scatter; a.bias_piv = L->d_bias;
+    a.partials = L->d_partials; a.counters = L->d_counters;
+    a.ldx = ldx; a.ldy = ldy; a.x_limit = pk->N; a.act = (int)act; a.out_mode = out_mode;
+    const int group = pp::gemv_group_batch(pk->wdtype);
+    const int y_elt = out_mode == pp::OUT_PIVOTED_F16 ? 2 : 4;
+    for (int b0 = 0; b0 < batch; b0 += group) {
+        a.batch = batch - b0 < group ? batch - b0 : group;
+        a.x = static_cast<const char*>(x) + (size_t)b0 * ldx * x_elt;
+        a.y = static_cast<char*>(y) + (size_t)b0 * ldy * y_elt;
+        if (pp::launch_gemv(pk->wdtype, pk->B, a, L->n_items, L->max_item_tiles, stream) != cudaSuccess)
+            return PP_ERR_CUDA;
+    }
+    return PP_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+pp_status_t pp_layer_create(pp_layer_t** out, int M, int N, int B, const int32_t* row_perm,
+                            const int32_t* col_perm, const int32_t* tile_list, int64_t T,
+                            const void* tile_values, pp_dtype_t wdtype, const float* bias) {
+    if (!out) return PP_ERR_INVALID_ARG;
+    *out = nullptr;
+    pp_packed* pk = nullptr;
+    pp_status_t st = pp_pack_create(&pk, M, N, B, row_perm, col_perm, tile_list, T, tile_values, wdtype, bias);
+    if (st != PP_OK) return st;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { pp_pack_destroy(pk); cudaGetLastError(); return PP_ERR_CUDA; }
+    pp_layer* L = new (std::nothrow) pp_layer();
+    if (!L) { pp_pack_destroy(pk); return PP_ERR_ALLOC; }
+    L->pk = pk;
+    L->n_items = (int)pk->items.size();
+    L->max_item_tiles = pk->max_item_tiles;
+    bool ok = upload(&L->d_values, pk->values.data(), pk->values.size()) &&
+              upload(&L->d_items, pk->items.data(), pk->items.size() * sizeof(pp::WorkItem)) &&
+              upload(&L->d_tile_col, pk->tile_col.data(), pk->tile_col.size() * 4) &&
+              upload(&L->d_gather, pk->gather_idx.data(), pk->gather_idx.size() * 4) &&
+              upload(&L->d_scatter, pk->scatter_idx.data(), pk->scatter_idx.size() * 4) &&
+              upload(&L->d_bias, pk->bias_piv.data(), pk->bias_piv.size() * 4);
+    if (ok) {
+        const size_t pbytes = (size_t)pk->n_slots * B * pp::kMaxGroupBatch * sizeof(float);
+        ok = cudaMalloc(reinterpret_cast<void**>(&L->d_partials), pbytes ? pbytes : 16) == cudaSuccess &&
+             cudaMalloc(reinterpret_cast<void**>(&L->d_counters), (size_t)pk->Mb * sizeof(int)) == cudaSuccess &&
+             cudaMemset(L->d_counters, 0, (size_t)pk->Mb * sizeof(int)) == cudaSuccess;
+    }
+    if (!ok) {
+        const cudaError_t e = cudaGetLastError();
+        free_layer(L);
+        return e == cudaErrorMemoryAllocation ? PP_ERR_ALLOC : PP_ERR_CUDA;
+    }
+    // the fragment-ordered values now live on the device; drop the host copy
+    std::vector<unsigned char>().swap(pk->values);
+    *out = L;
+    return PP_OK;
+}
+
+pp_status_t pp_layer_clone(pp_layer_t** out, const pp_layer_t* src) {
+    if (!out) return PP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!src) return PP_ERR_INVALID_ARG;
+    pp_layer* L = new (std::nothrow) pp_layer();
+    pp_packed* pk = new (std::nothrow) pp_packed(*src->pk);
+    if (!L || !pk) { delete L; delete pk; return PP_ERR_ALLOC; }
+    L->pk = pk;
+    L->n_items = src->n_items;
+    L->max_item_tiles = src->max_item_tiles;
+    const size_t esz = pk->wdtype == PP_F16 ? 2 : 4;
+    const size_t vbytes = (size_t)pk->T * pk->B * pk->B * esz;
+    const size_t pbytes = (size_t)pk->n_slots * pk->B * pp::kMaxGroupBatch * sizeof(float);
+    auto dup = [](auto** dst, const void* s, size_t bytes) {
+        *dst = nullptr;
+        if (cudaMalloc(reinterpret_cast<void**>(dst), bytes ? bytes : 16) != cudaSuccess) return false;
+        return bytes == 0 || cudaMemcpy(*dst, s, bytes, cudaMemcpyDeviceToDevice) == cudaSuccess;
+    };
+    bool ok = dup(&L->d_values, src->d_values, vbytes) &&
+              dup(&L->d_items, src->d_items, pk->items.size() * sizeof(pp::WorkItem)) &&
+              dup(&L->d_tile_col, src->d_tile_col, pk->tile_col.size() * 4) &&
+              dup(&L->d_gather, src->d_gather, pk->gather_idx.size() * 4) &&
+              dup(&L->d_scatter, src->d_scatter, pk->scatter_idx.size() * 4) &&
+              dup(&L->d_bias, src->d_bias, pk->bias_piv.size() * 4) &&
+              cudaMalloc(reinterpret_cast<void**>(&L->d_partials), pbytes ? pbytes : 16) == cudaSuccess &&
+              cudaMalloc(reinterpret_cast<void**>(&L->d_counters), (size_t)pk->Mb * sizeof(int)) == cudaSuccess &&
+              cudaMemset(L->d_counters, 0, (size_t)pk->Mb * sizeof(int)) == cudaSuccess;
+    if (!ok) {
+        const cudaError_t e = cudaGetLastError();
+        free_layer(L);
+        return e == cudaErrorMemoryAllocation ? PP_ERR_ALLOC : PP_ERR_CUDA;
+    }
+    *out = L;
+    return PP_OK;
+}
+
+pp_status_t pp_layer_destroy(pp_layer_t* layer) {
+    free_layer(layer);
+    return PP_OK;
+}
+
+pp_status_t pp_forward(pp_layer_t* L, const void* x, void* y, int batch, pp_act_t act, void* cuda_stream) {
+    if (!L || !x || !y || batch < 1 || x == y) return PP_ERR_INVALID_ARG;
+    if (act != PP_ACT_IDENTITY && act != PP_ACT_RELU) return PP_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y)) return PP_ERR_INVALID_ARG;
+    const pp_packed* pk = L->pk;
+    return run_layer(L, L->d_gather, x, pk->N, pk->wdtype == PP_F16 ? 2 : 4, y, pk->M, pp::OUT_SCATTER_F32,
+                     batch, act, static_cast<cudaStream_t>(cuda_stream));
+}
+
+pp_status_t pp_chain_create(pp_chain_t** out, pp_layer_t* const* layers, const pp_act_t* acts, int n_layers,
+                            int max_batch) {
+    if (!out) return PP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!layers || !acts || n_layers < 1 || max_batch < 1) return PP_ERR_INVALID_ARG;
+    for (int l = 0; l < n_layers; ++l) {
+        if (!layers[l]) return PP_ERR_INVALID_ARG;
+        if (acts[l] != PP_ACT_IDENTITY && acts[l] != PP_ACT_RELU) return PP_ERR_INVALID_ARG;
+        if (l > 0 && layers[l]->pk->N != layers[l - 1]->pk->M) return PP_ERR_INVALID_ARG;
+    }
+    pp_chain* C = new (std::nothrow) pp_chain();
+    if (!C) return PP_ERR_ALLOC;
+    C->layers.assign(layers, layers + n_layers);
+    C->acts.assign(acts, acts + n_layers);
+    C->max_batch = max_batch;
+    C->d_q.assign((size_t)n_layers, nullptr);
+    C->d_inter.assign((size_t)n_layers, nullptr);
+    bool ok = true;
+    pp_status_t st = PP_OK;
+    for (int l = 1; l < n_layers && ok; ++l) {
+        const pp_packed* A = layers[l - 1]->pk;
+        const pp_packed* Bk = layers[l]->pk;
+        std::vector<int32_t> q((size_t)Bk->Npad);
+        st = pp_fold_perm(A->row_perm.data(), A->M, A->Mpad, Bk->col_perm.data(), Bk->N, Bk->Npad, q.data());
+        if (st != PP_OK) { ok = false; break; }
+        ok = upload(&C->d_q[(size_t)l], q.data(), q.size() * 4);
+        const size_t elt = Bk->wdtype == PP_F16 ? 2 : 4;
+        ok = ok && cudaMalloc(&C->d_inter[(size_t)l - 1], (size_t)max_batch * A->Mpad * elt) == cudaSuccess;
+        if (!ok) st = PP_ERR_ALLOC;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        pp_chain_destroy(C);
+        return st;
+    }
+    *out = C;
+    return PP_OK;
+}
+
+pp_status_t pp_chain_destroy(pp_chain_t* C) {
+    if (!C) return PP_OK;
+    for (int32_t* q : C->d_q) cudaFree(q);
+    for (void* b : C->d_inter) cudaFree(b);
+    delete C;
+    return PP_OK;
+}
+
+pp_status_t pp_chain_forward(pp_chain_t* C, const void* x, void* y, int batch, void* cuda_stream) {
+    if (!C || !x || !y || batch < 1 || batch > C->max_batch || x == y) return PP_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y)) return PP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int n = (int)C->layers.size();
+    const void* cur = x;
+    for (int l = 0; l < n; ++l) {
+        pp_layer* L = C->layers[(size_t)l];
+        const pp_packed* pk = L->pk;
+        const int x_elt = pk->wdtype == PP_F16 ? 2 : 4;
+        const int32_t* gather = l == 0 ? L->d_gather : C->d_q[(size_t)l];
+        const int ldx = l == 0 ? pk->N : C->layers[(size_t)l - 1]->pk->Mpad;
+        pp_status_t st;
+        if (l == n - 1) {
+            st = run_layer(L, gather, cur, ldx, x_elt, y, pk->M, pp::OUT_SCATTER_F32, batch, C->acts[(size_t)l], stream);
+        } else {
+            const bool next_f16 = C->layers[(size_t)l + 1]->pk->wdtype == PP_F16;
+            st = run_layer(L, gather, cur, ldx, x_elt, C->d_inter[(size_t)l], pk->Mpad,
+                           next_f16 ? pp::OUT_PIVOTED_F16 : pp::OUT_PIVOTED_F32, batch, C->acts[(size_t)l], stream);
+            cur = C->d_inter[(size_t)l];
+        }
+        if (st != PP_OK) return st;
+    }
+    return PP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,59 @@
+// Internal structures shared by the host packer, the API layer and the kernels.
+#pragma once
+#include <cstdint>
+#include <vector>
+
+#include "pp.h"
+
+namespace pp {
+
+// One unit of kernel work: a run of consecutive kept tiles of one block-row.
+// The fragment indices are in 512-byte units into the packed value array.
+struct WorkItem {
+    int32_t frag_base;    // fragment of (row-group 0, first tile of the run, k-fragment 0)
+    int32_t rg_stride;    // fragments between consecutive row-groups of this block-row
+    int32_t nf;           // fragments per row-group in this run (= ntiles * frags_per_tile_row)
+    int32_t col_off;      // index into tile_col[] of the run's first tile
+    int32_t ntiles;       // tiles in the run (0 for a block-row without tiles)
+    int32_t br;           // block-row
+    int32_t part_nparts;  // part | (nparts << 16): position of this run among the block-row's runs
+    int32_t slot_base;    // first partial-sum slot of the block-row (valid when nparts > 1)
+};
+static_assert(sizeof(WorkItem) == 32, "WorkItem is read as two 16-byte words");
+
+constexpr int kMaxGroupBatch = 32;   // batch columns one streaming-kernel launch handles
+constexpr int kMaxRunColumns = 2048;  // pivoted columns (tiles x B) one work item may span
+
+// Geometry of the fragment layout for a (dtype, B) pair.
+struct FragGeom {
+    int rg_rows;   // rows covered by one fragment (row-group height)
+    int kf;        // columns covered by one fragment
+    int n_rg;      // row-groups per tile      = B / rg_rows
+    int fpt;       // fragments per tile per row-group = B / kf
+};
+inline FragGeom frag_geom(pp_dtype_t dt, int B) {
+    FragGeom g;
+    if (dt == PP_F16) { g.rg_rows = 16; g.kf = 16; }
+    else { g.rg_rows = B < 32 ? B : 32; g.kf = 128 / g.rg_rows; }
+    g.n_rg = B / g.rg_rows;
+    g.fpt = B / g.kf;
+    return g;
+}
+
+}  // namespace pp
+
+// Host-side result of packing one layer.
+struct pp_packed {
+    int M, N, B, Mb, Nb, Mpad, Npad;
+    int64_t T;
+    pp_dtype_t wdtype;
+    std::vector<int32_t> row_perm, col_perm, inv_row_perm;   // copies of the caller's arrays
+    std::vector<int32_t> row_ptr, col_ptr, tile_col;         // block-row-compressed index arrays
+    std::vector<int32_t> gather_idx, scatter_idx;
+    std::vector<float> bias_piv;
+    std::vector<unsigned char> values;                       // fragment-ordered tile values
+    std::vector<pp::WorkItem> items;
+    int max_item_tiles;
+    int n_slots;
+    bool has_bias;
+};

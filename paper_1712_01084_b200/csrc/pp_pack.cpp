@@ -1,0 +1,281 @@
+// Host-side pivot-format packer: validation, block-row-compressed index arrays,
+// fragment-ordered tile values, pivoted bias, work list, permutation folding.
+// Pure host code (no CUDA calls), so it can be exercised without a GPU.
+#include <algorithm>
+#include <cstring>
+#include <new>
+#include <numeric>
+
+#include "pp_internal.h"
+
+namespace {
+
+int g_target_kib = 32;     // tile-value kilobytes per work item
+int g_min_items = 296;     // the splitter keeps halving the run length until it has this many items
+
+bool is_bijection(const int32_t* p, int64_t n) {
+    std::vector<unsigned char> seen((size_t)n, 0);
+    for (int64_t k = 0; k < n; ++k) {
+        if (p[k] < 0 || p[k] >= n || seen[(size_t)p[k]]) return false;
+        seen[(size_t)p[k]] = 1;
+    }
+    return true;
+}
+
+// Byte offset, inside a 512-byte fragment, of tile element (r, c) relative to the
+// fragment's origin, plus which fragment (rg, f) it falls in.
+struct ElemPos { int rg, f, byte; };
+
+inline ElemPos elem_pos(pp_dtype_t dt, const pp::FragGeom& g, int r, int c) {
+    ElemPos e;
+    if (dt == PP_F16) {
+        // 16x16 operand fragment of the warp-level matrix-multiply instruction: lane = 4*(row%8) + (col%8)/2,
+        // element slot = (col%2) + 2*(row/8) + 4*(col/8)  -> 8 halves (16 bytes) per lane.
+        e.rg = r / 16; e.f = c / 16;
+        int rr = r % 16, cc = c % 16;
+        int lane = 4 * (rr % 8) + (cc % 8) / 2;
+        int slot = (cc % 2) + 2 * (rr / 8) + 4 * (cc / 8);
+        e.byte = lane * 16 + slot * 2;
+    } else {
+        // lane = row (and, for 16-row tiles, which half of the 8 columns); 4 consecutive columns per lane.
+        e.rg = r / g.rg_rows; e.f = c / g.kf;
+        int rr = r % g.rg_rows, cc = c % g.kf;
+        int lane = rr + g.rg_rows * (cc / 4);
+        e.byte = lane * 16 + (cc % 4) * 4;
+    }
+    return e;
+}
+
+void build_items(pp_packed* p) {
+    const pp::FragGeom g = pp::frag_geom(p->wdtype, p->B);
+    const int esz = p->wdtype == PP_F16 ? 2 : 4;
+    const int64_t tile_bytes = (int64_t)p->B * p->B * esz;
+    int64_t run = std::max<int64_t>(1, (int64_t)g_target_kib * 1024 / tile_bytes);
+    run = std::min<int64_t>(run, std::max(1, pp::kMaxRunColumns / p->B));   // staged x must fit shared memory
+    auto count_items = [&](int64_t r) {
+        int64_t n = 0;
+        for (int br = 0; br < p->Mb; ++br) {
+            int64_t k = p->row_ptr[br + 1] - p->row_ptr[br];
+            n += std::max<int64_t>(1, (k + r - 1) / r);
+        }
+        return n;
+    };
+    while (run > 1 && count_items(run) < g_min_items) run = (run + 1) / 2;
+
+    p->items.clear();
+    p->max_item_tiles = 0;
+    p->n_slots = 0;
+    const int frags_per_tile = g.n_rg * g.fpt;
+    for (int br = 0; br < p->Mb; ++br) {
+        const int k = p->row_ptr[br + 1] - p->row_ptr[br];
+        const int nparts = std::max<int>(1, (int)((k + run - 1) / run));
+        const int slot_base = nparts > 1 ? p->n_slots : 0;
+        if (nparts > 1) p->n_slots += nparts;
+        for (int part = 0; part < nparts; ++part) {
+            const int j0 = (int)((int64_t)k * part / nparts), j1 = (int)((int64_t)k * (part + 1) / nparts);
+            pp::WorkItem it;
+            it.frag_base = p->row_ptr[br] * frags_per_tile + j0 * g.fpt;
+            it.rg_stride = k * g.fpt;
+            it.nf = (j1 - j0) * g.fpt;
+            it.col_off = p->col_ptr[br] + j0;
+            it.ntiles = j1 - j0;
+            it.br = br;
+            it.part_nparts = part | (nparts << 16);
+            it.slot_base = slot_base;
+            p->items.push_back(it);
+            p->max_item_tiles = std::max(p->max_item_tiles, j1 - j0);
+        }
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* pp_status_string(pp_status_t s) {
+    switch (s) {
+        case PP_OK: return "ok";
+        case PP_ERR_INVALID_ARG: return "invalid argument";
+        case PP_ERR_BAD_PERM: return "row_perm/col_perm is not a permutation of its padded range";
+        case PP_ERR_BAD_TILE: return "tile out of range or listed twice";
+        case PP_ERR_ALLOC: return "allocation failed";
+        case PP_ERR_CUDA: return "CUDA runtime error";
+        case PP_ERR_UNSUPPORTED: return "unsupported tile size, dtype or batch";
+        case PP_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+pp_status_t pp_set_tuning(int key, int value) {
+    if (key == 0 && value >= 1) { g_target_kib = value; return PP_OK; }
+    if (key == 1 && value >= 0) { g_min_items = value; return PP_OK; }
+    return PP_ERR_INVALID_ARG;
+}
+
+pp_status_t pp_pack_create(pp_packed_t** out, int M, int N, int B, const int32_t* row_perm,
+                           const int32_t* col_perm, const int32_t* tile_list, int64_t T,
+                           const void* tile_values, pp_dtype_t wdtype, const float* bias) {
+    if (!out) return PP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (M <= 0 || N <= 0 || B <= 0 || T < 0 || !row_perm || !col_perm) return PP_ERR_INVALID_ARG;
+    if (T > 0 && (!tile_list || !tile_values)) return PP_ERR_INVALID_ARG;
+    if (wdtype != PP_F32 && wdtype != PP_F16) return PP_ERR_INVALID_ARG;
+    if (B != 16 && B != 32 && B != 64) return PP_ERR_UNSUPPORTED;
+    const int Mb = (M + B - 1) / B, Nb = (N + B - 1) / B;
+    const int64_t Mpad = (int64_t)Mb * B, Npad = (int64_t)Nb * B;
+    if (Mpad > INT32_MAX || Npad > INT32_MAX || T > (int64_t)Mb * Nb) {
+        if (T > (int64_t)Mb * Nb) return PP_ERR_BAD_TILE;
+        return PP_ERR_INVALID_ARG;
+    }
+    if (!is_bijection(row_perm, Mpad) || !is_bijection(col_perm, Npad)) return PP_ERR_BAD_PERM;
+
+    pp_packed* p = new (std::nothrow) pp_packed();
+    if (!p) return PP_ERR_ALLOC;
+    try {
+        p->M = M; p->N = N; p->B = B; p->Mb = Mb; p->Nb = Nb; p->Mpad = (int)Mpad; p->Npad = (int)Npad;
+        p->T = T; p->wdtype = wdtype; p->has_bias = bias != nullptr;
+        p->row_perm.assign(row_perm, row_perm + Mpad);
+        p->col_perm.assign(col_perm, col_perm + Npad);
+        p->inv_row_perm.resize((size_t)Mpad);
+        for (int64_t i = 0; i < Mpad; ++i) p->inv_row_perm[(size_t)row_perm[i]] = (int32_t)i;
+
+        // sort tiles by (block_row, block_col), rejecting out-of-range and duplicate tiles
+        std::vector<int64_t> order((size_t)T);
+        std::iota(order.begin(), order.end(), 0);
+        for (int64_t t = 0; t < T; ++t) {
+            const int32_t br = tile_list[2 * t], bc = tile_list[2 * t + 1];
+            if (br < 0 || br >= Mb || bc < 0 || bc >= Nb) { delete p; return PP_ERR_BAD_TILE; }
+        }
+        std::sort(order.begin(), order.end(), [&](int64_t a, int64_t b) {
+            const int64_t ka = (int64_t)tile_list[2 * a] * Nb + tile_list[2 * a + 1];
+            const int64_t kb = (int64_t)tile_list[2 * b] * Nb + tile_list[2 * b + 1];
+            return ka < kb;
+        });
+        for (int64_t s = 1; s < T; ++s) {
+            const int64_t a = order[(size_t)s - 1], b = order[(size_t)s];
+            if (tile_list[2 * a] == tile_list[2 * b] && tile_list[2 * a + 1] == tile_list[2 * b + 1]) {
+                delete p; return PP_ERR_BAD_TILE;
+            }
+        }
+
+        // block-row-compressed index arrays; each block-row's column list padded to 4 entries with -1
+        p->row_ptr.assign((size_t)Mb + 1, 0);
+        for (int64_t t = 0; t < T; ++t) p->row_ptr[(size_t)tile_list[2 * t] + 1]++;
+        for (int br = 0; br < Mb; ++br) p->row_ptr[(size_t)br + 1] += p->row_ptr[(size_t)br];
+        p->col_ptr.assign((size_t)Mb + 1, 0);
+        for (int br = 0; br < Mb; ++br) {
+            const int k = p->row_ptr[(size_t)br + 1] - p->row_ptr[(size_t)br];
+            p->col_ptr[(size_t)br + 1] = p->col_ptr[(size_t)br] + (k + 3) / 4 * 4;
+        }
+        p->tile_col.assign((size_t)p->col_ptr[(size_t)Mb], -1);
+        for (int br = 0; br < Mb; ++br)
+            for (int s = p->row_ptr[(size_t)br]; s < p->row_ptr[(size_t)br + 1]; ++s)
+                p->tile_col[(size_t)(p->col_ptr[(size_t)br] + s - p->row_ptr[(size_t)br])] =
+                    tile_list[2 * order[(size_t)s] + 1];
+
+        // tile values -> fragment order
+        const pp::FragGeom g = pp::frag_geom(wdtype, B);
+        const int esz = wdtype == PP_F16 ? 2 : 4;
+        const int frags_per_tile = g.n_rg * g.fpt;
+        p->values.assign((size_t)T * B * B * esz, 0);
+        const unsigned char* src = static_cast<const unsigned char*>(tile_values);
+        for (int br = 0; br < Mb; ++br) {
+            const int r0 = p->row_ptr[(size_t)br], k = p->row_ptr[(size_t)br + 1] - r0;
+            for (int j = 0; j < k; ++j) {
+                const unsigned char* tile = src + (size_t)order[(size_t)(r0 + j)] * B * B * esz;
+                for (int r = 0; r < B; ++r)
+                    for (int c = 0; c < B; ++c) {
+                        const ElemPos e = elem_pos(wdtype, g, r, c);
+                        const size_t frag = (size_t)r0 * frags_per_tile + ((size_t)e.rg * k + j) * g.fpt + e.f;
+                        std::memcpy(&p->values[frag * 512 + e.byte], tile + ((size_t)r * B + c) * esz, esz);
+                    }
+            }
+        }
+
+        p->gather_idx.resize((size_t)Npad);
+        for (int64_t j = 0; j < Npad; ++j) p->gather_idx[(size_t)j] = col_perm[j] < N ? col_perm[j] : -1;
+        p->scatter_idx.resize((size_t)Mpad);
+        p->bias_piv.assign((size_t)Mpad, 0.0f);
+        for (int64_t i = 0; i < Mpad; ++i) {
+            const bool real = row_perm[i] < M;
+            p->scatter_idx[(size_t)i] = real ? row_perm[i] : -1;
+            if (real && bias) p->bias_piv[(size_t)i] = bias[row_perm[i]];
+        }
+        build_items(p);
+    } catch (const std::bad_alloc&) {
+        delete p;
+        return PP_ERR_ALLOC;
+    }
+    *out = p;
+    return PP_OK;
+}
+
+pp_status_t pp_pack_destroy(pp_packed_t* p) {
+    delete p;
+    return PP_OK;
+}
+
+pp_status_t pp_pack_info(const pp_packed_t* p, int64_t out[8]) {
+    if (!p || !out) return PP_ERR_INVALID_ARG;
+    out[0] = p->Mb; out[1] = p->Nb; out[2] = p->T; out[3] = (int64_t)p->tile_col.size();
+    out[4] = (int64_t)p->items.size(); out[5] = (int64_t)p->values.size();
+    out[6] = p->max_item_tiles; out[7] = p->n_slots;
+    return PP_OK;
+}
+
+pp_status_t pp_pack_get(const pp_packed_t* p, int which, void* dst, int64_t bytes) {
+    if (!p || !dst || bytes < 0) return PP_ERR_INVALID_ARG;
+    const void* src = nullptr;
+    size_t n = 0;
+    switch (which) {
+        case 0: src = p->row_ptr.data(); n = p->row_ptr.size() * 4; break;
+        case 1: src = p->col_ptr.data(); n = p->col_ptr.size() * 4; break;
+        case 2: src = p->tile_col.data(); n = p->tile_col.size() * 4; break;
+        case 3: src = p->gather_idx.data(); n = p->gather_idx.size() * 4; break;
+        case 4: src = p->scatter_idx.data(); n = p->scatter_idx.size() * 4; break;
+        case 5: src = p->bias_piv.data(); n = p->bias_piv.size() * 4; break;
+        case 6: src = p->values.data(); n = p->values.size(); break;
+        case 7: src = p->items.data(); n = p->items.size() * sizeof(pp::WorkItem); break;
+        case 8: src = p->inv_row_perm.data(); n = p->inv_row_perm.size() * 4; break;
+        default: return PP_ERR_INVALID_ARG;
+    }
+    if ((size_t)bytes < n) return PP_ERR_INVALID_ARG;
+    if (n) std::memcpy(dst, src, n);
+    return PP_OK;
+}
+
+pp_status_t pp_pack_unpack(const pp_packed_t* p, int32_t* tile_list_out, void* tile_values_out) {
+    if (!p || (p->T > 0 && (!tile_list_out || !tile_values_out))) return PP_ERR_INVALID_ARG;
+    const pp::FragGeom g = pp::frag_geom(p->wdtype, p->B);
+    const int esz = p->wdtype == PP_F16 ? 2 : 4, B = p->B;
+    const int frags_per_tile = g.n_rg * g.fpt;
+    unsigned char* dst = static_cast<unsigned char*>(tile_values_out);
+    for (int br = 0; br < p->Mb; ++br) {
+        const int r0 = p->row_ptr[(size_t)br], k = p->row_ptr[(size_t)br + 1] - r0;
+        for (int j = 0; j < k; ++j) {
+            tile_list_out[2 * (r0 + j)] = br;
+            tile_list_out[2 * (r0 + j) + 1] = p->tile_col[(size_t)(p->col_ptr[(size_t)br] + j)];
+            unsigned char* tile = dst + (size_t)(r0 + j) * B * B * esz;
+            for (int r = 0; r < B; ++r)
+                for (int c = 0; c < B; ++c) {
+                    const ElemPos e = elem_pos(p->wdtype, g, r, c);
+                    const size_t frag = (size_t)r0 * frags_per_tile + ((size_t)e.rg * k + j) * g.fpt + e.f;
+                    std::memcpy(tile + ((size_t)r * B + c) * esz, &p->values[frag * 512 + e.byte], esz);
+                }
+        }
+    }
+    return PP_OK;
+}
+
+pp_status_t pp_fold_perm(const int32_t* row_perm_A, int M_A, int M_pad_A, const int32_t* col_perm_B,
+                         int N_B, int N_pad_B, int32_t* q_out) {
+    if (!row_perm_A || !col_perm_B || !q_out || M_A <= 0 || N_B != M_A || M_pad_A < M_A || N_pad_B < N_B)
+        return PP_ERR_INVALID_ARG;
+    if (!is_bijection(row_perm_A, M_pad_A) || !is_bijection(col_perm_B, N_pad_B)) return PP_ERR_BAD_PERM;
+    std::vector<int32_t> inv((size_t)M_pad_A);
+    for (int i = 0; i < M_pad_A; ++i) inv[(size_t)row_perm_A[i]] = i;
+    for (int j = 0; j < N_pad_B; ++j) q_out[j] = col_perm_B[j] < N_B ? inv[(size_t)col_perm_B[j]] : -1;
+    return PP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,242 @@
+"""Parity of the CUDA library (through its C interface) against the fp64 oracle.
+
+Tolerances (|y - y_ref| <= rtol * (|W| |x|)_i + atol, the magnitude computed by
+the oracle): fp32 weights 1e-5 / 1e-6; fp16 weights with fp32 accumulation
+2e-3 / 1e-4.  Index and permutation handling is checked bit for bit with small
+integer data, for which every partial sum is exact in fp16 / fp32 / fp64."""
+import numpy as np
+import pytest
+
+from oracle import pp_oracle as po
+from paper_1712_01084_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+TOL = {np.dtype(np.float32): (1e-5, 1e-6), np.dtype(np.float16): (2e-3, 1e-4)}
+
+
+@pytest.fixture(scope="module")
+def pb():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_1712_01084_b200 import binding
+    binding.lib()                     # fails loudly if the library is not built
+    return binding
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _rand_layer(seed, M, N, B, dtype, density=0.4, bias=True, integer=False, empty_rows=()):
+    rng = np.random.default_rng(seed)
+    Mb, Nb = -(-M // B), -(-N // B)
+    grid = [(br, bc) for br in range(Mb) for bc in range(Nb) if br not in empty_rows]
+    T = max(1, int(density * len(grid)))
+    sel = rng.permutation(len(grid))[:T]
+    tl = np.array([grid[s] for s in sel], dtype=np.int32).reshape(-1, 2)
+    if integer:
+        tv = rng.integers(-4, 5, size=(T, B, B)).astype(dtype)
+        b = rng.integers(-8, 9, size=M).astype(np.float32) if bias else None
+    else:
+        tv = (rng.standard_normal((T, B, B)) / np.sqrt(N)).astype(dtype)
+        b = (rng.standard_normal(M) * 0.1).astype(np.float32) if bias else None
+    return synth.Layer(M, N, B, rng.permutation(Mb * B).astype(np.int32),
+                       rng.permutation(Nb * B).astype(np.int32), tl, tv, b)
+
+
+def _check(y_gpu, y_ref, a_ref, dtype, what=""):
+    rtol, atol = TOL[np.dtype(dtype)]
+    err = np.abs(y_gpu.astype(np.float64) - y_ref)
+    bound = rtol * a_ref + atol
+    worst = np.max(err / bound)
+    assert worst <= 1.0, f"{what}: worst error/bound = {worst:.3f}"
+
+
+def _run_and_check(pb, lay, x, act, what=""):
+    L = pb.Layer.from_synth(lay)
+    y = pb.pp_forward(L, _dev(x), act).cpu().numpy()
+    y_ref, _, a = po.layer_forward(lay, x.astype(np.float64), act=act, threads=8)
+    _check(y, y_ref, a, lay.tile_values.dtype, what)
+    L.close()
+    return y
+
+
+# ------------------------------------------------------------------ small sweeps
+@pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("B", [16, 32, 64])
+@pytest.mark.parametrize("batch", [1, 2, 3, 8, 9, 17, 33])
+def test_small_layers(pb, dtype, B, batch):
+    """Ragged M and N, unbalanced block-rows, one block-row without tiles, several tiles and a ragged tail."""
+    lay = _rand_layer(100 + B + batch, 5 * B - 3, 9 * B - 7, B, dtype, density=0.45, empty_rows=(2,))
+    x = np.random.default_rng(batch).uniform(-1, 1, (batch, lay.N)).astype(dtype)
+    for act in (0, 1):
+        _run_and_check(pb, lay, x, act, f"{dtype.__name__} B={B} batch={batch} act={act}")
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("target_kib", [1, 4, 64])
+def test_split_block_rows(pb, dtype, target_kib):
+    """Block-rows cut into many work items (cross-CTA reduction) and into one."""
+    pb.pp_set_tuning(0, target_kib)
+    try:
+        lay = _rand_layer(7, 200, 1500, 32, dtype, density=0.6)
+        for batch in (1, 5):
+            x = np.random.default_rng(3).uniform(-1, 1, (batch, lay.N)).astype(dtype)
+            _run_and_check(pb, lay, x, 1, f"target {target_kib} KiB batch {batch}")
+    finally:
+        pb.pp_set_tuning(0, 32)
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("B", [16, 32, 64])
+def test_integer_data_is_bit_exact(pb, dtype, B):
+    """Small-integer weights, inputs and bias: all sums exact, so any index or
+    permutation slip shows up as a bit difference."""
+    pb.pp_set_tuning(0, 2)
+    try:
+        lay = _rand_layer(50 + B, 4 * B - 1, 6 * B - 5, B, dtype, density=0.5, integer=True)
+        for batch in (1, 4, 11):
+            x = np.random.default_rng(5).integers(-2, 3, (batch, lay.N)).astype(dtype)
+            L = pb.Layer.from_synth(lay)
+            for act in (0, 1):
+                y = pb.pp_forward(L, _dev(x), act).cpu().numpy()
+                y_ref, _, _ = po.layer_forward(lay, x.astype(np.float64), act=act)
+                assert np.array_equal(y.astype(np.float64), y_ref)
+            L.close()
+    finally:
+        pb.pp_set_tuning(0, 32)
+
+
+def test_identity_perms_density_one(pb):
+    lay, rng = synth.make_layer(1, 256, 384, 64, wdtype="f32", tiles="balanced", k=6, identity_perms=True)
+    x = synth.draw_x(rng, 2, 384, -1, 1, "f32")
+    y = _run_and_check(pb, lay, x, 0, "dense identity")
+    Wd = np.block([[lay.tile_values[br * 6 + bc] for bc in range(6)] for br in range(4)]).astype(np.float64)
+    ref = x.astype(np.float64) @ Wd.T
+    assert np.max(np.abs(y - ref)) < 1e-5
+
+
+def test_deterministic_and_canaries(pb):
+    """Same inputs twice -> identical bits; memory around y is untouched."""
+    pb.pp_set_tuning(0, 2)
+    try:
+        lay = _rand_layer(9, 777, 1111, 32, np.float16, density=0.5)
+        L = pb.Layer.from_synth(lay)
+    finally:
+        pb.pp_set_tuning(0, 32)
+    x = _dev(np.random.default_rng(1).uniform(-1, 1, (3, lay.N)).astype(np.float16))
+    pad = 64
+    buf = torch.full((3 * lay.M + 2 * pad,), 12345.0, dtype=torch.float32, device="cuda")
+    out = buf[pad:pad + 3 * lay.M].view(3, lay.M)
+    y1 = pb.pp_forward(L, x, 1, out=out).clone()
+    assert torch.all(buf[:pad] == 12345.0) and torch.all(buf[-pad:] == 12345.0)
+    for _ in range(5):
+        y2 = pb.pp_forward(L, x, 1)
+        assert torch.equal(y1, y2)
+    L.close()
+
+
+def test_argument_errors(pb):
+    lay = _rand_layer(10, 64, 64, 32, np.float32)
+    L = pb.Layer.from_synth(lay)
+    x = torch.zeros(4096, device="cuda")
+    assert pb.lib().pp_forward(L._h, x.data_ptr() + 4, x.data_ptr() + 2048, 1, 0, None) == 1   # misaligned x
+    assert pb.lib().pp_forward(L._h, x.data_ptr(), x.data_ptr(), 1, 0, None) == 1     # aliasing
+    assert pb.lib().pp_forward(L._h, x.data_ptr(), x.data_ptr() + 2048, 0, 0, None) == 1  # batch 0
+    with pytest.raises(TypeError):
+        pb.pp_forward(L, torch.zeros(1, 64, device="cuda", dtype=torch.float16))
+    L.close()
+
+
+# ------------------------------------------------------------------ the five workloads
+def test_config1_full(pb):
+    wl = synth.config1()
+    _run_and_check(pb, wl.layers[0], wl.x, wl.layers[0].act, "config 1")
+
+
+def test_config2_full(pb):
+    wl = synth.config2()
+    _run_and_check(pb, wl.layers[0], wl.x, wl.layers[0].act, "config 2")
+
+
+def _chain_bound(layers, res, dtype_tol):
+    """Propagated end-to-end bound: e_{l} <= |W_l| e_{l-1} + tol_l (+ fp16 rounding of the stored output)."""
+    rtol, atol = dtype_tol
+    e = None
+    for li, lay in enumerate(layers):
+        xin, y, a = res[li]
+        tol = rtol * a + atol
+        if e is not None:
+            W = po.reconstruct(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values)
+            prop, _, _ = po.dense_forward(np.abs(W), None, e, 0, threads=8)
+            tol = tol + prop
+        if li + 1 < len(layers):
+            tol = tol + np.abs(y) * 2.0 ** -10 + 2.0 ** -24     # stored as fp16 (both sides round)
+        e = tol
+    return e
+
+
+@pytest.mark.parametrize("batch", [1, 8])
+def test_config3_chain_full(pb, batch):
+    wl = synth.config3(batch=batch)
+    layers = [pb.Layer.from_synth(l) for l in wl.layers]
+    chain = pb.Chain(layers, [l.act for l in wl.layers], max_batch=8)
+    y = pb.pp_chain_forward(chain, _dev(wl.x)).cpu().numpy().astype(np.float64)
+    res = po.chain_forward(wl.layers, wl.x.astype(np.float64), round_intermediate="f16", threads=8)
+    bound = _chain_bound(wl.layers, res, TOL[np.dtype(np.float16)])
+    worst = np.max(np.abs(y - res[-1][1]) / bound)
+    assert worst <= 1.0, f"chain end-to-end worst error/bound {worst:.3f}"
+    # teacher-forced per-layer check: every layer alone, fed the oracle's (rounded) input
+    for li, lay in enumerate(wl.layers):
+        xin = res[li][0].astype(np.float16)
+        yl = pb.pp_forward(layers[li], _dev(xin), lay.act).cpu().numpy()
+        _check(yl, res[li][1], res[li][2], np.float16, f"config 3 layer {li}")
+    chain.close()
+    for l in layers:
+        l.close()
+
+
+def test_chain_matches_layer_by_layer_bits(pb):
+    """Folded chain (pivoted intermediates) == unfolded evaluation with the same
+    kernels, bit for bit, on integer data; fp32 chain against the oracle."""
+    dims = [200, 150, 90, 33]
+    lays = []
+    for l in range(3):
+        lay = _rand_layer(300 + l, dims[l + 1], dims[l], 16, np.float32, density=0.5, integer=True)
+        lay.tile_values = np.sign(lay.tile_values) * (np.abs(lay.tile_values) > 3)   # entries in {-1,0,1}
+        lay.act = 1 if l < 2 else 0
+        lays.append(lay)
+    x = np.random.default_rng(2).integers(-1, 2, (3, dims[0])).astype(np.float32)
+    L = [pb.Layer.from_synth(l) for l in lays]
+    chain = pb.Chain(L, [l.act for l in lays], max_batch=4)
+    y = pb.pp_chain_forward(chain, _dev(x)).cpu().numpy()
+    cur = _dev(x)
+    for lay, Ld in zip(lays, L):
+        cur = pb.pp_forward(Ld, cur, lay.act)
+    assert np.array_equal(y, cur.cpu().numpy())
+    res = po.chain_forward(lays, x.astype(np.float64))
+    assert np.array_equal(y.astype(np.float64), res[-1][1])
+    chain.close()
+
+
+@pytest.mark.parametrize("k", [128, 16, 8])
+def test_config5_batch1_full(pb, k):
+    wl = synth.config5(k=k, batch=1)
+    _run_and_check(pb, wl.layers[0], wl.x, 0, f"config 5 k={k}")
+
+
+@pytest.mark.parametrize("batch", [16])
+def test_config5_small_batch_sampled_rows(pb, batch):
+    """Full size; the oracle evaluates a sample of output rows."""
+    wl = synth.config5(k=32, batch=batch)
+    lay = wl.layers[0]
+    L = pb.Layer.from_synth(lay)
+    y = pb.pp_forward(L, _dev(wl.x), 0).cpu().numpy()
+    W = po.reconstruct(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values)
+    rows = np.random.default_rng(0).choice(lay.M, 256, replace=False).astype(np.int32)
+    y_ref, a = po.dense_forward_rows(W, None, wl.x.astype(np.float64), 0, rows)
+    _check(y[:, rows], y_ref, a, np.float16, "config 5 batch 16 sampled")
+    L.close()

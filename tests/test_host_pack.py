@@ -1,0 +1,270 @@
+"""Host-side logic of the C library, exercised without a GPU: symbol export,
+packer round trip, index arrays, fragment layout, work list, permutation
+folding and error codes.  The last test walks the packed arrays with the same
+address arithmetic the kernels use and compares with the oracle, so every index
+the kernels form is checked for range on the CPU."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import pp_oracle as po
+from paper_1712_01084_b200 import binding as pb
+from paper_1712_01084_b200 import build as pbuild
+from paper_1712_01084_b200 import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    pbuild.build()
+
+
+def test_library_exports_every_declared_symbol():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            src = open(os.path.join(ROOT, "include", fn)).read()
+            src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+            names |= set(re.findall(r"\b(pp_[a-z0-9_]+)\s*\(", src))
+    assert {"pp_layer_create", "pp_forward", "pp_chain_forward", "pp_pack_create"} <= names
+    L = ctypes.CDLL(pb.LIB_PATH)
+    for n in sorted(names):
+        assert hasattr(L, n), f"{n} declared in include/ but not exported"
+
+
+def _random_layer(seed, M, N, B, dtype, density=0.4, bias=True):
+    rng = np.random.default_rng(seed)
+    Mb, Nb = -(-M // B), -(-N // B)
+    T = max(1, int(density * Mb * Nb))
+    flat = rng.permutation(Mb * Nb)[:T]          # deliberately unsorted
+    tl = np.stack([flat // Nb, flat % Nb], axis=1).astype(np.int32)
+    tv = rng.standard_normal((T, B, B)).astype(dtype)
+    return synth.Layer(M, N, B, rng.permutation(Mb * B).astype(np.int32), rng.permutation(Nb * B).astype(np.int32),
+                       tl, tv, rng.standard_normal(M).astype(np.float32) if bias else None)
+
+
+def _pack(lay):
+    return pb.Packed(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values, lay.bias)
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("B", [16, 32, 64])
+def test_round_trip_bit_exact(dtype, B):
+    lay = _random_layer(B + (dtype == np.float16), 5 * B - 3, 7 * B - 1, B, dtype)
+    pk = _pack(lay)
+    tl, tv = pk.unpack()
+    order = np.lexsort((lay.tile_list[:, 1], lay.tile_list[:, 0]))
+    assert np.array_equal(tl, lay.tile_list[order])
+    assert np.array_equal(tv.view(np.uint8), lay.tile_values[order].view(np.uint8))
+
+
+def test_index_arrays():
+    lay = _random_layer(3, 100, 200, 16, np.float16)
+    pk = _pack(lay)
+    row_ptr, col_ptr, tile_col = pk.get("row_ptr"), pk.get("col_ptr"), pk.get("tile_col")
+    assert row_ptr[0] == 0 and row_ptr[-1] == lay.T and col_ptr[0] == 0
+    order = np.lexsort((lay.tile_list[:, 1], lay.tile_list[:, 0]))
+    st = lay.tile_list[order]
+    for br in range(pk.Mb):
+        k = row_ptr[br + 1] - row_ptr[br]
+        seg = tile_col[col_ptr[br]:col_ptr[br + 1]]
+        assert len(seg) % 4 == 0 and len(seg) == -(-k // 4) * 4          # 16-byte aligned runs
+        assert np.array_equal(seg[:k], st[row_ptr[br]:row_ptr[br + 1], 1])
+        assert np.all(seg[k:] == -1)
+        assert np.all(np.diff(seg[:k]) > 0)
+    g = pk.get("gather_idx"); s = pk.get("scatter_idx"); b = pk.get("bias_piv")
+    assert np.array_equal(g, np.where(lay.col_perm < lay.N, lay.col_perm, -1))
+    assert np.array_equal(s, np.where(lay.row_perm < lay.M, lay.row_perm, -1))
+    real = lay.row_perm < lay.M
+    assert np.array_equal(b[real], lay.bias[lay.row_perm[real]]) and np.all(b[~real] == 0)
+    inv = pk.get("inv_row_perm")
+    assert np.array_equal(inv[lay.row_perm], np.arange(pk.Mb * 16))
+
+
+def test_fragment_layout_fp32_lane_is_row():
+    """fp32, B=32: fragment f of a tile holds columns 4f..4f+3, lane = row."""
+    lay = _random_layer(4, 64, 64, 32, np.float32, density=1.0)
+    pk = _pack(lay)
+    vals = pk.get("values").view(np.float32).reshape(-1, 32, 4)      # [frag][lane][q]
+    tl, tv = pk.unpack()
+    row_ptr = pk.get("row_ptr")
+    for br in range(pk.Mb):
+        k = row_ptr[br + 1] - row_ptr[br]
+        for j in range(k):
+            tile = tv[row_ptr[br] + j]
+            for f in range(8):
+                frag = row_ptr[br] * 8 + j * 8 + f
+                assert np.array_equal(vals[frag], tile[:, 4 * f:4 * f + 4])
+
+
+def test_fragment_layout_fp16_is_mma_operand():
+    """fp16: each 512-byte fragment is a 16x16 block in the register order of the
+    m16n8k16 A operand: lane = 4*(row%8) + (col%8)//2, slots (r,c),(r,c+1),(r+8,c),(r+8,c+1),(r,c+8),..."""
+    lay = _random_layer(5, 64, 128, 64, np.float16, density=1.0)
+    pk = _pack(lay)
+    vals = pk.get("values").view(np.float16).reshape(-1, 32, 8)
+    tl, tv = pk.unpack()
+    row_ptr = pk.get("row_ptr")
+    for br in range(pk.Mb):
+        k = row_ptr[br + 1] - row_ptr[br]
+        for j in range(k):
+            tile = tv[row_ptr[br] + j]
+            for rg in range(4):
+                for f in range(4):
+                    frag = row_ptr[br] * 16 + (rg * k + j) * 4 + f
+                    blk = tile[16 * rg:16 * rg + 16, 16 * f:16 * f + 16]
+                    for lane in range(32):
+                        g, t = lane // 4, lane % 4
+                        want = [blk[g, 2 * t], blk[g, 2 * t + 1], blk[g + 8, 2 * t], blk[g + 8, 2 * t + 1],
+                                blk[g, 2 * t + 8], blk[g, 2 * t + 9], blk[g + 8, 2 * t + 8], blk[g + 8, 2 * t + 9]]
+                        assert list(vals[frag, lane]) == want
+
+
+def test_work_items_cover_every_tile_once():
+    for target in (1, 8, 32, 1024):
+        pb.pp_set_tuning(0, target)
+        try:
+            lay = _random_layer(6, 300, 500, 32, np.float16, density=0.3)
+            pk = _pack(lay)
+            items, row_ptr, col_ptr = pk.get("items"), pk.get("row_ptr"), pk.get("col_ptr")
+            seen = np.zeros(lay.T, dtype=int)
+            per_br = {}
+            for it in items:
+                frag_base, rg_stride, nf, col_off, ntiles, br, pn, slot_base = [int(v) for v in it]
+                part, nparts = pn & 0xffff, pn >> 16
+                k = row_ptr[br + 1] - row_ptr[br]
+                j0 = col_off - col_ptr[br]
+                assert 0 <= j0 and j0 + ntiles <= max(k, 0) and nf == ntiles * 2 and rg_stride == k * 2
+                assert frag_base == row_ptr[br] * 4 + j0 * 2
+                seen[row_ptr[br] + j0: row_ptr[br] + j0 + ntiles] += 1
+                per_br.setdefault(br, []).append((part, nparts, slot_base))
+                assert ntiles * 32 <= 2048
+            assert np.all(seen == 1)
+            assert sorted(per_br) == list(range(pk.Mb))              # empty block-rows still get an item
+            slots = 0
+            for br, parts in per_br.items():
+                assert [p for p, _, _ in parts] == list(range(parts[0][1]))
+                if parts[0][1] > 1:
+                    slots += parts[0][1]
+            assert slots == pk.n_slots
+        finally:
+            pb.pp_set_tuning(0, 32)
+
+
+def test_fold_perm_hand_example(hand4):
+    rp = np.array(hand4["row_perm"], dtype=np.int32); cp = np.array(hand4["col_perm"], dtype=np.int32)
+    q = pb.pp_fold_perm(rp, 4, cp, 4)
+    assert list(q) == hand4["folded_q"]
+    # layer-2 pivoted input gathered from layer-1 pivoted output
+    y1_piv = np.array(hand4["layer1_piv_act"])
+    assert list(y1_piv[q]) == hand4["layer2_x_piv"]
+
+
+def test_fold_perm_property_with_padding():
+    """Gathering the producer's pivoted output through q equals scattering it to
+    original order and gathering through the consumer's col_perm (Section 4.2.1)."""
+    rng = np.random.default_rng(9)
+    M, BA, BB = 1000, 32, 16
+    MpA, NpB = -(-M // BA) * BA, -(-M // BB) * BB
+    rpA = rng.permutation(MpA).astype(np.int32); cpB = rng.permutation(NpB).astype(np.int32)
+    q = pb.pp_fold_perm(rpA, M, cpB, M)
+    y_piv = rng.standard_normal(MpA)
+    y = np.zeros(M)
+    real = rpA < M
+    y[rpA[real]] = y_piv[real]
+    want = np.where(cpB < M, y[np.minimum(cpB, M - 1)], 0.0)
+    got = np.where(q >= 0, y_piv[np.maximum(q, 0)], 0.0)
+    assert np.array_equal(got, want)
+    # identical permutations fold to the identity (cross-layer permutation elimination)
+    assert np.array_equal(pb.pp_fold_perm(rpA, MpA, rpA, MpA), np.arange(MpA))
+
+
+def test_error_codes():
+    lay = _random_layer(7, 64, 64, 32, np.float32)
+    bad = lay.row_perm.copy(); bad[0] = bad[1]
+    with pytest.raises(pb.PPError) as e:
+        pb.Packed(lay.M, lay.N, lay.B, bad, lay.col_perm, lay.tile_list, lay.tile_values)
+    assert e.value.status == 2
+    tl = np.concatenate([lay.tile_list, lay.tile_list[:1]]); tv = np.concatenate([lay.tile_values, lay.tile_values[:1]])
+    with pytest.raises(pb.PPError) as e:
+        pb.Packed(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, tl, tv)
+    assert e.value.status == 3
+    tl = lay.tile_list.copy(); tl[0, 1] = 99
+    with pytest.raises(pb.PPError) as e:
+        pb.Packed(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, tl, lay.tile_values)
+    assert e.value.status == 3
+    with pytest.raises(pb.PPError) as e:
+        pb.Packed(48, 48, 24, np.arange(48), np.arange(48), np.zeros((1, 2), np.int32), np.zeros((1, 24, 24), np.float32))
+    assert e.value.status == 6
+    L = pb.lib()
+    assert L.pp_pack_create(None, 1, 1, 16, None, None, None, 0, None, 0, None) == 1
+    assert L.pp_forward(None, None, None, 1, 0, None) == 1
+    assert L.pp_chain_forward(None, None, None, 1, None) == 1
+    assert b"permutation" in L.pp_status_string(2)
+
+
+# ------------------------------------------------ walk the packed arrays like a kernel
+def _emulate(pk, x, act, dtype):
+    """y from the packed arrays only, forming every index the way the kernels do."""
+    B = pk.B
+    f16 = dtype == np.float16
+    rg_rows = 16 if f16 else min(B, 32)
+    kf = 16 if f16 else 128 // rg_rows
+    n_rg = B // rg_rows
+    vals = pk.get("values").view(dtype)
+    n_frag = vals.size * vals.itemsize // 512
+    per_lane = 8 if f16 else 4
+    vals = vals.reshape(n_frag, 32, per_lane)
+    items, tile_col = pk.get("items"), pk.get("tile_col")
+    gather, scatter, bias = pk.get("gather_idx"), pk.get("scatter_idx"), pk.get("bias_piv")
+    y = np.full(pk.M, np.nan)
+    acc = np.zeros(pk.Mb * B)
+    for it in items:
+        frag_base, rg_stride, nf, col_off, ntiles, br, pn, _ = [int(v) for v in it]
+        xs = np.zeros(ntiles * B)
+        for c in range(ntiles * B):
+            col = tile_col[col_off + c // B]
+            assert 0 <= col < pk.Nb
+            idx = gather[col * B + c % B]
+            assert -1 <= idx < pk.N
+            xs[c] = x[idx] if idx >= 0 else 0.0
+        for rg in range(n_rg):
+            for i in range(nf):
+                frag = frag_base + rg * rg_stride + i
+                assert 0 <= frag < n_frag
+                for lane in range(32):
+                    if f16:
+                        g, t = lane // 4, lane % 4
+                        w = vals[frag, lane].astype(np.float64)
+                        k0 = i * 16 + 2 * t
+                        acc[br * B + rg * 16 + g] += w[0] * xs[k0] + w[1] * xs[k0 + 1] + w[4] * xs[k0 + 8] + w[5] * xs[k0 + 9]
+                        acc[br * B + rg * 16 + g + 8] += w[2] * xs[k0] + w[3] * xs[k0 + 1] + w[6] * xs[k0 + 8] + w[7] * xs[k0 + 9]
+                    else:
+                        row = lane % rg_rows
+                        k0 = i * kf + (lane // rg_rows) * 4
+                        acc[br * B + rg * rg_rows + row] += float(np.dot(vals[frag, lane].astype(np.float64), xs[k0:k0 + 4]))
+    for i in range(pk.Mb * B):
+        if scatter[i] >= 0:
+            v = acc[i] + bias[i]
+            y[scatter[i]] = max(v, 0.0) if act else v
+    return y
+
+
+@pytest.mark.parametrize("dtype,B", [(np.float32, 16), (np.float32, 32), (np.float32, 64),
+                                     (np.float16, 16), (np.float16, 32), (np.float16, 64)])
+def test_packed_walk_matches_oracle(dtype, B):
+    pb.pp_set_tuning(0, 4)          # small runs so block-rows are split into several items
+    try:
+        lay = _random_layer(20 + B, 3 * B - 5, 4 * B - 2, B, dtype, density=0.5)
+        pk = _pack(lay)
+    finally:
+        pb.pp_set_tuning(0, 32)
+    x = np.random.default_rng(1).uniform(-1, 1, lay.N).astype(dtype)
+    got = _emulate(pk, x.astype(np.float64), 1, dtype)
+    y, _, a = po.layer_forward(lay, x.astype(np.float64), act=1)
+    assert not np.any(np.isnan(got))
+    assert np.all(np.abs(got - y[0]) <= 1e-12 * (a[0] + 1))
