@@ -94,13 +94,17 @@ pp_status_t pp_pack_destroy(pp_packed_t* p);
 
 /* Sizes of the packed arrays: out[0]=Mb, [1]=Nb, [2]=T, [3]=length of tile_col
  * (padded), [4]=number of work items, [5]=bytes of packed values,
- * [6]=max tiles in one work item, [7]=number of partial-sum slots. */
-pp_status_t pp_pack_info(const pp_packed_t* p, int64_t out[8]);
+ * [6]=max tiles in one work item, [7]=number of partial-sum slots,
+ * [8]=S strips (row-groups of block-rows), [9]=F fragments (512-byte units of values),
+ * [10]=CTAs of the persistent kernel's plan, [11]=its cross-CTA partial-sum slots. */
+pp_status_t pp_pack_info(const pp_packed_t* p, int64_t out[12]);
 
 /* Copy one packed array to host memory `dst` of capacity `bytes`.
  * which: 0 row_ptr(int32[Mb+1]) 1 col_ptr(int32[Mb+1]) 2 tile_col(int32[])
  *        3 gather_idx(int32[N_pad]) 4 scatter_idx(int32[M_pad]) 5 bias_piv(float[M_pad])
- *        6 values (bytes) 7 work items (int32[n_items][8]) 8 inv_row_perm(int32[M_pad]) */
+ *        6 values (bytes) 7 work items (int32[n_items][8]) 8 inv_row_perm(int32[M_pad])
+ *        9 strip_start(int32[S+1]) 10 xoff(int32[F]) 11 CTA ranges (int32[G][4] =
+ *        p_begin,p_end,s_first,s_count) 12 strip info (int32[S][4] = first_cta,nparts,slot_base,0) */
 pp_status_t pp_pack_get(const pp_packed_t* p, int which, void* dst, int64_t bytes);
 
 /* Inverse of the value re-ordering: writes the sorted tile list (int32[T][2])
@@ -161,7 +165,11 @@ pp_status_t pp_chain_forward(pp_chain_t* chain, const void* x, void* y, int batc
 
 /* Tuning knobs read at pack / create time (process-wide; for experiments).
  * key 0: target kilobytes of tile values per work item (default 32)
- * key 1: lower bound on the number of work items the splitter aims for (default 296) */
+ * key 1: lower bound on the number of work items the splitter aims for (default 296)
+ * key 2: CTAs of the persistent kernel (default 296)
+ * key 3: minimum fragments per CTA of the persistent kernel (default 128)
+ * key 4: snap tolerance, percent of a CTA's share, for moving CTA boundaries onto strip boundaries (default 25)
+ * key 5: 0 = never use the persistent kernel, 1 = use it when batch <= 8 and x fits shared memory (default 1) */
 pp_status_t pp_set_tuning(int key, int value);
 
 #ifdef __cplusplus

@@ -115,10 +115,11 @@ class Packed:
         _check(lib().pp_pack_create(ctypes.byref(self._h), *args), "pp_pack_create")
         self.M, self.N, self.B = int(M), int(N), int(B)
         self.wdtype = np.asarray(tile_values).dtype
-        info = (ctypes.c_int64 * 8)()
+        info = (ctypes.c_int64 * 12)()
         _check(lib().pp_pack_info(self._h, info), "pp_pack_info")
         (self.Mb, self.Nb, self.T, self.n_tile_col, self.n_items, self.value_bytes,
-         self.max_item_tiles, self.n_slots) = [int(v) for v in info]
+         self.max_item_tiles, self.n_slots, self.n_strips, self.n_frags, self.stream_grid,
+         self.stream_slots) = [int(v) for v in info]
 
     def get(self, which: str) -> np.ndarray:
         Mpad, Npad = self.Mb * self.B, self.Nb * self.B
@@ -126,10 +127,14 @@ class Packed:
                 "tile_col": (2, np.int32, self.n_tile_col), "gather_idx": (3, np.int32, Npad),
                 "scatter_idx": (4, np.int32, Mpad), "bias_piv": (5, np.float32, Mpad),
                 "values": (6, np.uint8, self.value_bytes), "items": (7, np.int32, self.n_items * 8),
-                "inv_row_perm": (8, np.int32, Mpad)}[which]
+                "inv_row_perm": (8, np.int32, Mpad), "strip_start": (9, np.int32, self.n_strips + 1),
+                "xoff": (10, np.int32, self.n_frags), "cta_desc": (11, np.int32, self.stream_grid * 4),
+                "strip_info": (12, np.int32, self.n_strips * 4)}[which]
         out = np.empty(spec[2], dtype=spec[1])
         _check(lib().pp_pack_get(self._h, spec[0], out.ctypes.data_as(ctypes.c_void_p), out.nbytes), "pp_pack_get")
-        return out.reshape(-1, 8) if which == "items" else out
+        if which == "items":
+            return out.reshape(-1, 8)
+        return out.reshape(-1, 4) if which in ("cta_desc", "strip_info") else out
 
     def unpack(self):
         tl = np.empty((self.T, 2), dtype=np.int32)

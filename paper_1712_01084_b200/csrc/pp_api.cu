@@ -6,6 +6,7 @@
 
 #include "pp_gemv.cuh"
 #include "pp_internal.h"
+#include "pp_stream.cuh"
 
 struct pp_layer {
     pp_packed* pk = nullptr;       // host copy (index arrays are needed again when chains are folded)
@@ -19,6 +20,14 @@ struct pp_layer {
     int* d_counters = nullptr;
     int n_items = 0;
     int max_item_tiles = 0;
+    // persistent streaming kernel
+    int32_t* d_xoff = nullptr;
+    int32_t* d_strip_start = nullptr;
+    pp::CtaDesc* d_cta_desc = nullptr;
+    pp::StripInfo* d_strip_info = nullptr;
+    float* d_spartials = nullptr;
+    int* d_scounters = nullptr;
+    int stream_grid = 0;
 };
 
 struct pp_chain {
@@ -43,6 +52,8 @@ void free_layer(pp_layer* L) {
     if (!L) return;
     cudaFree(L->d_values); cudaFree(L->d_items); cudaFree(L->d_tile_col); cudaFree(L->d_gather);
     cudaFree(L->d_scatter); cudaFree(L->d_bias); cudaFree(L->d_partials); cudaFree(L->d_counters);
+    cudaFree(L->d_xoff); cudaFree(L->d_strip_start); cudaFree(L->d_cta_desc); cudaFree(L->d_strip_info);
+    cudaFree(L->d_spartials); cudaFree(L->d_scounters);
     pp_pack_destroy(L->pk);
     delete L;
 }
@@ -53,6 +64,17 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_elt, void* y, int ldy,
                       int out_mode, int batch, pp_act_t act, cudaStream_t stream) {
     const pp_packed* pk = L->pk;
+    if (pp::g_use_stream && batch <= pp::kStreamMaxBatch &&
+        pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, batch) <= pp::kStreamSmemLimit) {
+        pp::StreamArgs s{};
+        s.values = L->d_values; s.xoff = L->d_xoff; s.strip_start = L->d_strip_start;
+        s.cta_desc = L->d_cta_desc; s.strip_info = L->d_strip_info;
+        s.gather_idx = gather; s.scatter_idx = L->d_scatter; s.bias_piv = L->d_bias;
+        s.x = x; s.y = y; s.partials = L->d_spartials; s.counters = L->d_scounters;
+        s.ldx = ldx; s.ldy = ldy; s.x_limit = pk->N; s.n_pad = pk->Npad; s.batch = batch;
+        s.act = (int)act; s.out_mode = out_mode;
+        return pp::launch_stream(pk->wdtype, pk->B, s, L->stream_grid, stream) == cudaSuccess ? PP_OK : PP_ERR_CUDA;
+    }
     pp::GemvArgs a{};
     a.values = L->d_values; a.items = L->d_items; a.tile_col = L->d_tile_col;
     a.gather_idx = gather; a.scatter_idx = L->d_scatter; a.bias_piv = L->d_bias;
@@ -101,13 +123,27 @@ pp_status_t pp_layer_create(pp_layer_t** out, int M, int N, int B, const int32_t
              cudaMalloc(reinterpret_cast<void**>(&L->d_counters), (size_t)pk->Mb * sizeof(int)) == cudaSuccess &&
              cudaMemset(L->d_counters, 0, (size_t)pk->Mb * sizeof(int)) == cudaSuccess;
     }
+    if (ok) {
+        const int S = (int)pk->strip_info.size();
+        const int rg = pp::frag_geom(wdtype, B).rg_rows;
+        const size_t sp = (size_t)pk->stream_slots * rg * pp::kStreamMaxBatch * sizeof(float);
+        L->stream_grid = (int)pk->cta_desc.size();
+        ok = upload(&L->d_xoff, pk->xoff.data(), pk->xoff.size() * 4) &&
+             upload(&L->d_strip_start, pk->strip_start.data(), pk->strip_start.size() * 4) &&
+             upload(&L->d_cta_desc, pk->cta_desc.data(), pk->cta_desc.size() * sizeof(pp::CtaDesc)) &&
+             upload(&L->d_strip_info, pk->strip_info.data(), pk->strip_info.size() * sizeof(pp::StripInfo)) &&
+             cudaMalloc(reinterpret_cast<void**>(&L->d_spartials), sp ? sp : 16) == cudaSuccess &&
+             cudaMalloc(reinterpret_cast<void**>(&L->d_scounters), (size_t)(S ? S : 1) * sizeof(int)) == cudaSuccess &&
+             cudaMemset(L->d_scounters, 0, (size_t)(S ? S : 1) * sizeof(int)) == cudaSuccess;
+    }
     if (!ok) {
         const cudaError_t e = cudaGetLastError();
         free_layer(L);
         return e == cudaErrorMemoryAllocation ? PP_ERR_ALLOC : PP_ERR_CUDA;
     }
-    // the fragment-ordered values now live on the device; drop the host copy
+    // the fragment-ordered values and per-fragment offsets now live on the device; drop the host copies
     std::vector<unsigned char>().swap(pk->values);
+    std::vector<int32_t>().swap(pk->xoff);
     *out = L;
     return PP_OK;
 }
@@ -139,6 +175,20 @@ pp_status_t pp_layer_clone(pp_layer_t** out, const pp_layer_t* src) {
               cudaMalloc(reinterpret_cast<void**>(&L->d_partials), pbytes ? pbytes : 16) == cudaSuccess &&
               cudaMalloc(reinterpret_cast<void**>(&L->d_counters), (size_t)pk->Mb * sizeof(int)) == cudaSuccess &&
               cudaMemset(L->d_counters, 0, (size_t)pk->Mb * sizeof(int)) == cudaSuccess;
+    if (ok) {
+        const int S = (int)pk->strip_info.size();
+        const pp::FragGeom g = pp::frag_geom(pk->wdtype, pk->B);
+        const size_t F = (size_t)pk->T * g.n_rg * g.fpt;
+        const size_t sp = (size_t)pk->stream_slots * g.rg_rows * pp::kStreamMaxBatch * sizeof(float);
+        L->stream_grid = src->stream_grid;
+        ok = dup(&L->d_xoff, src->d_xoff, F * 4) &&
+             dup(&L->d_strip_start, src->d_strip_start, pk->strip_start.size() * 4) &&
+             dup(&L->d_cta_desc, src->d_cta_desc, pk->cta_desc.size() * sizeof(pp::CtaDesc)) &&
+             dup(&L->d_strip_info, src->d_strip_info, pk->strip_info.size() * sizeof(pp::StripInfo)) &&
+             cudaMalloc(reinterpret_cast<void**>(&L->d_spartials), sp ? sp : 16) == cudaSuccess &&
+             cudaMalloc(reinterpret_cast<void**>(&L->d_scounters), (size_t)(S ? S : 1) * sizeof(int)) == cudaSuccess &&
+             cudaMemset(L->d_scounters, 0, (size_t)(S ? S : 1) * sizeof(int)) == cudaSuccess;
+    }
     if (!ok) {
         const cudaError_t e = cudaGetLastError();
         free_layer(L);

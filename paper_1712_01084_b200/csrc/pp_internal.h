@@ -24,6 +24,27 @@ static_assert(sizeof(WorkItem) == 32, "WorkItem is read as two 16-byte words");
 constexpr int kMaxGroupBatch = 32;   // batch columns one streaming-kernel launch handles
 constexpr int kMaxRunColumns = 2048;  // pivoted columns (tiles x B) one work item may span
 
+// --- persistent streaming kernel (batch <= kStreamMaxBatch) ---------------------------------
+// A strip is one row-group of one block-row: its fragments are contiguous in the value array
+// and the strips follow each other in (block-row, row-group) order, so the whole layer is one
+// linear fragment sequence.  The plan cuts that sequence into one contiguous range per CTA.
+struct CtaDesc {
+    int32_t p_begin, p_end;   // fragment positions [p_begin, p_end) streamed by this CTA
+    int32_t s_first, s_count; // strips this CTA contributes to (consecutive); the first/last may be shared
+};
+struct StripInfo {
+    int32_t first_cta;        // first CTA that lists this strip
+    int32_t nparts;           // CTAs that list it (1: no cross-CTA reduction)
+    int32_t slot_base;        // first global partial-sum slot (valid when nparts > 1)
+    int32_t pad;
+};
+static_assert(sizeof(CtaDesc) == 16 && sizeof(StripInfo) == 16, "read as 16-byte words");
+constexpr int kStreamWarps = 16;          // warps per CTA
+constexpr int kStreamMaxStrips = 48;      // strips one CTA may list
+constexpr int kStreamSegSlots = kStreamMaxStrips + kStreamWarps;   // (strip, warp) partial slots in shared memory
+constexpr int kStreamMaxBatch = 8;
+extern int g_use_stream;
+
 // Geometry of the fragment layout for a (dtype, B) pair.
 struct FragGeom {
     int rg_rows;   // rows covered by one fragment (row-group height)
@@ -53,6 +74,12 @@ struct pp_packed {
     std::vector<float> bias_piv;
     std::vector<unsigned char> values;                       // fragment-ordered tile values
     std::vector<pp::WorkItem> items;
+    // plan of the persistent streaming kernel
+    std::vector<int32_t> strip_start;   // [S+1] fragment position of each strip
+    std::vector<int32_t> xoff;          // [F] per fragment: element offset of its columns in the pivoted x
+    std::vector<pp::CtaDesc> cta_desc;
+    std::vector<pp::StripInfo> strip_info;
+    int stream_slots;
     int max_item_tiles;
     int n_slots;
     bool has_bias;

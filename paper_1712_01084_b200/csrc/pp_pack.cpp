@@ -8,10 +8,17 @@
 
 #include "pp_internal.h"
 
+namespace pp {
+int g_use_stream = 1;      // 0: the API never picks the persistent kernel
+}
+
 namespace {
 
 int g_target_kib = 32;     // tile-value kilobytes per work item
 int g_min_items = 296;     // the splitter keeps halving the run length until it has this many items
+int g_stream_ctas = 296;   // CTAs of the persistent kernel (2 per SM on a 148-SM part)
+int g_stream_min_frags = 128;  // fewer CTAs are used rather than giving one less than this many fragments
+int g_stream_snap_pct = 25;    // a CTA boundary within this % of a CTA's share of a strip boundary moves onto it
 
 bool is_bijection(const int32_t* p, int64_t n) {
     std::vector<unsigned char> seen((size_t)n, 0);
@@ -88,6 +95,82 @@ void build_items(pp_packed* p) {
     }
 }
 
+// Plan of the persistent kernel: strips, per-fragment x offsets, one fragment range per CTA.
+void build_stream_plan(pp_packed* p) {
+    const pp::FragGeom g = pp::frag_geom(p->wdtype, p->B);
+    const int S = p->Mb * g.n_rg;
+    p->strip_start.assign((size_t)S + 1, 0);
+    for (int s = 0; s < S; ++s) {
+        const int br = s / g.n_rg;
+        p->strip_start[(size_t)s + 1] = p->strip_start[(size_t)s] + (p->row_ptr[(size_t)br + 1] - p->row_ptr[(size_t)br]) * g.fpt;
+    }
+    const int64_t F = p->strip_start[(size_t)S];
+    p->xoff.resize((size_t)F);
+    for (int s = 0; s < S; ++s) {
+        const int br = s / g.n_rg;
+        const int k = p->row_ptr[(size_t)br + 1] - p->row_ptr[(size_t)br];
+        for (int j = 0; j < k; ++j)
+            for (int f = 0; f < g.fpt; ++f)
+                p->xoff[(size_t)p->strip_start[(size_t)s] + (size_t)j * g.fpt + f] =
+                    p->tile_col[(size_t)p->col_ptr[(size_t)br] + j] * p->B + f * g.kf;
+    }
+
+    // CTA boundaries as (strip, offset) pairs, offset in [0, len); (S, 0) is the end.
+    struct Bnd { int s, off; };
+    auto less = [](const Bnd& a, const Bnd& b) { return a.s < b.s || (a.s == b.s && a.off < b.off); };
+    int64_t G = std::min<int64_t>(g_stream_ctas, F / std::max(1, g_stream_min_frags));
+    G = std::max<int64_t>(G, 1);
+    const int64_t share = (F + G - 1) / G;
+    const int64_t tol = share * g_stream_snap_pct / 100;
+    std::vector<Bnd> bnd;
+    bnd.push_back({0, 0});
+    for (int64_t c = 1; c < G; ++c) {
+        const int64_t pos = F * c / G;
+        // non-empty strip containing pos
+        int s = (int)(std::upper_bound(p->strip_start.begin(), p->strip_start.end(), (int32_t)pos) -
+                      p->strip_start.begin()) - 1;
+        if (s >= S) continue;
+        int64_t off = pos - p->strip_start[(size_t)s];
+        const int64_t len = p->strip_start[(size_t)s + 1] - p->strip_start[(size_t)s];
+        Bnd b;
+        if (off <= tol && off <= len - off) b = {s, 0};
+        else if (len - off <= tol) b = {s + 1, 0};
+        else b = {s, (int)off};
+        if (less(bnd.back(), b)) bnd.push_back(b);
+    }
+    const Bnd end{S, 0};
+    while (bnd.size() > 1 && !less(bnd.back(), end)) bnd.pop_back();
+    // no CTA may list more than kStreamMaxStrips strips
+    std::vector<Bnd> cut;
+    for (size_t c = 0; c < bnd.size(); ++c) {
+        const Bnd b0 = bnd[c], b1 = c + 1 < bnd.size() ? bnd[c + 1] : end;
+        cut.push_back(b0);
+        const int listed = b1.s - b0.s + (b1.off > 0 ? 1 : 0);
+        for (int q = pp::kStreamMaxStrips; q < listed; q += pp::kStreamMaxStrips) cut.push_back({b0.s + q, 0});
+    }
+    p->cta_desc.clear();
+    p->strip_info.assign((size_t)S, pp::StripInfo{-1, 0, 0, 0});
+    for (size_t c = 0; c < cut.size(); ++c) {
+        const Bnd b0 = cut[c], b1 = c + 1 < cut.size() ? cut[c + 1] : end;
+        pp::CtaDesc d;
+        d.p_begin = p->strip_start[(size_t)b0.s] + b0.off;
+        d.p_end = p->strip_start[(size_t)b1.s] + b1.off;
+        d.s_first = b0.s;
+        d.s_count = b1.s - b0.s + (b1.off > 0 ? 1 : 0);
+        for (int s = d.s_first; s < d.s_first + d.s_count; ++s) {
+            pp::StripInfo& si = p->strip_info[(size_t)s];
+            if (si.nparts == 0) si.first_cta = (int)c;
+            si.nparts++;
+        }
+        p->cta_desc.push_back(d);
+    }
+    p->stream_slots = 0;
+    for (int s = 0; s < S; ++s) {
+        pp::StripInfo& si = p->strip_info[(size_t)s];
+        if (si.nparts > 1) { si.slot_base = p->stream_slots; p->stream_slots += si.nparts; }
+    }
+}
+
 }  // namespace
 
 extern "C" {
@@ -109,6 +192,10 @@ const char* pp_status_string(pp_status_t s) {
 pp_status_t pp_set_tuning(int key, int value) {
     if (key == 0 && value >= 1) { g_target_kib = value; return PP_OK; }
     if (key == 1 && value >= 0) { g_min_items = value; return PP_OK; }
+    if (key == 2 && value >= 1) { g_stream_ctas = value; return PP_OK; }
+    if (key == 3 && value >= 1) { g_stream_min_frags = value; return PP_OK; }
+    if (key == 4 && value >= 0 && value <= 50) { g_stream_snap_pct = value; return PP_OK; }
+    if (key == 5 && (value == 0 || value == 1)) { pp::g_use_stream = value; return PP_OK; }
     return PP_ERR_INVALID_ARG;
 }
 
@@ -202,6 +289,7 @@ pp_status_t pp_pack_create(pp_packed_t** out, int M, int N, int B, const int32_t
             if (real && bias) p->bias_piv[(size_t)i] = bias[row_perm[i]];
         }
         build_items(p);
+        build_stream_plan(p);
     } catch (const std::bad_alloc&) {
         delete p;
         return PP_ERR_ALLOC;
@@ -215,8 +303,10 @@ pp_status_t pp_pack_destroy(pp_packed_t* p) {
     return PP_OK;
 }
 
-pp_status_t pp_pack_info(const pp_packed_t* p, int64_t out[8]) {
+pp_status_t pp_pack_info(const pp_packed_t* p, int64_t out[12]) {
     if (!p || !out) return PP_ERR_INVALID_ARG;
+    out[8] = (int64_t)p->strip_start.size() - 1; out[9] = (int64_t)p->xoff.size();
+    out[10] = (int64_t)p->cta_desc.size(); out[11] = p->stream_slots;
     out[0] = p->Mb; out[1] = p->Nb; out[2] = p->T; out[3] = (int64_t)p->tile_col.size();
     out[4] = (int64_t)p->items.size(); out[5] = (int64_t)p->values.size();
     out[6] = p->max_item_tiles; out[7] = p->n_slots;
@@ -237,6 +327,10 @@ pp_status_t pp_pack_get(const pp_packed_t* p, int which, void* dst, int64_t byte
         case 6: src = p->values.data(); n = p->values.size(); break;
         case 7: src = p->items.data(); n = p->items.size() * sizeof(pp::WorkItem); break;
         case 8: src = p->inv_row_perm.data(); n = p->inv_row_perm.size() * 4; break;
+        case 9: src = p->strip_start.data(); n = p->strip_start.size() * 4; break;
+        case 10: src = p->xoff.data(); n = p->xoff.size() * 4; break;
+        case 11: src = p->cta_desc.data(); n = p->cta_desc.size() * sizeof(pp::CtaDesc); break;
+        case 12: src = p->strip_info.data(); n = p->strip_info.size() * sizeof(pp::StripInfo); break;
         default: return PP_ERR_INVALID_ARG;
     }
     if ((size_t)bytes < n) return PP_ERR_INVALID_ARG;

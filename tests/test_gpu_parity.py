@@ -68,12 +68,36 @@ def _run_and_check(pb, lay, x, act, what=""):
 @pytest.mark.parametrize("dtype", [np.float32, np.float16])
 @pytest.mark.parametrize("B", [16, 32, 64])
 @pytest.mark.parametrize("batch", [1, 2, 3, 8, 9, 17, 33])
-def test_small_layers(pb, dtype, B, batch):
-    """Ragged M and N, unbalanced block-rows, one block-row without tiles, several tiles and a ragged tail."""
-    lay = _rand_layer(100 + B + batch, 5 * B - 3, 9 * B - 7, B, dtype, density=0.45, empty_rows=(2,))
-    x = np.random.default_rng(batch).uniform(-1, 1, (batch, lay.N)).astype(dtype)
-    for act in (0, 1):
-        _run_and_check(pb, lay, x, act, f"{dtype.__name__} B={B} batch={batch} act={act}")
+@pytest.mark.parametrize("persistent", [1, 0])
+def test_small_layers(pb, dtype, B, batch, persistent):
+    """Ragged M and N, unbalanced block-rows, one block-row without tiles, several tiles and a ragged tail;
+    through the persistent kernel (batch <= 8) and through the chunked kernel."""
+    if persistent and batch > 8:
+        pytest.skip("batch > 8 always takes the chunked kernel")
+    pb.pp_set_tuning(5, persistent)
+    try:
+        lay = _rand_layer(100 + B + batch, 5 * B - 3, 9 * B - 7, B, dtype, density=0.45, empty_rows=(2,))
+        x = np.random.default_rng(batch).uniform(-1, 1, (batch, lay.N)).astype(dtype)
+        for act in (0, 1):
+            _run_and_check(pb, lay, x, act, f"{dtype.__name__} B={B} batch={batch} act={act}")
+    finally:
+        pb.pp_set_tuning(5, 1)
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("ctas,min_frags,snap", [(296, 1, 0), (5, 1, 0), (37, 4, 50), (2000, 1, 25)])
+def test_persistent_kernel_partitions(pb, dtype, ctas, min_frags, snap):
+    """CTA ranges that cut strips in the middle (cross-CTA partial sums), that snap to strip
+    boundaries, fewer CTAs than strips and more CTAs than SMs can hold at once."""
+    pb.pp_set_tuning(2, ctas); pb.pp_set_tuning(3, min_frags); pb.pp_set_tuning(4, snap)
+    try:
+        for B in (16, 64):
+            lay = _rand_layer(11 + B, 9 * B - 3, 20 * B - 7, B, dtype, density=0.5, empty_rows=(0, 4))
+            for batch in (1, 3, 8):
+                x = np.random.default_rng(batch).uniform(-1, 1, (batch, lay.N)).astype(dtype)
+                _run_and_check(pb, lay, x, 1, f"ctas={ctas} B={B} batch={batch}")
+    finally:
+        pb.pp_set_tuning(2, 296); pb.pp_set_tuning(3, 128); pb.pp_set_tuning(4, 25)
 
 
 @pytest.mark.parametrize("dtype", [np.float32, np.float16])
@@ -92,10 +116,11 @@ def test_split_block_rows(pb, dtype, target_kib):
 
 @pytest.mark.parametrize("dtype", [np.float32, np.float16])
 @pytest.mark.parametrize("B", [16, 32, 64])
-def test_integer_data_is_bit_exact(pb, dtype, B):
+@pytest.mark.parametrize("persistent", [1, 0])
+def test_integer_data_is_bit_exact(pb, dtype, B, persistent):
     """Small-integer weights, inputs and bias: all sums exact, so any index or
     permutation slip shows up as a bit difference."""
-    pb.pp_set_tuning(0, 2)
+    pb.pp_set_tuning(0, 2); pb.pp_set_tuning(5, persistent); pb.pp_set_tuning(2, 23); pb.pp_set_tuning(3, 1)
     try:
         lay = _rand_layer(50 + B, 4 * B - 1, 6 * B - 5, B, dtype, density=0.5, integer=True)
         for batch in (1, 4, 11):
@@ -107,7 +132,7 @@ def test_integer_data_is_bit_exact(pb, dtype, B):
                 assert np.array_equal(y.astype(np.float64), y_ref)
             L.close()
     finally:
-        pb.pp_set_tuning(0, 32)
+        pb.pp_set_tuning(0, 32); pb.pp_set_tuning(5, 1); pb.pp_set_tuning(2, 296); pb.pp_set_tuning(3, 128)
 
 
 def test_identity_perms_density_one(pb):
@@ -119,23 +144,27 @@ def test_identity_perms_density_one(pb):
     assert np.max(np.abs(y - ref)) < 1e-5
 
 
-def test_deterministic_and_canaries(pb):
+@pytest.mark.parametrize("persistent", [1, 0])
+def test_deterministic_and_canaries(pb, persistent):
     """Same inputs twice -> identical bits; memory around y is untouched."""
-    pb.pp_set_tuning(0, 2)
+    pb.pp_set_tuning(0, 2); pb.pp_set_tuning(5, persistent); pb.pp_set_tuning(4, 0)
     try:
         lay = _rand_layer(9, 777, 1111, 32, np.float16, density=0.5)
         L = pb.Layer.from_synth(lay)
     finally:
-        pb.pp_set_tuning(0, 32)
+        pb.pp_set_tuning(0, 32); pb.pp_set_tuning(4, 25)
     x = _dev(np.random.default_rng(1).uniform(-1, 1, (3, lay.N)).astype(np.float16))
     pad = 64
     buf = torch.full((3 * lay.M + 2 * pad,), 12345.0, dtype=torch.float32, device="cuda")
     out = buf[pad:pad + 3 * lay.M].view(3, lay.M)
     y1 = pb.pp_forward(L, x, 1, out=out).clone()
     assert torch.all(buf[:pad] == 12345.0) and torch.all(buf[-pad:] == 12345.0)
-    for _ in range(5):
-        y2 = pb.pp_forward(L, x, 1)
-        assert torch.equal(y1, y2)
+    try:
+        for _ in range(5):
+            y2 = pb.pp_forward(L, x, 1)
+            assert torch.equal(y1, y2)
+    finally:
+        pb.pp_set_tuning(5, 1)
     L.close()
 
 

@@ -268,3 +268,132 @@ def test_packed_walk_matches_oracle(dtype, B):
     y, _, a = po.layer_forward(lay, x.astype(np.float64), act=1)
     assert not np.any(np.isnan(got))
     assert np.all(np.abs(got - y[0]) <= 1e-12 * (a[0] + 1))
+
+
+# ------------------------------------------------ persistent kernel's plan, walked like the kernel
+def _emulate_stream(pk, x, act, dtype):
+    """Follow the persistent kernel: per-CTA fragment ranges, 16 warps with equal shares, partial
+    sums parked per (strip, warp), per-strip sums in warp order, cross-CTA sums in CTA order."""
+    NW, MAXS = 16, 48
+    B = pk.B
+    f16 = dtype == np.float16
+    RG = 16 if f16 else min(B, 32)
+    vals = pk.get("values").view(dtype)
+    F = pk.n_frags
+    vals = vals.reshape(F, 32, 8 if f16 else 4)
+    xoff, sstart = pk.get("xoff"), pk.get("strip_start")
+    ctas, sinfo = pk.get("cta_desc"), pk.get("strip_info")
+    gather, scatter, bias = pk.get("gather_idx"), pk.get("scatter_idx"), pk.get("bias_piv")
+    xs = np.where(gather >= 0, x[np.maximum(gather, 0)], 0.0)
+    S = pk.n_strips
+    assert sstart[S] == F and S == pk.Mb * (B // RG)
+    covered = np.zeros(F, dtype=int)
+    gpart = {}
+    y_piv = np.full(S * RG, np.nan)
+    listed = np.zeros(S, dtype=int)
+    for c, (pb_, pe, s_first, s_count) in enumerate(ctas):
+        assert 1 <= s_count <= MAXS and 0 <= s_first and s_first + s_count <= S and pb_ <= pe
+        n = pe - pb_
+        wb = [pb_ + (n * w) // NW for w in range(NW + 1)]
+        loc = sstart[s_first:s_first + s_count + 1]
+        park = {}
+        for w in range(NW):
+            if wb[w] >= wb[w + 1]:
+                continue
+            ls = 0
+            while ls + 1 < s_count and loc[ls + 1] <= wb[w]:
+                ls += 1
+            seg_end = min(wb[w + 1], loc[ls + 1])
+            acc = np.zeros(RG)
+            for p in range(wb[w], wb[w + 1]):
+                if p == seg_end:
+                    assert ls + w not in park
+                    park[ls + w] = acc
+                    acc = np.zeros(RG)
+                    ls += 1
+                    while loc[ls + 1] <= p:
+                        ls += 1
+                    seg_end = min(wb[w + 1], loc[ls + 1])
+                assert loc[ls] <= p < loc[ls + 1]
+                covered[p] += 1
+                xo = xoff[p]
+                assert 0 <= xo and xo + (16 if f16 else (8 if RG == 16 else 4)) <= pk.Nb * B
+                for lane in range(32):
+                    wv = vals[p, lane].astype(np.float64)
+                    if f16:
+                        g, t = lane // 4, lane % 4
+                        k0 = xo + 2 * t
+                        acc[g] += wv[0] * xs[k0] + wv[1] * xs[k0 + 1] + wv[4] * xs[k0 + 8] + wv[5] * xs[k0 + 9]
+                        acc[g + 8] += wv[2] * xs[k0] + wv[3] * xs[k0 + 1] + wv[6] * xs[k0 + 8] + wv[7] * xs[k0 + 9]
+                    else:
+                        k0 = xo + (lane // RG) * 4
+                        acc[lane % RG] += float(np.dot(wv, xs[k0:k0 + 4]))
+            assert ls + w not in park and ls + w < MAXS + NW
+            park[ls + w] = acc
+        for ls in range(s_count):
+            s = s_first + ls
+            listed[s] += 1
+            lo, hi = max(loc[ls], pb_), min(loc[ls + 1], pe)
+            v = np.zeros(RG)
+            if lo < hi:
+                w_lo = max(w for w in range(NW) if wb[w] <= lo)
+                w_hi = max(w for w in range(NW) if wb[w] <= hi - 1)
+                for w in range(w_lo, w_hi + 1):
+                    if wb[w] < wb[w + 1]:
+                        v = v + park.pop(ls + w)
+            first_cta, nparts, slot_base, _ = sinfo[s]
+            if nparts == 1:
+                y_piv[s * RG:(s + 1) * RG] = v
+            else:
+                assert ls in (0, s_count - 1) and first_cta <= c < first_cta + nparts
+                gpart[slot_base + c - first_cta] = v
+        assert not park
+    assert np.all(covered == 1)
+    assert np.array_equal(listed, sinfo[:, 1])
+    for s in range(S):
+        first_cta, nparts, slot_base, _ = sinfo[s]
+        if nparts > 1:
+            y_piv[s * RG:(s + 1) * RG] = sum(gpart.pop(slot_base + q) for q in range(nparts))
+    assert not gpart
+    y = np.full(pk.M, np.nan)
+    for i in range(S * RG):
+        if scatter[i] >= 0:
+            v = y_piv[i] + bias[i]
+            y[scatter[i]] = max(v, 0.0) if act else v
+    return y
+
+
+@pytest.mark.parametrize("dtype,B", [(np.float32, 16), (np.float32, 32), (np.float32, 64),
+                                     (np.float16, 16), (np.float16, 32), (np.float16, 64)])
+@pytest.mark.parametrize("ctas,min_frags,snap", [(296, 128, 25), (7, 1, 0), (3, 1, 50), (1000, 1, 10)])
+def test_stream_plan_walk_matches_oracle(dtype, B, ctas, min_frags, snap):
+    pb.pp_set_tuning(2, ctas); pb.pp_set_tuning(3, min_frags); pb.pp_set_tuning(4, snap)
+    try:
+        lay = _random_layer(40 + B, 5 * B - 5, 6 * B - 2, B, dtype, density=0.5)
+        lay.tile_list = lay.tile_list[lay.tile_list[:, 0] != 1]          # block-row 1 has no tile
+        lay.tile_values = lay.tile_values[:len(lay.tile_list)]
+        pk = _pack(lay)
+    finally:
+        pb.pp_set_tuning(2, 296); pb.pp_set_tuning(3, 128); pb.pp_set_tuning(4, 25)
+    x = np.random.default_rng(1).uniform(-1, 1, lay.N).astype(dtype)
+    got = _emulate_stream(pk, x.astype(np.float64), 1, dtype)
+    y, _, a = po.layer_forward(lay, x.astype(np.float64), act=1)
+    assert not np.any(np.isnan(got))
+    assert np.all(np.abs(got - y[0]) <= 1e-12 * (a[0] + 1))
+
+
+def test_stream_plan_many_empty_strips_and_no_tiles():
+    """More strips than one CTA may list, most of them empty; and a layer without any tile."""
+    rng = np.random.default_rng(3)
+    M, N, B = 16 * 300, 64, 16
+    tl = np.array([[5, 1], [150, 0], [151, 3], [299, 2]], dtype=np.int32)
+    lay = synth.Layer(M, N, B, rng.permutation(M).astype(np.int32), rng.permutation(N).astype(np.int32), tl,
+                      rng.standard_normal((4, B, B)).astype(np.float16), rng.standard_normal(M).astype(np.float32))
+    for T in (4, 0):
+        lay.tile_list, lay.tile_values = tl[:T], lay.tile_values[:T]
+        pk = _pack(lay)
+        assert np.all(pk.get("cta_desc")[:, 3] <= 48)
+        x = rng.uniform(-1, 1, N).astype(np.float16)
+        got = _emulate_stream(pk, x.astype(np.float64), 0, np.float16)
+        y, _, a = po.layer_forward(lay, x.astype(np.float64), act=0)
+        assert np.all(np.abs(got - y[0]) <= 1e-12 * (a[0] + 1))
