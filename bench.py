@@ -306,7 +306,7 @@ def main():
                 "d2h_bytes_per_step": int(lay.M * 4), "steps": n_e2e},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                     "algorithmic_bytes_per_launch": abytes, "kernel": "gemv_f16_kernel<64,1>", "traffic": None},
+                     "algorithmic_bytes_per_launch": abytes, "kernel": "stream_f16_kernel<4>", "traffic": None},
         "clocks": clocks,
     }
 

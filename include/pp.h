@@ -168,8 +168,14 @@ pp_status_t pp_chain_forward(pp_chain_t* chain, const void* x, void* y, int batc
  * key 1: lower bound on the number of work items the splitter aims for (default 296)
  * key 2: CTAs of the persistent kernel (default 296)
  * key 3: minimum fragments per CTA of the persistent kernel (default 128)
- * key 4: snap tolerance, percent of a CTA's share, for moving CTA boundaries onto strip boundaries (default 25)
- * key 5: 0 = never use the persistent kernel, 1 = use it when batch <= 8 and x fits shared memory (default 1) */
+ * key 4: -1 (default) lets the packer choose the persistent kernel's partition; 0..100 forces an even split
+ *        over `key 2` CTAs (at least `key 3` fragments each) whose boundaries move onto a strip boundary when
+ *        closer to it than this percentage of a CTA's share
+ * key 5: 0 = never use the persistent kernel, 1 = use it when batch <= 8 and x fits shared memory (default 1)
+ * key 6: asynchronous 512-byte weight copies each warp of the persistent kernel keeps in flight: 4 (default) or 8
+ * key 7: batch 1 in the persistent kernel: 1 (default) reads x through the index array inside the multiply
+ *        loop, 0 permutes x into pivoted order in shared memory first (what batch 2..8 always do)
+ * key 8: 1 (default) launches the persistent kernel with programmatic stream serialization, 0 plainly */
 pp_status_t pp_set_tuning(int key, int value);
 
 #ifdef __cplusplus

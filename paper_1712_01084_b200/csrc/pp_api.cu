@@ -1,6 +1,7 @@
 // C entry points that own device memory: layers, forward calls, folded chains.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <new>
 #include <vector>
 
@@ -10,24 +11,32 @@
 
 struct pp_layer {
     pp_packed* pk = nullptr;       // host copy (index arrays are needed again when chains are folded)
+    // One read-only device allocation holds every packed array (small tables first, tile values
+    // last), so a forward call touches few pages; one more holds the scratch both kernels write.
+    unsigned char* d_arena = nullptr;
+    size_t arena_bytes = 0;
+    unsigned char* d_scratch = nullptr;
+    size_t scratch_bytes = 0;
+    // views into the arena
     void* d_values = nullptr;
     pp::WorkItem* d_items = nullptr;
     int32_t* d_tile_col = nullptr;
     int32_t* d_gather = nullptr;
     int32_t* d_scatter = nullptr;
     float* d_bias = nullptr;
-    float* d_partials = nullptr;
-    int* d_counters = nullptr;
-    int n_items = 0;
-    int max_item_tiles = 0;
-    // persistent streaming kernel
     int32_t* d_xoff = nullptr;
     int32_t* d_strip_start = nullptr;
     pp::CtaDesc* d_cta_desc = nullptr;
     pp::StripInfo* d_strip_info = nullptr;
-    float* d_spartials = nullptr;
-    int* d_scounters = nullptr;
+    // views into the scratch allocation
+    float* d_partials = nullptr;   // chunked kernel: [n_slots][B][kMaxGroupBatch]
+    int* d_counters = nullptr;     // chunked kernel: [Mb]
+    float* d_spartials = nullptr;  // persistent kernel: [stream_slots][rows per strip][kStreamMaxBatch]
+    int* d_scounters = nullptr;    // persistent kernel: [S]
+    int n_items = 0;
+    int max_item_tiles = 0;
     int stream_grid = 0;
+    int stream_max_rows = 0;       // most pivoted rows one CTA of the persistent plan lists
 };
 
 struct pp_chain {
@@ -50,30 +59,96 @@ bool upload(T** dst, const void* src, size_t bytes) {
 
 void free_layer(pp_layer* L) {
     if (!L) return;
-    cudaFree(L->d_values); cudaFree(L->d_items); cudaFree(L->d_tile_col); cudaFree(L->d_gather);
-    cudaFree(L->d_scatter); cudaFree(L->d_bias); cudaFree(L->d_partials); cudaFree(L->d_counters);
-    cudaFree(L->d_xoff); cudaFree(L->d_strip_start); cudaFree(L->d_cta_desc); cudaFree(L->d_strip_info);
-    cudaFree(L->d_spartials); cudaFree(L->d_scounters);
+    cudaFree(L->d_arena);
+    cudaFree(L->d_scratch);
     pp_pack_destroy(L->pk);
     delete L;
+}
+
+size_t round256(size_t n) { return (n + 255) / 256 * 256; }
+
+// Section sizes of the arena and the scratch allocation, in a fixed order.
+struct LayerLayout {
+    size_t off[10];       // cta_desc, strip_start, strip_info, scatter, bias, gather, tile_col, items, xoff, values
+    size_t arena_bytes;
+    size_t soff[4];       // partials, counters, spartials, scounters
+    size_t scratch_bytes;
+};
+
+LayerLayout layer_layout(const pp_packed* pk) {
+    const pp::FragGeom g = pp::frag_geom(pk->wdtype, pk->B);
+    const size_t esz = pk->wdtype == PP_F16 ? 2 : 4;
+    const size_t S = pk->strip_info.size();
+    const size_t F = (size_t)pk->T * g.n_rg * g.fpt;
+    const size_t sz[10] = {pk->cta_desc.size() * sizeof(pp::CtaDesc), (S + 1) * 4, S * sizeof(pp::StripInfo),
+                           (size_t)pk->Mpad * 4, (size_t)pk->Mpad * 4, (size_t)pk->Npad * 4, pk->tile_col.size() * 4,
+                           pk->items.size() * sizeof(pp::WorkItem), F * 4, (size_t)pk->T * pk->B * pk->B * esz};
+    LayerLayout lo;
+    size_t pos = 0;
+    for (int i = 0; i < 10; ++i) { lo.off[i] = pos; pos += round256(sz[i]); }
+    lo.arena_bytes = pos ? pos : 256;
+    const size_t ssz[4] = {(size_t)pk->n_slots * pk->B * pp::kMaxGroupBatch * 4, (size_t)pk->Mb * 4,
+                           (size_t)pk->stream_slots * g.rg_rows * pp::kStreamMaxBatch * 4, (S ? S : 1) * 4};
+    pos = 0;
+    for (int i = 0; i < 4; ++i) { lo.soff[i] = pos; pos += round256(ssz[i]); }
+    lo.scratch_bytes = pos;
+    return lo;
+}
+
+// Allocate both device blocks and point the views into them.
+bool alloc_layer(pp_layer* L, const LayerLayout& lo) {
+    if (cudaMalloc(reinterpret_cast<void**>(&L->d_arena), lo.arena_bytes) != cudaSuccess) return false;
+    if (cudaMalloc(reinterpret_cast<void**>(&L->d_scratch), lo.scratch_bytes) != cudaSuccess) return false;
+    if (cudaMemset(L->d_scratch, 0, lo.scratch_bytes) != cudaSuccess) return false;
+    // the persistent kernel's exchange slots rest at an all-ones NaN pattern
+    if (cudaMemset(L->d_scratch + lo.soff[2], 0xff, lo.soff[3] - lo.soff[2]) != cudaSuccess) return false;
+    L->arena_bytes = lo.arena_bytes;
+    L->scratch_bytes = lo.scratch_bytes;
+    unsigned char* a = L->d_arena;
+    L->d_cta_desc = reinterpret_cast<pp::CtaDesc*>(a + lo.off[0]);
+    L->d_strip_start = reinterpret_cast<int32_t*>(a + lo.off[1]);
+    L->d_strip_info = reinterpret_cast<pp::StripInfo*>(a + lo.off[2]);
+    L->d_scatter = reinterpret_cast<int32_t*>(a + lo.off[3]);
+    L->d_bias = reinterpret_cast<float*>(a + lo.off[4]);
+    L->d_gather = reinterpret_cast<int32_t*>(a + lo.off[5]);
+    L->d_tile_col = reinterpret_cast<int32_t*>(a + lo.off[6]);
+    L->d_items = reinterpret_cast<pp::WorkItem*>(a + lo.off[7]);
+    L->d_xoff = reinterpret_cast<int32_t*>(a + lo.off[8]);
+    L->d_values = a + lo.off[9];
+    unsigned char* sc = L->d_scratch;
+    L->d_partials = reinterpret_cast<float*>(sc + lo.soff[0]);
+    L->d_counters = reinterpret_cast<int*>(sc + lo.soff[1]);
+    L->d_spartials = reinterpret_cast<float*>(sc + lo.soff[2]);
+    L->d_scounters = reinterpret_cast<int*>(sc + lo.soff[3]);
+    return true;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Enqueue one layer in groups of batch columns.
-pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_elt, void* y, int ldy,
+pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_len, int x_elt, void* y, int ldy,
                       int out_mode, int batch, pp_act_t act, cudaStream_t stream) {
     const pp_packed* pk = L->pk;
-    if (pp::g_use_stream && batch <= pp::kStreamMaxBatch &&
-        pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, batch) <= pp::kStreamSmemLimit) {
+    int stage_mode = -1;
+    if (pp::g_use_stream && batch <= pp::kStreamMaxBatch) {
+        const bool rows_aligned = aligned16(x) && (batch == 1 || ((size_t)ldx * x_elt) % 16 == 0);
+        const int fast = gather ? (batch == 1 && pp::g_stage_direct ? 3 : 1) : 2;
+        if (rows_aligned && pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, fast) <= pp::kStreamSmemLimit)
+            stage_mode = fast;
+        else if (pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, 0) <= pp::kStreamSmemLimit)
+            stage_mode = 0;
+    }
+    if (stage_mode >= 0) {
         pp::StreamArgs s{};
+        s.stage_mode = stage_mode;
         s.values = L->d_values; s.xoff = L->d_xoff; s.strip_start = L->d_strip_start;
         s.cta_desc = L->d_cta_desc; s.strip_info = L->d_strip_info;
         s.gather_idx = gather; s.scatter_idx = L->d_scatter; s.bias_piv = L->d_bias;
         s.x = x; s.y = y; s.partials = L->d_spartials; s.counters = L->d_scounters;
-        s.ldx = ldx; s.ldy = ldy; s.x_limit = pk->N; s.n_pad = pk->Npad; s.batch = batch;
+        s.ldx = ldx; s.ldy = ldy; s.x_limit = pk->N; s.n_pad = pk->Npad; s.x_len = x_len; s.max_rows = L->stream_max_rows; s.batch = batch;
         s.act = (int)act; s.out_mode = out_mode;
-        return pp::launch_stream(pk->wdtype, pk->B, s, L->stream_grid, stream) == cudaSuccess ? PP_OK : PP_ERR_CUDA;
+        return pp::launch_stream(pk->wdtype, pk->B, s, pk->cta_desc.data(), L->stream_grid, stream) == cudaSuccess
+                   ? PP_OK : PP_ERR_CUDA;
     }
     pp::GemvArgs a{};
     a.values = L->d_values; a.items = L->d_items; a.tile_col = L->d_tile_col;
@@ -111,30 +186,21 @@ pp_status_t pp_layer_create(pp_layer_t** out, int M, int N, int B, const int32_t
     L->pk = pk;
     L->n_items = (int)pk->items.size();
     L->max_item_tiles = pk->max_item_tiles;
-    bool ok = upload(&L->d_values, pk->values.data(), pk->values.size()) &&
-              upload(&L->d_items, pk->items.data(), pk->items.size() * sizeof(pp::WorkItem)) &&
-              upload(&L->d_tile_col, pk->tile_col.data(), pk->tile_col.size() * 4) &&
-              upload(&L->d_gather, pk->gather_idx.data(), pk->gather_idx.size() * 4) &&
-              upload(&L->d_scatter, pk->scatter_idx.data(), pk->scatter_idx.size() * 4) &&
-              upload(&L->d_bias, pk->bias_piv.data(), pk->bias_piv.size() * 4);
+    L->stream_grid = (int)pk->cta_desc.size();
+    for (const pp::CtaDesc& c : pk->cta_desc)
+        L->stream_max_rows = std::max(L->stream_max_rows, c.s_count * pp::frag_geom(wdtype, B).rg_rows);
+    const LayerLayout lo = layer_layout(pk);
+    bool ok = alloc_layer(L, lo);
     if (ok) {
-        const size_t pbytes = (size_t)pk->n_slots * B * pp::kMaxGroupBatch * sizeof(float);
-        ok = cudaMalloc(reinterpret_cast<void**>(&L->d_partials), pbytes ? pbytes : 16) == cudaSuccess &&
-             cudaMalloc(reinterpret_cast<void**>(&L->d_counters), (size_t)pk->Mb * sizeof(int)) == cudaSuccess &&
-             cudaMemset(L->d_counters, 0, (size_t)pk->Mb * sizeof(int)) == cudaSuccess;
-    }
-    if (ok) {
-        const int S = (int)pk->strip_info.size();
-        const int rg = pp::frag_geom(wdtype, B).rg_rows;
-        const size_t sp = (size_t)pk->stream_slots * rg * pp::kStreamMaxBatch * sizeof(float);
-        L->stream_grid = (int)pk->cta_desc.size();
-        ok = upload(&L->d_xoff, pk->xoff.data(), pk->xoff.size() * 4) &&
-             upload(&L->d_strip_start, pk->strip_start.data(), pk->strip_start.size() * 4) &&
-             upload(&L->d_cta_desc, pk->cta_desc.data(), pk->cta_desc.size() * sizeof(pp::CtaDesc)) &&
-             upload(&L->d_strip_info, pk->strip_info.data(), pk->strip_info.size() * sizeof(pp::StripInfo)) &&
-             cudaMalloc(reinterpret_cast<void**>(&L->d_spartials), sp ? sp : 16) == cudaSuccess &&
-             cudaMalloc(reinterpret_cast<void**>(&L->d_scounters), (size_t)(S ? S : 1) * sizeof(int)) == cudaSuccess &&
-             cudaMemset(L->d_scounters, 0, (size_t)(S ? S : 1) * sizeof(int)) == cudaSuccess;
+        const void* src[10] = {pk->cta_desc.data(), pk->strip_start.data(), pk->strip_info.data(),
+                               pk->scatter_idx.data(), pk->bias_piv.data(), pk->gather_idx.data(),
+                               pk->tile_col.data(), pk->items.data(), pk->xoff.data(), pk->values.data()};
+        const size_t n[10] = {pk->cta_desc.size() * sizeof(pp::CtaDesc), pk->strip_start.size() * 4,
+                              pk->strip_info.size() * sizeof(pp::StripInfo), pk->scatter_idx.size() * 4,
+                              pk->bias_piv.size() * 4, pk->gather_idx.size() * 4, pk->tile_col.size() * 4,
+                              pk->items.size() * sizeof(pp::WorkItem), pk->xoff.size() * 4, pk->values.size()};
+        for (int i = 0; i < 10 && ok; ++i)
+            ok = n[i] == 0 || cudaMemcpy(L->d_arena + lo.off[i], src[i], n[i], cudaMemcpyHostToDevice) == cudaSuccess;
     }
     if (!ok) {
         const cudaError_t e = cudaGetLastError();
@@ -158,37 +224,11 @@ pp_status_t pp_layer_clone(pp_layer_t** out, const pp_layer_t* src) {
     L->pk = pk;
     L->n_items = src->n_items;
     L->max_item_tiles = src->max_item_tiles;
-    const size_t esz = pk->wdtype == PP_F16 ? 2 : 4;
-    const size_t vbytes = (size_t)pk->T * pk->B * pk->B * esz;
-    const size_t pbytes = (size_t)pk->n_slots * pk->B * pp::kMaxGroupBatch * sizeof(float);
-    auto dup = [](auto** dst, const void* s, size_t bytes) {
-        *dst = nullptr;
-        if (cudaMalloc(reinterpret_cast<void**>(dst), bytes ? bytes : 16) != cudaSuccess) return false;
-        return bytes == 0 || cudaMemcpy(*dst, s, bytes, cudaMemcpyDeviceToDevice) == cudaSuccess;
-    };
-    bool ok = dup(&L->d_values, src->d_values, vbytes) &&
-              dup(&L->d_items, src->d_items, pk->items.size() * sizeof(pp::WorkItem)) &&
-              dup(&L->d_tile_col, src->d_tile_col, pk->tile_col.size() * 4) &&
-              dup(&L->d_gather, src->d_gather, pk->gather_idx.size() * 4) &&
-              dup(&L->d_scatter, src->d_scatter, pk->scatter_idx.size() * 4) &&
-              dup(&L->d_bias, src->d_bias, pk->bias_piv.size() * 4) &&
-              cudaMalloc(reinterpret_cast<void**>(&L->d_partials), pbytes ? pbytes : 16) == cudaSuccess &&
-              cudaMalloc(reinterpret_cast<void**>(&L->d_counters), (size_t)pk->Mb * sizeof(int)) == cudaSuccess &&
-              cudaMemset(L->d_counters, 0, (size_t)pk->Mb * sizeof(int)) == cudaSuccess;
-    if (ok) {
-        const int S = (int)pk->strip_info.size();
-        const pp::FragGeom g = pp::frag_geom(pk->wdtype, pk->B);
-        const size_t F = (size_t)pk->T * g.n_rg * g.fpt;
-        const size_t sp = (size_t)pk->stream_slots * g.rg_rows * pp::kStreamMaxBatch * sizeof(float);
-        L->stream_grid = src->stream_grid;
-        ok = dup(&L->d_xoff, src->d_xoff, F * 4) &&
-             dup(&L->d_strip_start, src->d_strip_start, pk->strip_start.size() * 4) &&
-             dup(&L->d_cta_desc, src->d_cta_desc, pk->cta_desc.size() * sizeof(pp::CtaDesc)) &&
-             dup(&L->d_strip_info, src->d_strip_info, pk->strip_info.size() * sizeof(pp::StripInfo)) &&
-             cudaMalloc(reinterpret_cast<void**>(&L->d_spartials), sp ? sp : 16) == cudaSuccess &&
-             cudaMalloc(reinterpret_cast<void**>(&L->d_scounters), (size_t)(S ? S : 1) * sizeof(int)) == cudaSuccess &&
-             cudaMemset(L->d_scounters, 0, (size_t)(S ? S : 1) * sizeof(int)) == cudaSuccess;
-    }
+    L->stream_grid = src->stream_grid;
+    L->stream_max_rows = src->stream_max_rows;
+    const LayerLayout lo = layer_layout(pk);
+    const bool ok = lo.arena_bytes == src->arena_bytes && alloc_layer(L, lo) &&
+                    cudaMemcpy(L->d_arena, src->d_arena, lo.arena_bytes, cudaMemcpyDeviceToDevice) == cudaSuccess;
     if (!ok) {
         const cudaError_t e = cudaGetLastError();
         free_layer(L);
@@ -208,7 +248,7 @@ pp_status_t pp_forward(pp_layer_t* L, const void* x, void* y, int batch, pp_act_
     if (act != PP_ACT_IDENTITY && act != PP_ACT_RELU) return PP_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(y)) return PP_ERR_INVALID_ARG;
     const pp_packed* pk = L->pk;
-    return run_layer(L, L->d_gather, x, pk->N, pk->wdtype == PP_F16 ? 2 : 4, y, pk->M, pp::OUT_SCATTER_F32,
+    return run_layer(L, L->d_gather, x, pk->N, pk->N, pk->wdtype == PP_F16 ? 2 : 4, y, pk->M, pp::OUT_SCATTER_F32,
                      batch, act, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -271,12 +311,13 @@ pp_status_t pp_chain_forward(pp_chain_t* C, const void* x, void* y, int batch, v
         const int x_elt = pk->wdtype == PP_F16 ? 2 : 4;
         const int32_t* gather = l == 0 ? L->d_gather : C->d_q[(size_t)l];
         const int ldx = l == 0 ? pk->N : C->layers[(size_t)l - 1]->pk->Mpad;
+        const int x_len = ldx;      // the folded map names positions of the producer's padded pivoted output
         pp_status_t st;
         if (l == n - 1) {
-            st = run_layer(L, gather, cur, ldx, x_elt, y, pk->M, pp::OUT_SCATTER_F32, batch, C->acts[(size_t)l], stream);
+            st = run_layer(L, gather, cur, ldx, x_len, x_elt, y, pk->M, pp::OUT_SCATTER_F32, batch, C->acts[(size_t)l], stream);
         } else {
             const bool next_f16 = C->layers[(size_t)l + 1]->pk->wdtype == PP_F16;
-            st = run_layer(L, gather, cur, ldx, x_elt, C->d_inter[(size_t)l], pk->Mpad,
+            st = run_layer(L, gather, cur, ldx, x_len, x_elt, C->d_inter[(size_t)l], pk->Mpad,
                            next_f16 ? pp::OUT_PIVOTED_F16 : pp::OUT_PIVOTED_F32, batch, C->acts[(size_t)l], stream);
             cur = C->d_inter[(size_t)l];
         }

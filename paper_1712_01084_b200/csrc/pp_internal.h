@@ -44,6 +44,7 @@ constexpr int kStreamMaxStrips = 48;      // strips one CTA may list
 constexpr int kStreamSegSlots = kStreamMaxStrips + kStreamWarps;   // (strip, warp) partial slots in shared memory
 constexpr int kStreamMaxBatch = 8;
 extern int g_use_stream;
+extern int g_stage_direct;   // batch 1: read x through the index array instead of permuting it first
 
 // Geometry of the fragment layout for a (dtype, B) pair.
 struct FragGeom {

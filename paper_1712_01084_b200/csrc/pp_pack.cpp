@@ -10,6 +10,9 @@
 
 namespace pp {
 int g_use_stream = 1;      // 0: the API never picks the persistent kernel
+int g_stage_direct = 1;    // 0: batch 1 also materialises the pivoted x in shared memory
+extern int g_stream_depth; // weight-ring slots per warp of the persistent kernel (pp_stream.cu)
+extern int g_stream_pdl;   // programmatic dependent launch of the persistent kernel (pp_stream.cu)
 }
 
 namespace {
@@ -17,8 +20,10 @@ namespace {
 int g_target_kib = 32;     // tile-value kilobytes per work item
 int g_min_items = 296;     // the splitter keeps halving the run length until it has this many items
 int g_stream_ctas = 296;   // CTAs of the persistent kernel (2 per SM on a 148-SM part)
+int g_stream_sms = 148;    // SMs the partition is balanced for
 int g_stream_min_frags = 128;  // fewer CTAs are used rather than giving one less than this many fragments
-int g_stream_snap_pct = 25;    // a CTA boundary within this % of a CTA's share of a strip boundary moves onto it
+int g_stream_snap_pct = -1;    // >= 0: manual partition, a CTA boundary within this % of a CTA's share of a
+                               // strip boundary moves onto it; -1: the packer picks the partition itself
 
 bool is_bijection(const int32_t* p, int64_t n) {
     std::vector<unsigned char> seen((size_t)n, 0);
@@ -118,28 +123,65 @@ void build_stream_plan(pp_packed* p) {
     // CTA boundaries as (strip, offset) pairs, offset in [0, len); (S, 0) is the end.
     struct Bnd { int s, off; };
     auto less = [](const Bnd& a, const Bnd& b) { return a.s < b.s || (a.s == b.s && a.off < b.off); };
-    int64_t G = std::min<int64_t>(g_stream_ctas, F / std::max(1, g_stream_min_frags));
-    G = std::max<int64_t>(G, 1);
-    const int64_t share = (F + G - 1) / G;
-    const int64_t tol = share * g_stream_snap_pct / 100;
-    std::vector<Bnd> bnd;
-    bnd.push_back({0, 0});
-    for (int64_t c = 1; c < G; ++c) {
-        const int64_t pos = F * c / G;
-        // non-empty strip containing pos
-        int s = (int)(std::upper_bound(p->strip_start.begin(), p->strip_start.end(), (int32_t)pos) -
-                      p->strip_start.begin()) - 1;
-        if (s >= S) continue;
-        int64_t off = pos - p->strip_start[(size_t)s];
-        const int64_t len = p->strip_start[(size_t)s + 1] - p->strip_start[(size_t)s];
-        Bnd b;
-        if (off <= tol && off <= len - off) b = {s, 0};
-        else if (len - off <= tol) b = {s + 1, 0};
-        else b = {s, (int)off};
-        if (less(bnd.back(), b)) bnd.push_back(b);
-    }
     const Bnd end{S, 0};
-    while (bnd.size() > 1 && !less(bnd.back(), end)) bnd.pop_back();
+    // Even split of the fragment sequence into G ranges; a boundary closer than tol_pct % of a
+    // CTA's share to a strip boundary moves onto it (100: every boundary does -> no strip is shared).
+    auto make_bounds = [&](int64_t G, int tol_pct) {
+        const int64_t share = (F + G - 1) / G;
+        const int64_t tol = tol_pct >= 100 ? F : share * tol_pct / 100;
+        std::vector<Bnd> bnd;
+        bnd.push_back({0, 0});
+        for (int64_t c = 1; c < G; ++c) {
+            const int64_t pos = F * c / G;
+            int s = (int)(std::upper_bound(p->strip_start.begin(), p->strip_start.end(), (int32_t)pos) -
+                          p->strip_start.begin()) - 1;      // non-empty strip containing pos
+            if (s >= S) continue;
+            const int64_t off = pos - p->strip_start[(size_t)s];
+            const int64_t len = p->strip_start[(size_t)s + 1] - p->strip_start[(size_t)s];
+            Bnd b;
+            if (off <= tol && off <= len - off) b = {s, 0};
+            else if (len - off <= tol) b = {s + 1, 0};
+            else b = {s, (int)off};
+            if (less(bnd.back(), b)) bnd.push_back(b);
+        }
+        while (bnd.size() > 1 && !less(bnd.back(), end)) bnd.pop_back();
+        return bnd;
+    };
+    auto pos_of = [&](const Bnd& b) { return (int64_t)p->strip_start[(size_t)b.s] + b.off; };
+    // Rough time of a partition.  CTAs are placed round-robin on the SMs, so SM i carries CTAs
+    // i, i + n_sm, ...; the fullest SM at its share of the memory system sets the time.  A strip
+    // shared by two CTAs costs one atomic exchange at the end, one shared by more a counter round.
+    auto cost_us = [&](const std::vector<Bnd>& bnd) {
+        const int n_sm = std::max(1, g_stream_sms);
+        std::vector<int64_t> sm_load((size_t)n_sm, 0);
+        bool shared = false, shared_many = false;
+        for (size_t c = 0; c < bnd.size(); ++c) {
+            const Bnd b1 = c + 1 < bnd.size() ? bnd[c + 1] : end;
+            sm_load[c % (size_t)n_sm] += pos_of(b1) - pos_of(bnd[c]);
+            shared = shared || bnd[c].off > 0;
+            shared_many = shared_many || (bnd[c].off > 0 && b1.s == bnd[c].s && b1.off > 0);
+        }
+        const int64_t max_load = *std::max_element(sm_load.begin(), sm_load.end());
+        const double bw_sm = std::min(100e9, 6.0e12 / (double)std::min<size_t>(bnd.size(), (size_t)n_sm));
+        return (double)max_load * 512.0 / bw_sm * 1e6 + (shared_many ? 3.0 : shared ? 0.7 : 0.0);
+    };
+    std::vector<Bnd> bnd;
+    if (g_stream_snap_pct >= 0) {       // manual partition (experiments, tests)
+        const int64_t G = std::max<int64_t>(1, std::min<int64_t>(g_stream_ctas, F / std::max(1, g_stream_min_frags)));
+        bnd = make_bounds(G, g_stream_snap_pct);
+    } else {
+        int nonempty = 0;
+        for (int s = 0; s < S; ++s) nonempty += p->strip_start[(size_t)s + 1] > p->strip_start[(size_t)s];
+        const int64_t g_even = std::max<int64_t>(1, std::min<int64_t>(g_stream_ctas, F / 32));
+        bnd = make_bounds(g_even, 2);
+        double best = cost_us(bnd);
+        const int64_t g_hi = std::max<int64_t>(1, std::min<int64_t>(g_stream_ctas, nonempty));
+        for (int64_t G = g_hi; G >= std::max<int64_t>(1, g_hi / 2); --G) {
+            std::vector<Bnd> cand = make_bounds(G, 100);
+            const double c = cost_us(cand);
+            if (c < best - 1e-9) { best = c; bnd = std::move(cand); }
+        }
+    }
     // no CTA may list more than kStreamMaxStrips strips
     std::vector<Bnd> cut;
     for (size_t c = 0; c < bnd.size(); ++c) {
@@ -194,8 +236,11 @@ pp_status_t pp_set_tuning(int key, int value) {
     if (key == 1 && value >= 0) { g_min_items = value; return PP_OK; }
     if (key == 2 && value >= 1) { g_stream_ctas = value; return PP_OK; }
     if (key == 3 && value >= 1) { g_stream_min_frags = value; return PP_OK; }
-    if (key == 4 && value >= 0 && value <= 50) { g_stream_snap_pct = value; return PP_OK; }
+    if (key == 4 && value >= -1 && value <= 100) { g_stream_snap_pct = value; return PP_OK; }
     if (key == 5 && (value == 0 || value == 1)) { pp::g_use_stream = value; return PP_OK; }
+    if (key == 6 && (value == 4 || value == 6 || value == 8)) { pp::g_stream_depth = value; return PP_OK; }
+    if (key == 7 && (value == 0 || value == 1)) { pp::g_stage_direct = value; return PP_OK; }
+    if (key == 8 && (value == 0 || value == 1)) { pp::g_stream_pdl = value; return PP_OK; }
     return PP_ERR_INVALID_ARG;
 }
 

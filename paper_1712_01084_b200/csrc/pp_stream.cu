@@ -2,18 +2,29 @@
 //
 // The packed tile values of a layer form one linear sequence of 512-byte fragments (strip =
 // row-group of a block-row; a strip's fragments are contiguous and strips follow each other).
-// The host cuts that sequence into one contiguous range per CTA (2 CTAs per SM), and every warp
-// of a CTA streams an equal, contiguous share of its CTA's range:
-//   * Listing 1's group fetch is done ONCE per CTA for the whole pivoted input:
-//     xs[j] = x[gather_idx[j]] goes to shared memory while the first weight fragments are already
-//     in flight; after one barrier no warp waits for another until its range is finished;
-//   * each warp keeps kUnroll 128-bit loads (4 KiB) in flight and refills a slot as soon as it is
-//     consumed, so the load queue never drains at work-unit boundaries;
+// The host cuts that sequence into one contiguous range per CTA, and every warp of a CTA
+// streams an equal, contiguous share of its CTA's range:
+//   * Listing 1's group fetch is done ONCE per CTA for the whole layer input: x and the column
+//     index array are copied to shared memory with 16-byte asynchronous copies (issued first,
+//     so they are not queued behind the weight loads) and permuted there into pivoted order
+//     while the first weight fragments are in flight; after that barrier no warp waits for
+//     another until its range is finished;
+//   * the weights never pass through registers on their way in: each warp owns a ring of U
+//     512-byte slots in shared memory and keeps U 16-byte-per-lane asynchronous copies
+//     (cp.async groups) in flight, refilling a slot right after reading it (a register ring of
+//     plain loads serialises on the load scoreboard and measured 30 % slower; it also blocked the
+//     shared-memory permutation of x behind the outstanding weight loads);
 //   * where a warp's range crosses a strip boundary it parks the finished 16(32)-row partial sum
 //     in shared memory; after the final barrier the CTA adds the parks of every strip in warp
 //     order.  A strip shared by several CTAs (Section 4.1.5's "additional reduction step") goes
 //     through one global partial sum per CTA, added in CTA order by the last CTA to arrive.
-// Results are therefore independent of scheduling.  fp16 tiles: warp-level 16x8x16 tensor-core
+//   * everything the epilogue needs (row index array, pivoted bias, strip table) is fetched
+//     asynchronously at kernel start, so the tail is shared-memory work plus the stores;
+//   * the kernel is launched with programmatic stream serialization: it releases its successor
+//     at once (griddepcontrol.launch_dependents) and fetches tables and first weights before
+//     griddepcontrol.wait, so back-to-back layers overlap launch latency and prologue with the
+//     previous kernel's tail.  x is read, and y and scratch are written, only after the wait.
+// Results are independent of scheduling.  fp16 tiles: warp-level 16x8x16 tensor-core
 // instruction, batch on the 8-wide side, fp32 accumulate.  fp32 tiles: plain FMAs.
 #include <cuda_fp16.h>
 
@@ -24,7 +35,12 @@ namespace pp {
 namespace {
 
 constexpr int kThreads = kStreamWarps * 32;
-constexpr int kUnroll = 8;
+constexpr int kParamCtas = 320;       // CTA ranges that travel in the kernel parameters
+
+struct StreamLaunch {
+    StreamArgs a;
+    CtaDesc table[kParamCtas];
+};
 
 __device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
     uint4 v;
@@ -46,29 +62,58 @@ __device__ __forceinline__ void mma_16x8x16(float (&d)[4], const uint4& a, uint3
         : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b0), "r"(b1));
 }
 
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                 :: "r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc));
+}
+__device__ __forceinline__ void cp_async_4(void* smem_dst, const void* gsrc) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;"
+                 :: "r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc));
+}
+
 __device__ __forceinline__ int x_index(const StreamArgs& a, int pj) {
     if (a.gather_idx) return __ldg(a.gather_idx + pj);
     return pj < a.x_limit ? pj : -1;
 }
 
-// Shared-memory header shared by both kernels (all sizes in 4-byte words).
+// Shared memory: fixed header, then the regions whose size depends on the launch.
 struct SmemLayout {
-    int* sstart;    // [kStreamMaxStrips + 1] strip starts of this CTA's strips
-    int* wlohi;     // [kStreamMaxStrips] first | last << 8 warp that parked a partial for the strip
-    int* flags;     // [2]
-    float* segp;    // [kStreamSegSlots][RG][batch]
-    void* xs;       // staged x
+    int* sstart;     // [kStreamMaxStrips + 1] strip starts of this CTA's strips
+    int* wlohi;      // [kStreamMaxStrips] first | last << 8 warp that parked a partial for the strip
+    int* flags;      // [2]
+    int* wb;         // [kStreamWarps + 1] fragment position where each warp's range starts
+    int4* sinfo;     // [kStreamMaxStrips] strip table entries of this CTA's strips
+    int* rowdst;     // [max_rows] scatter_idx of this CTA's pivoted rows
+    float* rowbias;  // [max_rows] bias_piv of this CTA's pivoted rows
+    float* segp;     // [kStreamSegSlots][RG][batch] parked partial sums
+    uint4* ring;     // [kStreamWarps][U][32] weight fragments in flight
+    void* xs;        // staged pivoted x   [batch][xs_stride] (absent in staging mode 3)
+    int* idxs;       // staging modes 1, 3: gather_idx [n_pad]
+    void* raw;       // staging modes 1, 3: x as given [batch][raw_stride]
 };
-constexpr int kHeaderWords = 128;   // sstart (49) + wlohi (48) + flags (2), padded
+constexpr int kHeaderBytes = 512 + kStreamMaxStrips * 16;   // 512 B: sstart, wlohi, flags; then sinfo
 
-__device__ __forceinline__ SmemLayout carve(unsigned char* raw, int rg, int batch) {
+__host__ __device__ __forceinline__ size_t xs_bytes(int batch, int xs_stride, int esz) {
+    return ((size_t)batch * xs_stride * esz + 15) / 16 * 16;
+}
+
+__device__ __forceinline__ SmemLayout carve(unsigned char* base, int rg, int U, const StreamArgs& a, int esz) {
     SmemLayout L;
-    int* w = reinterpret_cast<int*>(raw);
+    int* w = reinterpret_cast<int*>(base);
     L.sstart = w;
     L.wlohi = w + 56;
-    L.flags = w + 112;
-    L.segp = reinterpret_cast<float*>(w + kHeaderWords);
-    L.xs = L.segp + kStreamSegSlots * rg * batch;
+    L.flags = w + 108;
+    L.wb = w + 110;
+    L.sinfo = reinterpret_cast<int4*>(base + 512);
+    L.rowdst = reinterpret_cast<int*>(base + kHeaderBytes);
+    L.rowbias = reinterpret_cast<float*>(L.rowdst + a.max_rows);
+    L.segp = L.rowbias + a.max_rows;
+    L.ring = reinterpret_cast<uint4*>(L.segp + kStreamSegSlots * rg * a.batch);
+    unsigned char* p = reinterpret_cast<unsigned char*>(L.ring + kStreamWarps * U * 32);
+    L.xs = p;
+    if (a.stage_mode != 3) p += xs_bytes(a.batch, a.xs_stride, esz);
+    L.idxs = reinterpret_cast<int*>(p);
+    L.raw = p + (size_t)a.n_pad * 4 + 16;     // 16 spare bytes in front: raw[-1] is the zero that index -1 reads
     return L;
 }
 
@@ -76,44 +121,153 @@ __device__ __forceinline__ int warp_begin(const CtaDesc& d, int w) {
     return d.p_begin + (int)(((long long)(d.p_end - d.p_begin) * w) / kStreamWarps);
 }
 
+__device__ __forceinline__ CtaDesc cta_range(const StreamLaunch& P) {
+    if (gridDim.x <= kParamCtas) return P.table[blockIdx.x];
+    const int4 dd = __ldg(reinterpret_cast<const int4*>(P.a.cta_desc) + blockIdx.x);
+    return CtaDesc{dd.x, dd.y, dd.z, dd.w};
+}
+
+// Phase 1a: asynchronous copies of the layer's own (immutable) tables: strip starts, strip table,
+// row index array and pivoted bias of this CTA's rows, and the column index array.  Nothing
+// here depends on the previous kernel in the stream, so it runs before griddepcontrol.wait.
+template <int RG>
+__device__ __forceinline__ void issue_static(const StreamArgs& a, const CtaDesc& d, const SmemLayout& L) {
+    const int tid = threadIdx.x;
+    for (int i = tid; i <= d.s_count; i += kThreads) cp_async_4(L.sstart + i, a.strip_start + d.s_first + i);
+    for (int i = tid; i < d.s_count; i += kThreads) cp_async_16(L.sinfo + i, a.strip_info + d.s_first + i);
+    const int n_rows = d.s_count * RG, row0 = d.s_first * RG;
+    for (int i = tid; i < n_rows; i += kThreads) {
+        cp_async_4(L.rowdst + i, a.scatter_idx + row0 + i);
+        cp_async_4(L.rowbias + i, a.bias_piv + row0 + i);
+    }
+    if (a.stage_mode == 1 || a.stage_mode == 3)
+        for (int i = tid; i < a.n_pad / 4; i += kThreads) cp_async_16(L.idxs + 4 * i, a.gather_idx + 4 * i);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// Phase 1b (after griddepcontrol.wait): Listing 1's group fetch, for the whole layer input.
+// Mode 1 copies x to shared memory (permuted in phase 3 through the index array copied in
+// phase 1a), mode 3 (batch 1) copies x and lets the multiply loop read it through the index
+// array, mode 2 (input already in pivoted order) copies straight into place; mode 0 leaves the
+// gather to phase 3.
+template <typename T>
+__device__ __forceinline__ void issue_x(const StreamArgs& a, const SmemLayout& L) {
+    constexpr int EPC = 16 / (int)sizeof(T);
+    const int tid = threadIdx.x;
+    if (tid == 0) asm volatile("prefetch.global.L2 [%0];" :: "l"(a.y));   // warm the translation of the output page
+    if (a.stage_mode != 0) {
+        const bool via_raw = a.stage_mode != 2;
+        const T* x = static_cast<const T*>(a.x);
+        T* dst = via_raw ? static_cast<T*>(L.raw) : static_cast<T*>(L.xs);
+        const int dst_stride = via_raw ? a.raw_stride : a.xs_stride;
+        // modes 1, 3 copy every element a gather index may name (x_len); mode 2 copies the N real
+        // columns (the padding columns up to n_pad are zero-filled in phase 3)
+        const int n_chunks = (via_raw ? a.x_len : a.x_limit) / EPC;
+        for (int b = 0; b < a.batch; ++b)
+            for (int i = tid; i < n_chunks; i += kThreads)
+                cp_async_16(dst + b * dst_stride + i * EPC, x + (size_t)b * a.ldx + i * EPC);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// Phase 3: wait for the copies of phases 1 and 2, finish the staged pivoted x.
+template <typename T, int U>
+__device__ __forceinline__ void finish_stage(const StreamArgs& a, const SmemLayout& L) {
+    constexpr int EPC = 16 / (int)sizeof(T);
+    const int tid = threadIdx.x;
+    const T* x = static_cast<const T*>(a.x);
+    T* xs = static_cast<T*>(L.xs);
+    if (a.stage_mode != 0) {
+        // ragged tail of each row (fewer than 16 bytes) and, in mode 2, the zero padding
+        const bool via_raw = a.stage_mode != 2;
+        T* dst = via_raw ? static_cast<T*>(L.raw) : xs;
+        const int dst_stride = via_raw ? a.raw_stride : a.xs_stride;
+        const int n_src = via_raw ? a.x_len : a.x_limit;
+        const int n_dst = via_raw ? a.x_len : a.n_pad;
+        if (a.stage_mode == 3 && tid == 0) dst[-1] = T(0.0f);
+        const int done = n_src / EPC * EPC;
+        for (int b = 0; b < a.batch; ++b)
+            for (int j = done + tid; j < n_dst; j += kThreads)
+                dst[b * dst_stride + j] = j < n_src ? x[(size_t)b * a.ldx + j] : T(0.0f);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");   // tables, first weight fragments and x have landed
+    if (a.stage_mode == 1) {
+        __syncthreads();
+        const T* raw = static_cast<const T*>(L.raw);
+#pragma unroll 8
+        for (int j = tid; j < a.n_pad; j += kThreads) {
+            const int idx = L.idxs[j];
+            for (int b = 0; b < a.batch; ++b)
+                xs[b * a.xs_stride + j] = idx >= 0 ? raw[b * a.raw_stride + idx] : T(0.0f);
+        }
+    } else if (a.stage_mode == 0) {
+        for (int j0 = tid; j0 < a.n_pad; j0 += 8 * kThreads) {
+            int idx[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int j = j0 + q * kThreads;
+                idx[q] = j < a.n_pad ? x_index(a, j) : -1;
+            }
+            for (int b = 0; b < a.batch; ++b) {
+                T v[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) v[q] = idx[q] >= 0 ? x[(size_t)b * a.ldx + idx[q]] : T(0.0f);
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (j0 + q * kThreads < a.n_pad) xs[b * a.xs_stride + j0 + q * kThreads] = v[q];
+            }
+        }
+    }
+    __syncthreads();
+}
+
+constexpr unsigned kEmptySlot = 0xffffffffu;   // exchange slots rest at this NaN pattern
+
 // Everything after the last barrier of the streaming phase: per-strip sums, cross-CTA reduction,
 // bias + activation + (scatter | pivoted store).  RG = rows per strip.
+//
+// A strip shared by exactly two CTAs needs no counter and no fence: each CTA swaps its partial sum
+// into the strip's exchange slot; whoever gets the resting pattern back was first and is done,
+// the other gets the first one's partial sum back, adds its own (a + b == b + a bit for bit, so the
+// order of arrival cannot change the result), stores the row and puts the resting pattern back.
+// Strips shared by three or more CTAs publish one partial sum per CTA and the last CTA to bump the
+// strip's counter adds them in CTA order.
 template <int RG>
 __device__ __forceinline__ void finalize(const StreamArgs& a, const CtaDesc& d, const SmemLayout& L) {
     const int tid = threadIdx.x;
     const int batch = a.batch;
     const int per_strip = RG * batch;
 
-    auto emit = [&](int i, int b, float v) {
-        v += __ldg(a.bias_piv + i);
+    auto emit = [&](int ls, int r, int b, float v) {
+        const int lr = ls * RG + r;
+        v += L.rowbias[lr];
         if (a.act == PP_ACT_RELU) v = fmaxf(v, 0.0f);
         if (a.out_mode == OUT_SCATTER_F32) {
-            const int dst = __ldg(a.scatter_idx + i);
+            const int dst = L.rowdst[lr];
             if (dst >= 0) static_cast<float*>(a.y)[(size_t)b * a.ldy + dst] = v;
-        } else if (a.out_mode == OUT_PIVOTED_F32) {
-            static_cast<float*>(a.y)[(size_t)b * a.ldy + i] = v;
         } else {
-            static_cast<__half*>(a.y)[(size_t)b * a.ldy + i] = __float2half_rn(v);
+            const int i = d.s_first * RG + lr;
+            if (a.out_mode == OUT_PIVOTED_F32) static_cast<float*>(a.y)[(size_t)b * a.ldy + i] = v;
+            else static_cast<__half*>(a.y)[(size_t)b * a.ldy + i] = __float2half_rn(v);
         }
     };
 
-    // which warps parked a partial for each strip (their ranges intersect the strip inside this CTA)
+    // which warps parked a partial for each strip (their ranges intersect the strip inside this CTA);
+    // L.wb holds the warps' range starts (written in the prologue)
     for (int ls = tid; ls < d.s_count; ls += kThreads) {
         const int lo = max(L.sstart[ls], d.p_begin), hi = min(L.sstart[ls + 1], d.p_end);
         int w_lo = 1, w_hi = 0;
         if (lo < hi) {
             w_lo = w_hi = 0;
             for (int w = 1; w < kStreamWarps; ++w) {
-                const int wb = warp_begin(d, w);
-                if (wb <= lo) w_lo = w;
-                if (wb <= hi - 1) w_hi = w;
+                if (L.wb[w] <= lo) w_lo = w;
+                if (L.wb[w] <= hi - 1) w_hi = w;
             }
         }
         L.wlohi[ls] = w_lo | (w_hi << 8);
     }
     __syncthreads();
 
-    bool shared_any = false;
     const int n_out = d.s_count * per_strip;
     for (int e = tid; e < n_out; e += kThreads) {
         const int ls = e / per_strip, rem = e - ls * per_strip;
@@ -121,32 +275,34 @@ __device__ __forceinline__ void finalize(const StreamArgs& a, const CtaDesc& d, 
         const int wl = L.wlohi[ls] & 0xff, wh = L.wlohi[ls] >> 8;
         float v = 0.0f;
         for (int w = wl; w <= wh; ++w)      // warps with an empty range parked nothing
-            if (warp_begin(d, w) < warp_begin(d, w + 1)) v += L.segp[((ls + w) * RG + r) * batch + b];
-        const int s = d.s_first + ls;
-        const int4 info = __ldg(reinterpret_cast<const int4*>(a.strip_info) + s);
+            if (L.wb[w] < L.wb[w + 1]) v += L.segp[((ls + w) * RG + r) * batch + b];
+        const int4 info = L.sinfo[ls];
         if (info.y == 1) {
-            emit(s * RG + r, b, v);
+            emit(ls, r, b, v);
+        } else if (info.y == 2) {
+            unsigned* slot = reinterpret_cast<unsigned*>(a.partials + (size_t)info.z * (RG * kStreamMaxBatch) + rem);
+            unsigned mine = __float_as_uint(v);
+            if (mine == kEmptySlot) mine = 0x7fc00000u;          // a NaN stays a NaN, but not the resting pattern
+            const unsigned other = atomicExch(slot, mine);
+            if (other != kEmptySlot) {
+                emit(ls, r, b, v + __uint_as_float(other));
+                *slot = kEmptySlot;
+            }
         } else {
             a.partials[(size_t)(info.z + (int)blockIdx.x - info.x) * (RG * kStreamMaxBatch) + rem] = v;
-            shared_any = true;
         }
     }
     // only the first and the last strip of a CTA can be shared with a neighbour
     const int ls_edge[2] = {0, d.s_count - 1};
     int4 edge[2];
-#pragma unroll
-    for (int k = 0; k < 2; ++k) {
-        edge[k] = make_int4(0, 1, 0, 0);
-        if (d.s_count > 0 && (k == 0 || d.s_count > 1))
-            edge[k] = __ldg(reinterpret_cast<const int4*>(a.strip_info) + d.s_first + ls_edge[k]);
-    }
-    if (edge[0].y == 1 && edge[1].y == 1) return;      // uniform for the CTA
-    (void)shared_any;
+    edge[0] = L.sinfo[0];
+    edge[1] = d.s_count > 1 ? L.sinfo[d.s_count - 1] : make_int4(0, 1, 0, 0);
+    if (edge[0].y <= 2 && edge[1].y <= 2) return;      // uniform for the CTA
     __threadfence();
     __syncthreads();
     if (tid < 2) {
         int last = 0;
-        if (edge[tid].y > 1) {
+        if (edge[tid].y > 2) {
             const int old = atomicAdd(a.counters + d.s_first + ls_edge[tid], 1);
             last = (old == edge[tid].y - 1);
         }
@@ -157,55 +313,88 @@ __device__ __forceinline__ void finalize(const StreamArgs& a, const CtaDesc& d, 
     for (int k = 0; k < 2; ++k) {
         if (!L.flags[k]) continue;
         __threadfence();
-        const int s = d.s_first + ls_edge[k];
         const float* base = a.partials + (size_t)edge[k].z * (RG * kStreamMaxBatch);
         for (int e = tid; e < per_strip; e += kThreads) {
             float v = 0.0f;
             for (int p = 0; p < edge[k].y; ++p) v += ld_cg(base + (size_t)p * (RG * kStreamMaxBatch) + e);
             const int r = e / batch, b = e - r * batch;
-            emit(s * RG + r, b, v);
+            emit(ls_edge[k], r, b, v);
         }
-        if (tid == 0) a.counters[s] = 0;
+        if (tid == 0) a.counters[d.s_first + ls_edge[k]] = 0;
     }
 }
 
+// Per-warp weight ring.  prologue(): fill the U slots (one cp.async group per slot, committed even
+// when empty so that group counting stays uniform).  Inside the main loop, slot u is read after
+// cp.async.wait_group U-1 and refilled with fragment p + U.
+template <int U>
+struct WeightRing {
+    uint4* slot;           // this lane's 16 bytes of slot 0; slot u is slot + 32 * u
+    const uint4* vals;     // this lane's 16 bytes of fragment 0
+    __device__ __forceinline__ void fill(int u, int p, int wend) const {
+        if (p < wend) cp_async_16(slot + 32 * u, vals + (size_t)p * 32);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    __device__ __forceinline__ void prologue(int wbeg, int wend) const {
+#pragma unroll
+        for (int u = 0; u < U; ++u) fill(u, wbeg + u, wend);
+    }
+    __device__ __forceinline__ uint4 take(int u) const {
+        asm volatile("cp.async.wait_group %0;" :: "n"(U - 1) : "memory");
+        return slot[32 * u];
+    }
+};
+
+// Column offsets of 32 consecutive fragments, one per lane, fetched one block ahead.
+struct XoffWindow {
+    const int32_t* xoff;
+    int cur, nxt, base;    // cur covers fragments [base, base + 32)
+    __device__ __forceinline__ void init(const int32_t* table, int wbeg, int wend, int lane) {
+        xoff = table; base = wbeg;
+        cur = wbeg + lane < wend ? __ldg(xoff + wbeg + lane) : 0;
+        nxt = wbeg + 32 + lane < wend ? __ldg(xoff + wbeg + 32 + lane) : 0;
+    }
+    __device__ __forceinline__ int get(int p, int wend, int lane) {
+        if (p - base == 32) {
+            base += 32; cur = nxt;
+            nxt = base + 32 + lane < wend ? __ldg(xoff + base + 32 + lane) : 0;
+        }
+        return __shfl_sync(0xffffffffu, cur, p - base);
+    }
+};
+
 // ------------------------------------------------------------------ fp16 tiles
-__global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const StreamArgs a) {
+template <int U>
+__global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_constant__ StreamLaunch P) {
     constexpr int RG = 16;
+    const StreamArgs& a = P.a;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    const SmemLayout L = carve(smem_raw, RG, a.batch);
+    const SmemLayout L = carve(smem_raw, RG, U, a, 2);
     __half* xs = static_cast<__half*>(L.xs);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
-    const int4 dd = __ldg(reinterpret_cast<const int4*>(a.cta_desc) + blockIdx.x);
-    const CtaDesc d{dd.x, dd.y, dd.z, dd.w};
+    const CtaDesc d = cta_range(P);
     const int wbeg = warp_begin(d, warp), wend = warp_begin(d, warp + 1);
+    if (tid <= kStreamWarps) L.wb[tid] = warp_begin(d, tid);
 
-    // 1. first weight fragments (and their x offsets) in flight
-    const uint4* vals = reinterpret_cast<const uint4*>(a.values) + lane;
-    uint4 w[kUnroll];
-    int xo[kUnroll];
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-        const int p = wbeg + u;
-        if (p < wend) {
-            w[u] = ldg_stream(vals + (size_t)p * 32);
-            xo[u] = __ldg(a.xoff + p);
-        }
-    }
+    // 1. the next kernel in the stream may start its own prologue; this one prefetches what does
+    //    not depend on its predecessor: tables, first U weight fragments, column offsets
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    issue_static<RG>(a, d, L);
+    const WeightRing<U> ring{L.ring + (warp * U) * 32 + lane, reinterpret_cast<const uint4*>(a.values) + lane};
+    ring.prologue(wbeg, wend);
+    XoffWindow xw;
+    xw.init(a.xoff, wbeg, wend, lane);
 
-    // 2. group fetch of the whole pivoted x, once per CTA
-    for (int i = tid; i <= d.s_count; i += kThreads) L.sstart[i] = __ldg(a.strip_start + d.s_first + i);
-    const __half* x = static_cast<const __half*>(a.x);
-    for (int j = tid; j < a.n_pad; j += kThreads) {
-        const int idx = x_index(a, j);
-        for (int b = 0; b < a.batch; ++b)
-            xs[b * a.xs_stride + j] = idx >= 0 ? x[(size_t)b * a.ldx + idx] : __float2half(0.0f);
-    }
-    __syncthreads();
+    // 2. everything before this kernel in the stream is complete from here on: fetch x
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    issue_x<__half>(a, L);
 
-    // 3. stream this warp's share
+    // 3. pivoted x in shared memory
+    finish_stage<__half, U>(a, L);
+
+    // 4. stream this warp's share
     float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     auto park = [&](int slot) {
         float* r0 = L.segp + (slot * RG + g) * a.batch;
@@ -218,10 +407,12 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const StreamArg
         while (ls + 1 < d.s_count && L.sstart[ls + 1] <= wbeg) ++ls;
         int seg_end = min(wend, L.sstart[ls + 1]);
         const bool has_x = g < a.batch;
+        const bool direct = a.stage_mode == 3;
+        const unsigned short* rawu = static_cast<const unsigned short*>(L.raw);
         const __half* xrow = xs + g * a.xs_stride + 2 * t;
-        for (int base = wbeg; base < wend; base += kUnroll) {
+        for (int base = wbeg; base < wend; base += U) {
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
+            for (int u = 0; u < U; ++u) {
                 const int p = base + u;
                 if (p < wend) {
                     if (p == seg_end) {
@@ -230,59 +421,54 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const StreamArg
                         do { ++ls; } while (L.sstart[ls + 1] <= p);
                         seg_end = min(wend, L.sstart[ls + 1]);
                     }
-                    const uint4 wa = w[u];
-                    const int xoff = xo[u];
-                    if (p + kUnroll < wend) {
-                        w[u] = ldg_stream(vals + (size_t)(p + kUnroll) * 32);
-                        xo[u] = __ldg(a.xoff + p + kUnroll);
-                    }
+                    const int xoff = xw.get(p, wend, lane);
                     uint32_t b0 = 0u, b1 = 0u;
-                    if (has_x) {
+                    if (direct) {            // batch 1: read x through the index array (index -1 reads raw[-1] = 0)
+                        if (g == 0) {
+                            const int2 i0 = *reinterpret_cast<const int2*>(L.idxs + xoff + 2 * t);
+                            const int2 i1 = *reinterpret_cast<const int2*>(L.idxs + xoff + 2 * t + 8);
+                            b0 = (uint32_t)rawu[i0.x] | ((uint32_t)rawu[i0.y] << 16);
+                            b1 = (uint32_t)rawu[i1.x] | ((uint32_t)rawu[i1.y] << 16);
+                        }
+                    } else if (has_x) {
                         b0 = *reinterpret_cast<const uint32_t*>(xrow + xoff);
                         b1 = *reinterpret_cast<const uint32_t*>(xrow + xoff + 8);
                     }
+                    const uint4 wa = ring.take(u);
+                    ring.fill(u, p + U, wend);
                     mma_16x8x16(acc, wa, b0, b1);
                 }
             }
         }
         park(ls + warp);
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     finalize<RG>(a, d, L);
 }
 
 // ------------------------------------------------------------------ fp32 tiles
-template <int RG, int NB>
-__global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const StreamArgs a) {
+template <int RG, int NB, int U>
+__global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const __grid_constant__ StreamLaunch P) {
+    const StreamArgs& a = P.a;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    const SmemLayout L = carve(smem_raw, RG, a.batch);
+    const SmemLayout L = carve(smem_raw, RG, U, a, 4);
     float* xs = static_cast<float*>(L.xs);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int4 dd = __ldg(reinterpret_cast<const int4*>(a.cta_desc) + blockIdx.x);
-    const CtaDesc d{dd.x, dd.y, dd.z, dd.w};
+    const CtaDesc d = cta_range(P);
     const int wbeg = warp_begin(d, warp), wend = warp_begin(d, warp + 1);
+    if (tid <= kStreamWarps) L.wb[tid] = warp_begin(d, tid);
 
-    const uint4* vals = reinterpret_cast<const uint4*>(a.values) + lane;
-    uint4 w[kUnroll];
-    int xo[kUnroll];
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-        const int p = wbeg + u;
-        if (p < wend) {
-            w[u] = ldg_stream(vals + (size_t)p * 32);
-            xo[u] = __ldg(a.xoff + p);
-        }
-    }
-
-    for (int i = tid; i <= d.s_count; i += kThreads) L.sstart[i] = __ldg(a.strip_start + d.s_first + i);
-    const float* x = static_cast<const float*>(a.x);
-    for (int j = tid; j < a.n_pad; j += kThreads) {
-        const int idx = x_index(a, j);
-        for (int b = 0; b < a.batch; ++b)
-            xs[b * a.xs_stride + j] = idx >= 0 ? __ldg(x + (size_t)b * a.ldx + idx) : 0.0f;
-    }
-    __syncthreads();
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    issue_static<RG>(a, d, L);
+    const WeightRing<U> ring{L.ring + (warp * U) * 32 + lane, reinterpret_cast<const uint4*>(a.values) + lane};
+    ring.prologue(wbeg, wend);
+    XoffWindow xw;
+    xw.init(a.xoff, wbeg, wend, lane);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    issue_x<float>(a, L);
+    finish_stage<float, U>(a, L);
 
     float acc[NB][2];
 #pragma unroll
@@ -301,9 +487,11 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const StreamArg
         while (ls + 1 < d.s_count && L.sstart[ls + 1] <= wbeg) ++ls;
         int seg_end = min(wend, L.sstart[ls + 1]);
         const float* xlane = xs + (lane / RG) * 4;
-        for (int base = wbeg; base < wend; base += kUnroll) {
+        const bool direct = a.stage_mode == 3;
+        const float* rawf = static_cast<const float*>(L.raw);
+        for (int base = wbeg; base < wend; base += U) {
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
+            for (int u = 0; u < U; ++u) {
                 const int p = base + u;
                 if (p < wend) {
                     if (p == seg_end) {
@@ -311,14 +499,19 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const StreamArg
                         do { ++ls; } while (L.sstart[ls + 1] <= p);
                         seg_end = min(wend, L.sstart[ls + 1]);
                     }
-                    const uint4 wa = w[u];
-                    const int xoff = xo[u];
-                    if (p + kUnroll < wend) {
-                        w[u] = ldg_stream(vals + (size_t)(p + kUnroll) * 32);
-                        xo[u] = __ldg(a.xoff + p + kUnroll);
-                    }
+                    const int xoff = xw.get(p, wend, lane);
+                    const uint4 wa = ring.take(u);
+                    ring.fill(u, p + U, wend);
                     const float w0 = __uint_as_float(wa.x), w1 = __uint_as_float(wa.y);
                     const float w2 = __uint_as_float(wa.z), w3 = __uint_as_float(wa.w);
+                    if (direct) {            // batch 1: read x through the index array (index -1 reads raw[-1] = 0)
+                        const int4 ii = *reinterpret_cast<const int4*>(L.idxs + xoff + (lane / RG) * 4);
+                        acc[0][0] = fmaf(w0, rawf[ii.x], acc[0][0]);
+                        acc[0][1] = fmaf(w1, rawf[ii.y], acc[0][1]);
+                        acc[0][0] = fmaf(w2, rawf[ii.z], acc[0][0]);
+                        acc[0][1] = fmaf(w3, rawf[ii.w], acc[0][1]);
+                        continue;
+                    }
 #pragma unroll
                     for (int b = 0; b < NB; ++b) {
                         if (b < a.batch) {
@@ -334,12 +527,13 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const StreamArg
         }
         park(ls + warp);
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     finalize<RG>(a, d, L);
 }
 
 template <auto Kernel>
-cudaError_t launch_one(const StreamArgs& a, int grid, size_t smem, cudaStream_t stream) {
+cudaError_t launch_one(const StreamLaunch& P, int grid, size_t smem, cudaStream_t stream) {
     static bool configured = false;   // one flag per kernel instantiation
     if (smem > kStreamSmemLimit) return cudaErrorInvalidValue;
     if (!configured && smem > 48 * 1024) {
@@ -348,37 +542,66 @@ cudaError_t launch_one(const StreamArgs& a, int grid, size_t smem, cudaStream_t 
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    Kernel<<<grid, kThreads, smem, stream>>>(a);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_stream_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, Kernel, P);
 }
 
-template <int RG>
-cudaError_t launch_f32(const StreamArgs& a, int grid, size_t smem, cudaStream_t stream) {
-    if (a.batch == 1) return launch_one<stream_f32_kernel<RG, 1>>(a, grid, smem, stream);
-    if (a.batch == 2) return launch_one<stream_f32_kernel<RG, 2>>(a, grid, smem, stream);
-    if (a.batch <= 4) return launch_one<stream_f32_kernel<RG, 4>>(a, grid, smem, stream);
-    return launch_one<stream_f32_kernel<RG, 8>>(a, grid, smem, stream);
+template <int RG, int U>
+cudaError_t launch_f32(const StreamLaunch& P, int grid, size_t smem, cudaStream_t stream) {
+    if (P.a.batch == 1) return launch_one<stream_f32_kernel<RG, 1, U>>(P, grid, smem, stream);
+    if (P.a.batch == 2) return launch_one<stream_f32_kernel<RG, 2, U>>(P, grid, smem, stream);
+    if (P.a.batch <= 4) return launch_one<stream_f32_kernel<RG, 4, U>>(P, grid, smem, stream);
+    return launch_one<stream_f32_kernel<RG, 8, U>>(P, grid, smem, stream);
 }
 
 int xs_stride_for(pp_dtype_t dt, int n_pad) { return dt == PP_F16 ? n_pad + 8 : n_pad + 4; }
 
 }  // namespace
 
-size_t stream_smem_bytes(pp_dtype_t dt, int B, int n_pad, int batch) {
+int g_stream_depth = 4;   // ring slots per warp (4, 6 or 8)
+int g_stream_pdl = 1;     // launch with programmatic stream serialization (prologue overlaps the previous kernel)
+
+size_t stream_smem_bytes(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode) {
     const int rg = frag_geom(dt, B).rg_rows;
-    const size_t esz = dt == PP_F16 ? 2 : 4;
-    return (size_t)kHeaderWords * 4 + (size_t)kStreamSegSlots * rg * batch * 4 +
-           (size_t)batch * xs_stride_for(dt, n_pad) * esz + 16;
+    const int esz = dt == PP_F16 ? 2 : 4;
+    size_t bytes = (size_t)kHeaderBytes + (size_t)max_rows * 8 + (size_t)kStreamSegSlots * rg * batch * 4 +
+                   (size_t)kStreamWarps * g_stream_depth * 512;
+    if (stage_mode != 3) bytes += xs_bytes(batch, xs_stride_for(dt, n_pad), esz);
+    if (stage_mode == 1 || stage_mode == 3)
+        bytes += (size_t)n_pad * 4 + 16 + (size_t)batch * ((x_len + 15) / 16 * 16) * esz;
+    return bytes;
 }
 
-cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a_in, int grid, cudaStream_t stream) {
+cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a_in, const CtaDesc* host_table, int grid,
+                          cudaStream_t stream) {
     if (grid <= 0) return cudaSuccess;
-    StreamArgs a = a_in;
-    if (a.batch < 1 || a.batch > kStreamMaxBatch) return cudaErrorInvalidValue;
+    StreamLaunch P;
+    P.a = a_in;
+    StreamArgs& a = P.a;
+    if (a.batch < 1 || a.batch > kStreamMaxBatch || (a.stage_mode == 3 && a.batch != 1)) return cudaErrorInvalidValue;
     a.xs_stride = xs_stride_for(dt, a.n_pad);
-    const size_t smem = stream_smem_bytes(dt, B, a.n_pad, a.batch);
-    if (dt == PP_F16) return launch_one<stream_f16_kernel>(a, grid, smem, stream);
-    return B < 32 ? launch_f32<16>(a, grid, smem, stream) : launch_f32<32>(a, grid, smem, stream);
+    a.raw_stride = (a.x_len + 15) / 16 * 16;
+    a.max_rows = (a.max_rows + 3) / 4 * 4;
+    if (grid <= kParamCtas)
+        for (int c = 0; c < grid; ++c) P.table[c] = host_table[c];
+    const size_t smem = stream_smem_bytes(dt, B, a.n_pad, a.x_len, a.max_rows, a.batch, a.stage_mode);
+    const bool deep = g_stream_depth == 8;
+    if (dt == PP_F16) {
+        if (g_stream_depth == 6) return launch_one<stream_f16_kernel<6>>(P, grid, smem, stream);
+        return deep ? launch_one<stream_f16_kernel<8>>(P, grid, smem, stream)
+                    : launch_one<stream_f16_kernel<4>>(P, grid, smem, stream);
+    }
+    if (B < 32) return deep ? launch_f32<16, 8>(P, grid, smem, stream) : launch_f32<16, 4>(P, grid, smem, stream);
+    return deep ? launch_f32<32, 8>(P, grid, smem, stream) : launch_f32<32, 4>(P, grid, smem, stream);
 }
 
 }  // namespace pp

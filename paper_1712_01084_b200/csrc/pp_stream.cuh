@@ -22,17 +22,30 @@ struct StreamArgs {
     int ldx, ldy;
     int x_limit;                 // with gather_idx == NULL: columns >= x_limit read 0
     int n_pad;                   // pivoted columns staged into shared memory
+    int x_len;                   // elements of an x row that gather_idx may name
+    int max_rows;                // most pivoted rows (strips x rows per strip) any CTA of the plan lists
+    int raw_stride;              // staging mode 1: row stride of the shared-memory copy of x (set by the launcher)
     int xs_stride;               // shared-memory row stride of the staged x, in elements
     int batch;
     int act;
     int out_mode;                // pp::OutMode
+    int stage_mode;              // 0: gather x from global memory; 1: copy x and gather_idx to shared
+                                 // memory, permute there (needs 16-byte aligned rows); 2: x is already
+                                 // in pivoted order (gather_idx == NULL), copy it (same alignment rule);
+                                 // 3: batch 1 only: copy x and gather_idx as in 1 and read x through the
+                                 // index array inside the multiply loop (no permutation pass)
 };
 
 // Shared memory the kernel needs for this (dtype, n_pad, batch); the caller falls back to the
 // chunked kernel when it exceeds kStreamSmemLimit.
-size_t stream_smem_bytes(pp_dtype_t dt, int B, int n_pad, int batch);
+size_t stream_smem_bytes(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode);
+extern int g_stream_depth;   // weight-ring slots per warp: 4, 6 or 8
+extern int g_stream_pdl;     // 1: launch with programmatic stream serialization
 constexpr size_t kStreamSmemLimit = 200 * 1024;
 
-cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a, int grid, cudaStream_t stream);
+// host_table: the plan's CTA ranges in host memory (grid entries); small plans travel to the
+// kernel inside its parameters so that no CTA starts with a dependent global load.
+cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a, const CtaDesc* host_table, int grid,
+                          cudaStream_t stream);
 
 }  // namespace pp

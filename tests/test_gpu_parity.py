@@ -85,6 +85,22 @@ def test_small_layers(pb, dtype, B, batch, persistent):
 
 
 @pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("B", [16, 32, 64])
+@pytest.mark.parametrize("direct,depth", [(0, 4), (1, 8), (0, 8)])
+def test_persistent_kernel_batch1_variants(pb, dtype, B, direct, depth):
+    """Batch 1 with x permuted in shared memory first (direct=0) or read through the index array in
+    the multiply loop (direct=1, the default), and with 4 or 8 weight copies in flight per warp."""
+    pb.pp_set_tuning(7, direct); pb.pp_set_tuning(6, depth)
+    try:
+        lay = _rand_layer(70 + B, 7 * B - 3, 11 * B - 9, B, dtype, density=0.5, empty_rows=(1,))
+        x = np.random.default_rng(B).uniform(-1, 1, (1, lay.N)).astype(dtype)
+        for act in (0, 1):
+            _run_and_check(pb, lay, x, act, f"direct={direct} depth={depth} B={B}")
+    finally:
+        pb.pp_set_tuning(7, 1); pb.pp_set_tuning(6, 4)
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float16])
 @pytest.mark.parametrize("ctas,min_frags,snap", [(296, 1, 0), (5, 1, 0), (37, 4, 50), (2000, 1, 25)])
 def test_persistent_kernel_partitions(pb, dtype, ctas, min_frags, snap):
     """CTA ranges that cut strips in the middle (cross-CTA partial sums), that snap to strip
@@ -97,7 +113,7 @@ def test_persistent_kernel_partitions(pb, dtype, ctas, min_frags, snap):
                 x = np.random.default_rng(batch).uniform(-1, 1, (batch, lay.N)).astype(dtype)
                 _run_and_check(pb, lay, x, 1, f"ctas={ctas} B={B} batch={batch}")
     finally:
-        pb.pp_set_tuning(2, 296); pb.pp_set_tuning(3, 128); pb.pp_set_tuning(4, 25)
+        pb.pp_set_tuning(2, 296); pb.pp_set_tuning(3, 128); pb.pp_set_tuning(4, -1)
 
 
 @pytest.mark.parametrize("dtype", [np.float32, np.float16])
@@ -152,7 +168,7 @@ def test_deterministic_and_canaries(pb, persistent):
         lay = _rand_layer(9, 777, 1111, 32, np.float16, density=0.5)
         L = pb.Layer.from_synth(lay)
     finally:
-        pb.pp_set_tuning(0, 32); pb.pp_set_tuning(4, 25)
+        pb.pp_set_tuning(0, 32); pb.pp_set_tuning(4, -1)
     x = _dev(np.random.default_rng(1).uniform(-1, 1, (3, lay.N)).astype(np.float16))
     pad = 64
     buf = torch.full((3 * lay.M + 2 * pad,), 12345.0, dtype=torch.float32, device="cuda")

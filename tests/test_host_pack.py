@@ -374,7 +374,7 @@ def test_stream_plan_walk_matches_oracle(dtype, B, ctas, min_frags, snap):
         lay.tile_values = lay.tile_values[:len(lay.tile_list)]
         pk = _pack(lay)
     finally:
-        pb.pp_set_tuning(2, 296); pb.pp_set_tuning(3, 128); pb.pp_set_tuning(4, 25)
+        pb.pp_set_tuning(2, 296); pb.pp_set_tuning(3, 128); pb.pp_set_tuning(4, -1)
     x = np.random.default_rng(1).uniform(-1, 1, lay.N).astype(dtype)
     got = _emulate_stream(pk, x.astype(np.float64), 1, dtype)
     y, _, a = po.layer_forward(lay, x.astype(np.float64), act=1)
