@@ -163,6 +163,41 @@ pp_status_t pp_chain_destroy(pp_chain_t* chain);
 pp_status_t pp_chain_forward(pp_chain_t* chain, const void* x, void* y, int batch,
                              void* cuda_stream);
 
+/* ------------------------------------------------------------------------- *
+ * Forward call that allocates nothing (the paper has no counterpart; this is a
+ * packaging of pp_forward's small-batch kernel).
+ *
+ * For callers that may not allocate device memory where they run inference: a
+ * real-time loop that owns one fixed arena, a process whose device memory pool
+ * belongs to another runtime, a context in which cudaMalloc's implicit
+ * synchronisation is forbidden.  Such a caller
+ *   1. packs the layer on the host (pp_pack_create),
+ *   2. asks for the size of the layer's device image (pp_pack_device_image_bytes),
+ *      writes the image into host memory (pp_pack_device_image) and copies it to
+ *      device memory it owns, 256-byte aligned,
+ *   3. calls pp_forward_noalloc with that device pointer.
+ * The scratch memory that CTAs sharing a strip of rows reduce through is a fixed
+ * array of 1 MiB inside the library, resident on every GPU that loads it.
+ * pp_forward_noalloc calls no cudaMalloc / cudaFree and no allocating routine.
+ *
+ * p             host, a packed layer; must stay alive while calls are in flight
+ * device_image  device, the uploaded image of p (pp_pack_device_image), 256-byte aligned
+ * x, y, act, cuda_stream   as pp_forward; batch must be 1..8
+ * Errors: PP_ERR_UNSUPPORTED when batch > 8, when the layer's reduction scratch
+ * (shared strips x rows x 8 floats, plus one counter per strip) exceeds the
+ * 1 MiB array, when its plan has more than 320 CTAs or when x does not fit
+ * shared memory; PP_ERR_INVALID_ARG for NULL / misaligned pointers;
+ * PP_ERR_CUDA when a runtime call fails.
+ * The first call on a device looks up the array's device address; make that call
+ * before any stream capture.  All calls on a device share the array: it is re-
+ * initialised by two memsets enqueued ahead of the kernel, and two calls that
+ * overlap on the GPU (different streams) race on it. */
+pp_status_t pp_pack_device_image_bytes(const pp_packed_t* p, int64_t* bytes);
+pp_status_t pp_pack_device_image(const pp_packed_t* p, void* host_dst, int64_t bytes);
+pp_status_t pp_forward_noalloc(const pp_packed_t* p, const void* device_image,
+                               const void* x, void* y, int batch, pp_act_t act,
+                               void* cuda_stream);
+
 /* Tuning knobs read at pack / create time (process-wide; for experiments).
  * key 0: target kilobytes of tile values per work item (default 32)
  * key 1: lower bound on the number of work items the splitter aims for (default 296)

@@ -63,6 +63,9 @@ def lib() -> ctypes.CDLL:
         "pp_chain_destroy": (ci, [vp]),
         "pp_chain_forward": (ci, [vp, vp, vp, ci, vp]),
         "pp_set_tuning": (ci, [ci, ci]),
+        "pp_pack_device_image_bytes": (ci, [vp, i64p]),
+        "pp_pack_device_image": (ci, [vp, vp, c64]),
+        "pp_forward_noalloc": (ci, [vp, vp, vp, vp, ci, ci, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(L, name)
@@ -142,6 +145,15 @@ class Packed:
         _check(lib().pp_pack_unpack(self._h, tl.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
                                     tv.ctypes.data_as(ctypes.c_void_p)), "pp_pack_unpack")
         return tl, tv
+
+    def device_image(self) -> np.ndarray:
+        """Host copy of the layer image that pp_forward_noalloc reads from device memory."""
+        n = ctypes.c_int64()
+        _check(lib().pp_pack_device_image_bytes(self._h, ctypes.byref(n)), "pp_pack_device_image_bytes")
+        img = np.empty(n.value, dtype=np.uint8)
+        _check(lib().pp_pack_device_image(self._h, img.ctypes.data_as(ctypes.c_void_p), n.value),
+               "pp_pack_device_image")
+        return img
 
     def close(self):
         if self._h:
@@ -245,6 +257,24 @@ def pp_forward(layer: Layer, x, act: int = PP_ACT_IDENTITY, out=None, stream=Non
     _check(lib().pp_forward(layer._h, ctypes.c_void_p(x2.data_ptr()), ctypes.c_void_p(y.data_ptr()),
                             batch, int(act), _stream_ptr(stream)), "pp_forward")
     return y
+
+
+def pp_forward_noalloc(packed: Packed, device_image, x, act: int = PP_ACT_IDENTITY, out=None, stream=None):
+    """pp_forward for callers that may not allocate: `device_image` is a CUDA uint8 tensor holding
+    packed.device_image(); `out` must be given (this function creates no tensor)."""
+    import torch
+    x2 = _check_x(x, packed.N, packed.wdtype)
+    batch = x2.shape[0]
+    if out is None:
+        raise ValueError("out must be provided: this entry point allocates nothing")
+    _require_cuda(out, "out")
+    _require_cuda(device_image, "device_image")
+    if out.dtype != torch.float32 or out.numel() != batch * packed.M:
+        raise ValueError("out must be float32 [batch][M]")
+    _check(lib().pp_forward_noalloc(packed._h, ctypes.c_void_p(device_image.data_ptr()),
+                                    ctypes.c_void_p(x2.data_ptr()), ctypes.c_void_p(out.data_ptr()),
+                                    batch, int(act), _stream_ptr(stream)), "pp_forward_noalloc")
+    return out
 
 
 class Chain:
