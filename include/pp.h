@@ -164,6 +164,29 @@ pp_status_t pp_chain_forward(pp_chain_t* chain, const void* x, void* y, int batc
                              void* cuda_stream);
 
 /* ------------------------------------------------------------------------- *
+ * Recurrent use: one pivoted layer as the gate matrix of an LSTM cell.  The
+ * paper names recurrent networks only as users of FC layers; the cell below is
+ * the usual one.  With z_t = [x_t ; h_{t-1}] (I + H entries) and g = W z_t
+ * (4H rows, original order: [0,H) input gate i, [H,2H) forget gate f, [2H,3H)
+ * candidate g, [3H,4H) output gate o; a bias given to the layer is part of g):
+ *     c_t = sig(f) c_{t-1} + sig(i) tanh(g),     h_t = sig(o) tanh(c_t).
+ * Following Section 4.2.1 the recurrence keeps z in the layer's pivoted column
+ * order for all steps: the matrix-vector kernel reads it without a gather and
+ * the gate kernel writes h_t straight to the pivoted positions step t+1 reads.
+ * gates: a layer with M = 4H, N = I + H; it must outlive the handle.  Buffers
+ * for max_steps steps are allocated at create.
+ * x_seq  device, [steps][I], element type of the layer, 16-byte aligned
+ * h      device, [H], element type of the layer: in h_0, out h_T (h is stored
+ *        rounded to that type after every step, because it is a layer input)
+ * c      device, float[H]: in c_0, out c_T
+ * Enqueues 1 + 2*steps kernels on the stream; no synchronisation. */
+typedef struct pp_lstm pp_lstm_t;
+pp_status_t pp_lstm_create(pp_lstm_t** out, pp_layer_t* gates, int I, int H, int max_steps);
+pp_status_t pp_lstm_destroy(pp_lstm_t* lstm);
+pp_status_t pp_lstm_forward(pp_lstm_t* lstm, const void* x_seq, void* h, float* c, int steps,
+                            void* cuda_stream);
+
+/* ------------------------------------------------------------------------- *
  * Forward call that allocates nothing (the paper has no counterpart; this is a
  * packaging of pp_forward's small-batch kernel).
  *

@@ -63,6 +63,9 @@ def lib() -> ctypes.CDLL:
         "pp_chain_destroy": (ci, [vp]),
         "pp_chain_forward": (ci, [vp, vp, vp, ci, vp]),
         "pp_set_tuning": (ci, [ci, ci]),
+        "pp_lstm_create": (ci, [ctypes.POINTER(vp), vp, ci, ci, ci]),
+        "pp_lstm_destroy": (ci, [vp]),
+        "pp_lstm_forward": (ci, [vp, vp, vp, vp, ci, vp]),
         "pp_pack_device_image_bytes": (ci, [vp, i64p]),
         "pp_pack_device_image": (ci, [vp, vp, c64]),
         "pp_forward_noalloc": (ci, [vp, vp, vp, vp, ci, ci, vp]),
@@ -318,3 +321,43 @@ def pp_chain_forward(chain: Chain, x, out=None, stream=None):
     _check(lib().pp_chain_forward(chain._h, ctypes.c_void_p(x2.data_ptr()), ctypes.c_void_p(y.data_ptr()),
                                   batch, _stream_ptr(stream)), "pp_chain_forward")
     return y
+
+
+class Lstm:
+    """LSTM cell around one pivoted gate layer (pp_lstm_create / pp_lstm_forward)."""
+
+    def __init__(self, gates: Layer, I: int, H: int, max_steps: int):
+        self.gates = gates                  # keep the layer alive
+        self.I, self.H, self.max_steps = int(I), int(H), int(max_steps)
+        self._h = ctypes.c_void_p()
+        _check(lib().pp_lstm_create(ctypes.byref(self._h), gates._h, self.I, self.H, self.max_steps), "pp_lstm_create")
+
+    def forward(self, x_seq, h, c, stream=None):
+        return pp_lstm_forward(self, x_seq, h, c, stream=stream)
+
+    def close(self):
+        if self._h:
+            lib().pp_lstm_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def pp_lstm_forward(lstm: Lstm, x_seq, h, c, stream=None):
+    """Runs x_seq.shape[0] steps; h (layer dtype, [H]) and c (float32, [H]) are updated in place."""
+    import torch
+    for t, name in ((x_seq, "x_seq"), (h, "h"), (c, "c")):
+        _require_cuda(t, name)
+    want = torch.float16 if lstm.gates.wdtype == np.float16 else torch.float32
+    if x_seq.dtype != want or h.dtype != want or c.dtype != torch.float32:
+        raise TypeError("x_seq and h must have the layer's element type, c must be float32")
+    if x_seq.dim() != 2 or x_seq.shape[1] != lstm.I or h.numel() != lstm.H or c.numel() != lstm.H:
+        raise ValueError("x_seq must be [steps][I], h and c [H]")
+    _check(lib().pp_lstm_forward(lstm._h, ctypes.c_void_p(x_seq.data_ptr()), ctypes.c_void_p(h.data_ptr()),
+                                 ctypes.c_void_p(c.data_ptr()), int(x_seq.shape[0]), _stream_ptr(stream)),
+           "pp_lstm_forward")
+    return h, c

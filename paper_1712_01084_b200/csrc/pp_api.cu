@@ -7,6 +7,7 @@
 
 #include "pp_gemv.cuh"
 #include "pp_internal.h"
+#include "pp_lstm.cuh"
 #include "pp_stream.cuh"
 
 struct pp_layer {
@@ -37,6 +38,15 @@ struct pp_layer {
     int max_item_tiles = 0;
     int stream_grid = 0;
     int stream_max_rows = 0;       // most pivoted rows one CTA of the persistent plan lists
+};
+
+struct pp_lstm {
+    pp_layer* gates = nullptr;
+    int I = 0, H = 0, max_steps = 0;
+    int32_t* d_inv_row = nullptr;
+    int32_t* d_inv_col = nullptr;
+    void* d_z = nullptr;           // [max_steps + 1][N_pad] inputs of every step in pivoted order
+    float* d_g = nullptr;          // [M_pad] gate pre-activations in pivoted order
 };
 
 struct pp_chain {
@@ -127,8 +137,9 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 // Enqueue one layer in groups of batch columns.
 pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_len, int x_elt, void* y, int ldy,
-                      int out_mode, int batch, pp_act_t act, cudaStream_t stream) {
+                      int out_mode, int batch, pp_act_t act, cudaStream_t stream, int x_limit = -1) {
     const pp_packed* pk = L->pk;
+    if (x_limit < 0) x_limit = pk->N;      // without a gather map: columns at or beyond x_limit read 0
     int stage_mode = -1;
     if (pp::g_use_stream && batch <= pp::kStreamMaxBatch) {
         const bool rows_aligned = aligned16(x) && (batch == 1 || ((size_t)ldx * x_elt) % 16 == 0);
@@ -145,7 +156,7 @@ pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx
         s.cta_desc = L->d_cta_desc; s.strip_info = L->d_strip_info;
         s.gather_idx = gather; s.scatter_idx = L->d_scatter; s.bias_piv = L->d_bias;
         s.x = x; s.y = y; s.partials = L->d_spartials; s.counters = L->d_scounters;
-        s.ldx = ldx; s.ldy = ldy; s.x_limit = pk->N; s.n_pad = pk->Npad; s.x_len = x_len; s.max_rows = L->stream_max_rows; s.batch = batch;
+        s.ldx = ldx; s.ldy = ldy; s.x_limit = x_limit; s.n_pad = pk->Npad; s.x_len = x_len; s.max_rows = L->stream_max_rows; s.batch = batch;
         s.act = (int)act; s.out_mode = out_mode;
         return pp::launch_stream(pk->wdtype, pk->B, s, pk->cta_desc.data(), L->stream_grid, stream) == cudaSuccess
                    ? PP_OK : PP_ERR_CUDA;
@@ -154,7 +165,7 @@ pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx
     a.values = L->d_values; a.items = L->d_items; a.tile_col = L->d_tile_col;
     a.gather_idx = gather; a.scatter_idx = L->d_scatter; a.bias_piv = L->d_bias;
     a.partials = L->d_partials; a.counters = L->d_counters;
-    a.ldx = ldx; a.ldy = ldy; a.x_limit = pk->N; a.act = (int)act; a.out_mode = out_mode;
+    a.ldx = ldx; a.ldy = ldy; a.x_limit = x_limit; a.act = (int)act; a.out_mode = out_mode;
     const int group = pp::gemv_group_batch(pk->wdtype);
     const int y_elt = out_mode == pp::OUT_PIVOTED_F16 ? 2 : 4;
     for (int b0 = 0; b0 < batch; b0 += group) {
@@ -322,6 +333,61 @@ pp_status_t pp_chain_forward(pp_chain_t* C, const void* x, void* y, int batch, v
             cur = C->d_inter[(size_t)l];
         }
         if (st != PP_OK) return st;
+    }
+    return PP_OK;
+}
+
+pp_status_t pp_lstm_create(pp_lstm_t** out, pp_layer_t* gates, int I, int H, int max_steps) {
+    if (!out) return PP_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!gates || I < 1 || H < 1 || max_steps < 1) return PP_ERR_INVALID_ARG;
+    const pp_packed* pk = gates->pk;
+    if (pk->M != 4 * H || pk->N != I + H) return PP_ERR_INVALID_ARG;
+    pp_lstm* R = new (std::nothrow) pp_lstm();
+    if (!R) return PP_ERR_ALLOC;
+    R->gates = gates; R->I = I; R->H = H; R->max_steps = max_steps;
+    std::vector<int32_t> inv_col((size_t)pk->Npad);
+    for (int j = 0; j < pk->Npad; ++j) inv_col[(size_t)pk->col_perm[(size_t)j]] = j;
+    const size_t elt = pk->wdtype == PP_F16 ? 2 : 4;
+    const bool ok = upload(&R->d_inv_row, pk->inv_row_perm.data(), pk->inv_row_perm.size() * 4) &&
+                    upload(&R->d_inv_col, inv_col.data(), inv_col.size() * 4) &&
+                    cudaMalloc(&R->d_z, (size_t)(max_steps + 1) * pk->Npad * elt) == cudaSuccess &&
+                    cudaMalloc(reinterpret_cast<void**>(&R->d_g), (size_t)pk->Mpad * 4) == cudaSuccess;
+    if (!ok) {
+        const cudaError_t e = cudaGetLastError();
+        pp_lstm_destroy(R);
+        return e == cudaErrorMemoryAllocation ? PP_ERR_ALLOC : PP_ERR_CUDA;
+    }
+    *out = R;
+    return PP_OK;
+}
+
+pp_status_t pp_lstm_destroy(pp_lstm_t* R) {
+    if (!R) return PP_OK;
+    cudaFree(R->d_inv_row); cudaFree(R->d_inv_col); cudaFree(R->d_z); cudaFree(R->d_g);
+    delete R;
+    return PP_OK;
+}
+
+pp_status_t pp_lstm_forward(pp_lstm_t* R, const void* x_seq, void* h, float* c, int steps, void* cuda_stream) {
+    if (!R || !x_seq || !h || !c || steps < 1 || steps > R->max_steps) return PP_ERR_INVALID_ARG;
+    if (!aligned16(x_seq) || !aligned16(h) || !aligned16(c)) return PP_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    pp_layer* L = R->gates;
+    const pp_packed* pk = L->pk;
+    const int elt = pk->wdtype == PP_F16 ? 2 : 4;
+    pp::LstmArgs a{};
+    a.gather_idx = L->d_gather; a.inv_row = R->d_inv_row; a.inv_col = R->d_inv_col;
+    a.z = R->d_z; a.x_seq = x_seq; a.h = h; a.c = c; a.g_piv = R->d_g;
+    a.I = R->I; a.H = R->H; a.n_pad = pk->Npad; a.steps = steps; a.f16 = pk->wdtype == PP_F16;
+    if (pp::launch_lstm_prepare(a, stream) != cudaSuccess) return PP_ERR_CUDA;
+    for (int t = 0; t < steps; ++t) {
+        const char* zt = static_cast<const char*>(R->d_z) + (size_t)t * pk->Npad * elt;
+        // the input is already in pivoted order: no gather map, every pivoted column is real
+        pp_status_t st = run_layer(L, nullptr, zt, pk->Npad, pk->Npad, elt, R->d_g, pk->Mpad, pp::OUT_PIVOTED_F32, 1,
+                                   PP_ACT_IDENTITY, stream, pk->Npad);
+        if (st != PP_OK) return st;
+        if (pp::launch_lstm_gates(a, t, stream) != cudaSuccess) return PP_ERR_CUDA;
     }
     return PP_OK;
 }
