@@ -195,6 +195,98 @@ def time_graph(pb, torch, replicas, x, y, act, steps, warmup, chunk=500):
         return stream, graphs, chunk, e0, e1
 
 
+def time_enqueue(torch, enqueue, calls_per_graph, replays=20):
+    """Mean device time (us) of one call: `enqueue(i, stream_ptr)` is captured `calls_per_graph`
+    times into a CUDA graph that is replayed `replays` times between two events."""
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        sp = ctypes.c_void_p(stream.cuda_stream)
+        for i in range(calls_per_graph):
+            enqueue(i, sp)                               # warm-up, plain launches
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            cp = ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+            for i in range(calls_per_graph):
+                enqueue(i, cp)
+        g.replay()
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(replays):
+            g.replay()
+        e1.record(stream)
+        stream.synchronize()
+    return e0.elapsed_time(e1) * 1e3 / (replays * calls_per_graph)
+
+
+def other_workloads(pb, torch, synth):
+    """Latency of the other synthetic workloads: cold (calls rotate over copies of the layers that
+    together exceed twice the L2) and warm (one copy, weights may sit in L2)."""
+    out = {}
+
+    def check(st):
+        if st != 0:
+            raise pb.PPError(st, "forward")
+
+    def layer_case(name, wl, batch):
+        lay = wl.layers[0]
+        L0 = pb.Layer.from_synth(lay)
+        wbytes = lay.T * lay.B * lay.B * lay.tile_values.dtype.itemsize
+        R = max(2, -(-2 * L2_BYTES // wbytes) + 1)
+        reps = [L0] + [L0.clone() for _ in range(R - 1)]
+        x = torch.from_numpy(wl.x).cuda()
+        y = torch.empty((batch, lay.M), dtype=torch.float32, device="cuda")
+        fn = pb.lib().pp_forward
+        cold = time_enqueue(torch, lambda i, sp: check(fn(reps[i % R]._h, x.data_ptr(), y.data_ptr(), batch, lay.act, sp)), R * max(1, 64 // R))
+        warm = time_enqueue(torch, lambda i, sp: check(fn(L0._h, x.data_ptr(), y.data_ptr(), batch, lay.act, sp)), 64)
+        pk = pb.Packed(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values, lay.bias)
+        ab = algorithmic_bytes(lay, batch, pk.n_tile_col)
+        out[name] = {"us_cold": round(cold, 3), "us_warm": round(warm, 3), "GBps_cold": round(ab / cold / 1e3, 1),
+                     "algorithmic_bytes": ab, "copies": R}
+        for r in reps:
+            r.close()
+
+    layer_case("cfg1_fc1024_f32_b32_d25_batch1", synth.config1(), 1)
+    layer_case("cfg2_fc4096_f32_b64_d12.5_batch1", synth.config2(), 1)
+    for batch in (16, 128):
+        layer_case(f"cfg5_fc8192_f16_b64_k128_batch{batch}", synth.config5(k=128, batch=batch), batch)
+
+    for batch in (1, 8):
+        wl = synth.config3(batch=batch)
+        wbytes = sum(l.T * l.B * l.B * 2 for l in wl.layers)
+        R = -(-2 * L2_BYTES // wbytes) + 1
+        chains = []
+        for _ in range(R):
+            layers = [pb.Layer.from_synth(l) for l in wl.layers] if not chains else [l.clone() for l in chains[0].layers]
+            chains.append(pb.Chain(layers, [l.act for l in wl.layers], max_batch=8))
+        x = torch.from_numpy(wl.x).cuda()
+        y = torch.empty((batch, wl.layers[-1].M), dtype=torch.float32, device="cuda")
+        fn = pb.lib().pp_chain_forward
+        cold = time_enqueue(torch, lambda i, sp: check(fn(chains[i % R]._h, x.data_ptr(), y.data_ptr(), batch, sp)), R * 2)
+        warm = time_enqueue(torch, lambda i, sp: check(fn(chains[0]._h, x.data_ptr(), y.data_ptr(), batch, sp)), 32)
+        out[f"cfg3_chain_batch{batch}"] = {"us_cold": round(cold, 3), "us_warm": round(warm, 3), "layers": 3,
+                                            "us_per_layer_cold": round(cold / 3, 3), "tile_bytes": wbytes, "copies": R}
+        for c in chains:
+            c.close()
+            for l in c.layers:
+                l.close()
+
+    wl = synth.config4(steps=256)
+    lay, H, I = wl.layers[0], wl.extra["H"], wl.extra["I"]
+    L = pb.Layer.from_synth(lay)
+    cell = pb.Lstm(L, I, H, max_steps=256)
+    xs = torch.from_numpy(wl.x).cuda()
+    h = torch.zeros(H, dtype=torch.float16, device="cuda")
+    c = torch.zeros(H, dtype=torch.float32, device="cuda")
+    fn = pb.lib().pp_lstm_forward
+    us = time_enqueue(torch, lambda i, sp: check(fn(cell._h, xs.data_ptr(), h.data_ptr(), c.data_ptr(), 256, sp)), 1, replays=5)
+    out["cfg4_lstm_256_steps"] = {"us_total": round(us, 1), "us_per_step": round(us / 256, 3),
+                                  "tile_bytes_per_step": lay.T * lay.B * lay.B * 2, "note": "weights L2-resident across steps"}
+    cell.close(); L.close()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -204,6 +296,7 @@ def main():
     ap.add_argument("--k", type=int, default=128, help="kept tiles per block-row (of 128)")
     ap.add_argument("--no-sweep", action="store_true", help="skip the density sweep")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    ap.add_argument("--no-configs", action="store_true", help="skip the other synthetic workloads")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -332,6 +425,11 @@ def main():
                                        "speedup_vs_dense": None if base is None else round(base / us_k, 3),
                                        "linearity": None if base is None else round(base / us_k * k / 128, 3)}
         out["density_sweep"] = sweep
+
+    if rank == 0 and world == 1 and not args.no_configs:
+        for r in reps:
+            r.close()
+        out["other_workloads"] = other_workloads(pb, torch, synth)
 
     if rank == 0 and world == 1 and not args.no_cpu:
         wl0 = synth.config5(k=args.k, batch=1)

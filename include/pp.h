@@ -133,6 +133,10 @@ pp_status_t pp_layer_create(pp_layer_t** out, int M, int N, int B,
                             const float* bias);
 pp_status_t pp_layer_destroy(pp_layer_t* layer);
 
+/* Raised by a kernel whose bounded device-side wait gave up (the call's output is then invalid).
+ * Synchronises with the device; *status is PP_OK or PP_ERR_TIMEOUT.  The flag is cleared by the read. */
+pp_status_t pp_layer_status(pp_layer_t* layer, pp_status_t* status);
+
 /* Independent device copy of a layer (own weights, index arrays and scratch), e.g. to
  * serve several streams at once or to rotate copies so that repeated timing runs do not
  * find the weights in L2.  Errors: PP_ERR_INVALID_ARG, PP_ERR_ALLOC, PP_ERR_CUDA. */
@@ -141,9 +145,10 @@ pp_status_t pp_layer_clone(pp_layer_t** out, const pp_layer_t* src);
 /* y = act(W x + b) (Eq. 2, Listing 1 with both permutations).
  * x   device, [batch][N] row-major, element type = the layer's wdtype, 16-byte aligned
  * y   device, [batch][M] row-major, float, must not alias x
- * batch >= 1.  batch < 64 (and every fp32 layer) runs the streaming
- * matrix-vector kernel in groups of up to 32 columns; fp16 layers with B = 64
- * and batch >= 64 run the tensor-core tile kernel.
+ * batch >= 1.  batch <= 8 runs the persistent matrix-vector kernel; larger batches run it in
+ * groups of 8 columns or the chunked kernel in groups of up to 32; fp16 layers with B = 64 and
+ * batch >= 64 run the tensor-core tile kernel in chunks of 128 rows (such layers keep a second,
+ * row-major copy of their tiles on the device for it).
  * cuda_stream: a cudaStream_t (NULL = default stream).  Enqueues only. */
 pp_status_t pp_forward(pp_layer_t* layer, const void* x, void* y, int batch,
                        pp_act_t act, void* cuda_stream);
@@ -233,7 +238,8 @@ pp_status_t pp_forward_noalloc(const pp_packed_t* p, const void* device_image,
  * key 6: asynchronous 512-byte weight copies each warp of the persistent kernel keeps in flight: 4 (default) or 8
  * key 7: batch 1 in the persistent kernel: 1 (default) reads x through the index array inside the multiply
  *        loop, 0 permutes x into pivoted order in shared memory first (what batch 2..8 always do)
- * key 8: 1 (default) launches the persistent kernel with programmatic stream serialization, 0 plainly */
+ * key 8: 1 (default) launches the persistent kernel with programmatic stream serialization, 0 plainly
+ * key 9: smallest batch for which fp16 layers with B = 64 take the tensor-core tile path (default 64; 0 = never) */
 pp_status_t pp_set_tuning(int key, int value);
 
 #ifdef __cplusplus

@@ -58,6 +58,7 @@ def lib() -> ctypes.CDLL:
         "pp_layer_create": (ci, create_args),
         "pp_layer_destroy": (ci, [vp]),
         "pp_layer_clone": (ci, [ctypes.POINTER(vp), vp]),
+        "pp_layer_status": (ci, [vp, ctypes.POINTER(ci)]),
         "pp_forward": (ci, [vp, vp, vp, ci, ci, vp]),
         "pp_chain_create": (ci, [ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(ci), ci, ci]),
         "pp_chain_destroy": (ci, [vp]),
@@ -218,6 +219,12 @@ class Layer:
 
     def forward(self, x, act: int = PP_ACT_IDENTITY, out=None, stream=None):
         return pp_forward(self, x, act, out=out, stream=stream)
+
+    def status(self) -> int:
+        """PP_OK, or PP_ERR_TIMEOUT when a kernel's bounded wait gave up (synchronises; clears the flag)."""
+        st = ctypes.c_int(0)
+        _check(lib().pp_layer_status(self._h, ctypes.byref(st)), "pp_layer_status")
+        return st.value
 
     def close(self):
         if self._h:

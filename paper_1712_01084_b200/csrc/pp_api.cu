@@ -9,6 +9,7 @@
 #include "pp_internal.h"
 #include "pp_lstm.cuh"
 #include "pp_stream.cuh"
+#include "pp_tile.cuh"
 
 struct pp_layer {
     pp_packed* pk = nullptr;       // host copy (index arrays are needed again when chains are folded)
@@ -38,6 +39,17 @@ struct pp_layer {
     int max_item_tiles = 0;
     int stream_grid = 0;
     int stream_max_rows = 0;       // most pivoted rows one CTA of the persistent plan lists
+    // tensor-core tile path (fp16, B = 64): row_ptr, col_ptr and the row-major tiles in one block,
+    // the permuted-input chunk and the status word in another
+    unsigned char* d_tile = nullptr;
+    size_t tile_bytes = 0;
+    int32_t* d_row_ptr = nullptr;
+    int32_t* d_col_ptr = nullptr;
+    void* d_tiles_rm = nullptr;
+    unsigned char* d_tile_scratch = nullptr;
+    void* d_x_piv = nullptr;
+    int* d_status = nullptr;
+    pp::TilePlan* tile_plan = nullptr;
 };
 
 struct pp_lstm {
@@ -71,6 +83,9 @@ void free_layer(pp_layer* L) {
     if (!L) return;
     cudaFree(L->d_arena);
     cudaFree(L->d_scratch);
+    cudaFree(L->d_tile);
+    cudaFree(L->d_tile_scratch);
+    pp::tile_plan_destroy(L->tile_plan);
     pp_pack_destroy(L->pk);
     delete L;
 }
@@ -130,6 +145,35 @@ bool alloc_layer(pp_layer* L, const LayerLayout& lo) {
     L->d_counters = reinterpret_cast<int*>(sc + lo.soff[1]);
     L->d_spartials = reinterpret_cast<float*>(sc + lo.soff[2]);
     L->d_scounters = reinterpret_cast<int*>(sc + lo.soff[3]);
+    return true;
+}
+
+// Device blocks and tensor maps of the tensor-core tile path.  `host` uploads from the packed layer,
+// otherwise the weights block is copied from another layer's.  A layer that is not eligible, or a
+// driver without the tensor-map encoder, simply has no tile path (tile_plan stays NULL).
+bool tile_setup(pp_layer* L, const pp_layer* from) {
+    const pp_packed* pk = L->pk;
+    if (pk->wdtype != PP_F16 || pk->B != 64) return true;
+    const size_t rp = round256((size_t)(pk->Mb + 1) * 4), tb = (size_t)pk->T * 64 * 64 * 2;
+    L->tile_bytes = 2 * rp + round256(tb);
+    if (cudaMalloc(reinterpret_cast<void**>(&L->d_tile), L->tile_bytes) != cudaSuccess) return false;
+    const size_t xb = round256((size_t)pp::kTileBatch * pk->Npad * 2);
+    if (cudaMalloc(reinterpret_cast<void**>(&L->d_tile_scratch), xb + 256) != cudaSuccess) return false;
+    if (cudaMemset(L->d_tile_scratch, 0, xb + 256) != cudaSuccess) return false;
+    L->d_row_ptr = reinterpret_cast<int32_t*>(L->d_tile);
+    L->d_col_ptr = reinterpret_cast<int32_t*>(L->d_tile + rp);
+    L->d_tiles_rm = L->d_tile + 2 * rp;
+    L->d_x_piv = L->d_tile_scratch;
+    L->d_status = reinterpret_cast<int*>(L->d_tile_scratch + xb);
+    if (from) {
+        if (cudaMemcpy(L->d_tile, from->d_tile, L->tile_bytes, cudaMemcpyDeviceToDevice) != cudaSuccess) return false;
+    } else {
+        if (cudaMemcpy(L->d_row_ptr, pk->row_ptr.data(), (size_t)(pk->Mb + 1) * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(L->d_col_ptr, pk->col_ptr.data(), (size_t)(pk->Mb + 1) * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+            (tb && cudaMemcpy(L->d_tiles_rm, pk->tiles_rm.data(), tb, cudaMemcpyHostToDevice) != cudaSuccess))
+            return false;
+    }
+    L->tile_plan = pp::tile_plan_create(L->d_tiles_rm, pk->T, L->d_x_piv, pk->Npad);
     return true;
 }
 
@@ -213,13 +257,15 @@ pp_status_t pp_layer_create(pp_layer_t** out, int M, int N, int B, const int32_t
         for (int i = 0; i < 10 && ok; ++i)
             ok = n[i] == 0 || cudaMemcpy(L->d_arena + lo.off[i], src[i], n[i], cudaMemcpyHostToDevice) == cudaSuccess;
     }
+    ok = ok && tile_setup(L, nullptr);
     if (!ok) {
         const cudaError_t e = cudaGetLastError();
         free_layer(L);
         return e == cudaErrorMemoryAllocation ? PP_ERR_ALLOC : PP_ERR_CUDA;
     }
-    // the fragment-ordered values and per-fragment offsets now live on the device; drop the host copies
+    // the tile values and per-fragment offsets now live on the device; drop the host copies
     std::vector<unsigned char>().swap(pk->values);
+    std::vector<unsigned char>().swap(pk->tiles_rm);
     std::vector<int32_t>().swap(pk->xoff);
     *out = L;
     return PP_OK;
@@ -239,13 +285,27 @@ pp_status_t pp_layer_clone(pp_layer_t** out, const pp_layer_t* src) {
     L->stream_max_rows = src->stream_max_rows;
     const LayerLayout lo = layer_layout(pk);
     const bool ok = lo.arena_bytes == src->arena_bytes && alloc_layer(L, lo) &&
-                    cudaMemcpy(L->d_arena, src->d_arena, lo.arena_bytes, cudaMemcpyDeviceToDevice) == cudaSuccess;
+                    cudaMemcpy(L->d_arena, src->d_arena, lo.arena_bytes, cudaMemcpyDeviceToDevice) == cudaSuccess &&
+                    tile_setup(L, src);
     if (!ok) {
         const cudaError_t e = cudaGetLastError();
         free_layer(L);
         return e == cudaErrorMemoryAllocation ? PP_ERR_ALLOC : PP_ERR_CUDA;
     }
     *out = L;
+    return PP_OK;
+}
+
+pp_status_t pp_layer_status(pp_layer_t* L, pp_status_t* status) {
+    if (!L || !status) return PP_ERR_INVALID_ARG;
+    *status = PP_OK;
+    if (!L->d_status) return PP_OK;
+    int flag = 0;
+    if (cudaMemcpy(&flag, L->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return PP_ERR_CUDA;
+    if (flag) {
+        *status = PP_ERR_TIMEOUT;
+        if (cudaMemset(L->d_status, 0, sizeof(int)) != cudaSuccess) return PP_ERR_CUDA;
+    }
     return PP_OK;
 }
 
@@ -259,8 +319,24 @@ pp_status_t pp_forward(pp_layer_t* L, const void* x, void* y, int batch, pp_act_
     if (act != PP_ACT_IDENTITY && act != PP_ACT_RELU) return PP_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(y)) return PP_ERR_INVALID_ARG;
     const pp_packed* pk = L->pk;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (L->tile_plan && pp::g_tile_min_batch > 0 && batch >= pp::g_tile_min_batch && (size_t)pk->N * 2 <= 48 * 1024) {
+        // tensor-core tile path, 128 batch rows at a time
+        pp::TileArgs t{};
+        t.row_ptr = L->d_row_ptr; t.col_ptr = L->d_col_ptr; t.tile_col = L->d_tile_col;
+        t.scatter_idx = L->d_scatter; t.bias_piv = L->d_bias; t.status = L->d_status;
+        t.ldy = pk->M; t.act = (int)act;
+        for (int b0 = 0; b0 < batch; b0 += pp::kTileBatch) {
+            t.batch = batch - b0 < pp::kTileBatch ? batch - b0 : pp::kTileBatch;
+            t.y = static_cast<float*>(y) + (size_t)b0 * pk->M;
+            const char* xc = static_cast<const char*>(x) + (size_t)b0 * pk->N * 2;
+            if (pp::launch_tile(L->tile_plan, t, xc, pk->N, pk->N, L->d_gather, pk->Npad, L->d_x_piv, pk->Mb, stream) != cudaSuccess)
+                return PP_ERR_CUDA;
+        }
+        return PP_OK;
+    }
     return run_layer(L, L->d_gather, x, pk->N, pk->N, pk->wdtype == PP_F16 ? 2 : 4, y, pk->M, pp::OUT_SCATTER_F32,
-                     batch, act, static_cast<cudaStream_t>(cuda_stream));
+                     batch, act, stream);
 }
 
 pp_status_t pp_chain_create(pp_chain_t** out, pp_layer_t* const* layers, const pp_act_t* acts, int n_layers,

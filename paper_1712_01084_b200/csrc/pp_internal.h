@@ -44,6 +44,7 @@ constexpr int kStreamMaxStrips = 48;      // strips one CTA may list
 constexpr int kStreamSegSlots = kStreamMaxStrips + kStreamWarps;   // (strip, warp) partial slots in shared memory
 constexpr int kStreamMaxBatch = 8;
 extern int g_use_stream;
+extern int g_tile_min_batch;  // fp16 B = 64 layers take the tensor-core tile path from this batch on (0: never)
 extern int g_stage_direct;   // batch 1: read x through the index array instead of permuting it first
 
 // Geometry of the fragment layout for a (dtype, B) pair.
@@ -74,6 +75,7 @@ struct pp_packed {
     std::vector<int32_t> gather_idx, scatter_idx;
     std::vector<float> bias_piv;
     std::vector<unsigned char> values;                       // fragment-ordered tile values
+    std::vector<unsigned char> tiles_rm;                     // fp16, B = 64 only: sorted tiles, row-major (tensor-core path)
     std::vector<pp::WorkItem> items;
     // plan of the persistent streaming kernel
     std::vector<int32_t> strip_start;   // [S+1] fragment position of each strip

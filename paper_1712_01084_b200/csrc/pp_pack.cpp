@@ -10,6 +10,7 @@
 
 namespace pp {
 int g_use_stream = 1;      // 0: the API never picks the persistent kernel
+int g_tile_min_batch = 64;
 int g_stage_direct = 1;    // 0: batch 1 also materialises the pivoted x in shared memory
 extern int g_stream_depth; // weight-ring slots per warp of the persistent kernel (pp_stream.cu)
 extern int g_stream_pdl;   // programmatic dependent launch of the persistent kernel (pp_stream.cu)
@@ -241,6 +242,7 @@ pp_status_t pp_set_tuning(int key, int value) {
     if (key == 6 && (value == 4 || value == 6 || value == 8)) { pp::g_stream_depth = value; return PP_OK; }
     if (key == 7 && (value == 0 || value == 1)) { pp::g_stage_direct = value; return PP_OK; }
     if (key == 8 && (value == 0 || value == 1)) { pp::g_stream_pdl = value; return PP_OK; }
+    if (key == 9 && value >= 0) { pp::g_tile_min_batch = value; return PP_OK; }
     return PP_ERR_INVALID_ARG;
 }
 
@@ -322,6 +324,12 @@ pp_status_t pp_pack_create(pp_packed_t** out, int M, int N, int B, const int32_t
                         std::memcpy(&p->values[frag * 512 + e.byte], tile + ((size_t)r * B + c) * esz, esz);
                     }
             }
+        }
+
+        if (wdtype == PP_F16 && B == 64) {       // row-major copy of the sorted tiles for the tensor-core path
+            p->tiles_rm.resize((size_t)T * B * B * 2);
+            for (int64_t s2 = 0; s2 < T; ++s2)
+                std::memcpy(&p->tiles_rm[(size_t)s2 * B * B * 2], src + (size_t)order[(size_t)s2] * B * B * 2, (size_t)B * B * 2);
         }
 
         p->gather_idx.resize((size_t)Npad);

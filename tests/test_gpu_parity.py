@@ -285,3 +285,48 @@ def test_config5_small_batch_sampled_rows(pb, batch):
     y_ref, a = po.dense_forward_rows(W, None, wl.x.astype(np.float64), 0, rows)
     _check(y[:, rows], y_ref, a, np.float16, "config 5 batch 16 sampled")
     L.close()
+
+
+# ------------------------------------------------------------------ tensor-core tile path (batch >= 64)
+@pytest.mark.parametrize("batch", [64, 100, 128, 129, 300])
+def test_tile_path_small_layer(pb, batch):
+    """fp16, B = 64: ragged sizes, unbalanced block-rows, one block-row without tiles, batch chunks of 128
+    with a ragged last chunk; compared element by element, and bit for bit on integer data."""
+    lay = _rand_layer(900 + batch, 5 * 64 - 3, 9 * 64 - 7, 64, np.float16, density=0.45, empty_rows=(2,))
+    x = np.random.default_rng(batch).uniform(-1, 1, (batch, lay.N)).astype(np.float16)
+    L = pb.Layer.from_synth(lay)
+    for act in (0, 1):
+        y = pb.pp_forward(L, _dev(x), act).cpu().numpy()
+        assert L.status() == 0
+        y_ref, _, a = po.layer_forward(lay, x.astype(np.float64), act=act, threads=8)
+        _check(y, y_ref, a, np.float16, f"tile path batch={batch} act={act}")
+    L.close()
+    lay = _rand_layer(950 + batch, 4 * 64 - 1, 6 * 64 - 5, 64, np.float16, density=0.5, integer=True)
+    x = np.random.default_rng(5).integers(-2, 3, (batch, lay.N)).astype(np.float16)
+    L = pb.Layer.from_synth(lay)
+    y = pb.pp_forward(L, _dev(x), 1).cpu().numpy()
+    y_ref, _, _ = po.layer_forward(lay, x.astype(np.float64), act=1, threads=8)
+    assert np.array_equal(y.astype(np.float64), y_ref)
+    # the same batch through the matrix-vector kernels gives the same integers
+    pb.pp_set_tuning(9, 0)
+    try:
+        y2 = pb.pp_forward(L, _dev(x), 1).cpu().numpy()
+    finally:
+        pb.pp_set_tuning(9, 64)
+    assert np.array_equal(y, y2)
+    L.close()
+
+
+def test_config5_batch128_tile_path_sampled_rows(pb):
+    """Full size (8192 x 8192, density 25 %), batch 128, in the launch configuration the bench times;
+    the oracle evaluates a sample of output rows."""
+    wl = synth.config5(k=32, batch=128)
+    lay = wl.layers[0]
+    L = pb.Layer.from_synth(lay)
+    y = pb.pp_forward(L, _dev(wl.x), 0).cpu().numpy()
+    assert L.status() == 0
+    W = po.reconstruct(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values)
+    rows = np.random.default_rng(0).choice(lay.M, 96, replace=False).astype(np.int32)
+    y_ref, a = po.dense_forward_rows(W, None, wl.x.astype(np.float64), 0, rows)
+    _check(y[:, rows], y_ref, a, np.float16, "config 5 batch 128 sampled")
+    L.close()
