@@ -49,7 +49,7 @@ struct pp_layer {
     unsigned char* d_tile_scratch = nullptr;
     void* d_x_piv = nullptr;
     int* d_status = nullptr;
-    pp::TilePlan* tile_plan = nullptr;
+    bool tile_ok = false;
 };
 
 struct pp_lstm {
@@ -85,7 +85,6 @@ void free_layer(pp_layer* L) {
     cudaFree(L->d_scratch);
     cudaFree(L->d_tile);
     cudaFree(L->d_tile_scratch);
-    pp::tile_plan_destroy(L->tile_plan);
     pp_pack_destroy(L->pk);
     delete L;
 }
@@ -170,48 +169,70 @@ bool tile_setup(pp_layer* L, const pp_layer* from) {
     } else {
         if (cudaMemcpy(L->d_row_ptr, pk->row_ptr.data(), (size_t)(pk->Mb + 1) * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
             cudaMemcpy(L->d_col_ptr, pk->col_ptr.data(), (size_t)(pk->Mb + 1) * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
-            (tb && cudaMemcpy(L->d_tiles_rm, pk->tiles_rm.data(), tb, cudaMemcpyHostToDevice) != cudaSuccess))
+            (tb && cudaMemcpy(L->d_tiles_rm, pk->tiles_rm.data(), tb, cudaMemcpyHostToDevice) != cudaSuccess))   // already swizzled by the packer
             return false;
     }
-    L->tile_plan = pp::tile_plan_create(L->d_tiles_rm, pk->T, L->d_x_piv, pk->Npad);
+    L->tile_ok = true;
     return true;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Enqueue one layer in groups of batch columns.
+// Persistent kernel for up to kStreamMaxBatch columns; PP_ERR_UNSUPPORTED when x does not fit shared memory.
+pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_len, int x_elt, void* y, int ldy,
+                       int out_mode, int batch, pp_act_t act, cudaStream_t stream, int x_limit) {
+    const pp_packed* pk = L->pk;
+    int stage_mode = -1;
+    const bool rows_aligned = aligned16(x) && (batch == 1 || ((size_t)ldx * x_elt) % 16 == 0);
+    const int fast = gather ? (batch == 1 && pp::g_stage_direct ? 3 : 1) : 2;
+    if (rows_aligned && pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, fast) <= pp::kStreamSmemLimit)
+        stage_mode = fast;
+    else if (pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, 0) <= pp::kStreamSmemLimit)
+        stage_mode = 0;
+    if (stage_mode < 0) return PP_ERR_UNSUPPORTED;
+    pp::StreamArgs s{};
+    s.stage_mode = stage_mode;
+    s.values = L->d_values; s.xoff = L->d_xoff; s.strip_start = L->d_strip_start;
+    s.cta_desc = L->d_cta_desc; s.strip_info = L->d_strip_info;
+    s.gather_idx = gather; s.scatter_idx = L->d_scatter; s.bias_piv = L->d_bias;
+    s.x = x; s.y = y; s.partials = L->d_spartials; s.counters = L->d_scounters;
+    s.ldx = ldx; s.ldy = ldy; s.x_limit = x_limit; s.n_pad = pk->Npad; s.x_len = x_len; s.max_rows = L->stream_max_rows; s.batch = batch;
+    s.act = (int)act; s.out_mode = out_mode;
+    return pp::launch_stream(pk->wdtype, pk->B, s, pk->cta_desc.data(), L->stream_grid, stream) == cudaSuccess
+               ? PP_OK : PP_ERR_CUDA;
+}
+
+// Enqueue one layer.  Batch <= 8: one launch of the persistent kernel.  Larger batches: the
+// persistent kernel in groups of 8 columns while that re-reads the weights at most three times
+// (it streams them about three times faster than the chunked kernel), else the chunked kernel
+// in groups of up to 32 (fp16) or 8 (fp32) columns.
 pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_len, int x_elt, void* y, int ldy,
                       int out_mode, int batch, pp_act_t act, cudaStream_t stream, int x_limit = -1) {
     const pp_packed* pk = L->pk;
     if (x_limit < 0) x_limit = pk->N;      // without a gather map: columns at or beyond x_limit read 0
-    int stage_mode = -1;
-    if (pp::g_use_stream && batch <= pp::kStreamMaxBatch) {
-        const bool rows_aligned = aligned16(x) && (batch == 1 || ((size_t)ldx * x_elt) % 16 == 0);
-        const int fast = gather ? (batch == 1 && pp::g_stage_direct ? 3 : 1) : 2;
-        if (rows_aligned && pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, fast) <= pp::kStreamSmemLimit)
-            stage_mode = fast;
-        else if (pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, 0) <= pp::kStreamSmemLimit)
-            stage_mode = 0;
-    }
-    if (stage_mode >= 0) {
-        pp::StreamArgs s{};
-        s.stage_mode = stage_mode;
-        s.values = L->d_values; s.xoff = L->d_xoff; s.strip_start = L->d_strip_start;
-        s.cta_desc = L->d_cta_desc; s.strip_info = L->d_strip_info;
-        s.gather_idx = gather; s.scatter_idx = L->d_scatter; s.bias_piv = L->d_bias;
-        s.x = x; s.y = y; s.partials = L->d_spartials; s.counters = L->d_scounters;
-        s.ldx = ldx; s.ldy = ldy; s.x_limit = x_limit; s.n_pad = pk->Npad; s.x_len = x_len; s.max_rows = L->stream_max_rows; s.batch = batch;
-        s.act = (int)act; s.out_mode = out_mode;
-        return pp::launch_stream(pk->wdtype, pk->B, s, pk->cta_desc.data(), L->stream_grid, stream) == cudaSuccess
-                   ? PP_OK : PP_ERR_CUDA;
+    const int y_elt = out_mode == pp::OUT_PIVOTED_F16 ? 2 : 4;
+    const int chunk_group = pp::gemv_group_batch(pk->wdtype);
+    const int stream_passes = (batch + pp::kStreamMaxBatch - 1) / pp::kStreamMaxBatch;
+    const int chunk_passes = (batch + chunk_group - 1) / chunk_group;
+    if (pp::g_use_stream && stream_passes <= 3 * chunk_passes) {
+        bool done = true;
+        for (int b0 = 0; b0 < batch; b0 += pp::kStreamMaxBatch) {
+            const int nb = batch - b0 < pp::kStreamMaxBatch ? batch - b0 : pp::kStreamMaxBatch;
+            const pp_status_t st = run_stream(L, gather, static_cast<const char*>(x) + (size_t)b0 * ldx * x_elt, ldx, x_len,
+                                              x_elt, static_cast<char*>(y) + (size_t)b0 * ldy * y_elt, ldy, out_mode, nb, act,
+                                              stream, x_limit);
+            if (st == PP_ERR_UNSUPPORTED && b0 == 0) { done = false; break; }   // x too large to stage: chunked kernel
+            if (st != PP_OK) return st;
+        }
+        if (done) return PP_OK;
     }
     pp::GemvArgs a{};
     a.values = L->d_values; a.items = L->d_items; a.tile_col = L->d_tile_col;
     a.gather_idx = gather; a.scatter_idx = L->d_scatter; a.bias_piv = L->d_bias;
     a.partials = L->d_partials; a.counters = L->d_counters;
     a.ldx = ldx; a.ldy = ldy; a.x_limit = x_limit; a.act = (int)act; a.out_mode = out_mode;
-    const int group = pp::gemv_group_batch(pk->wdtype);
-    const int y_elt = out_mode == pp::OUT_PIVOTED_F16 ? 2 : 4;
+    const int group = chunk_group;
     for (int b0 = 0; b0 < batch; b0 += group) {
         a.batch = batch - b0 < group ? batch - b0 : group;
         a.x = static_cast<const char*>(x) + (size_t)b0 * ldx * x_elt;
@@ -320,17 +341,18 @@ pp_status_t pp_forward(pp_layer_t* L, const void* x, void* y, int batch, pp_act_
     if (!aligned16(x) || !aligned16(y)) return PP_ERR_INVALID_ARG;
     const pp_packed* pk = L->pk;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (L->tile_plan && pp::g_tile_min_batch > 0 && batch >= pp::g_tile_min_batch && (size_t)pk->N * 2 <= 48 * 1024) {
+    if (L->tile_ok && pp::g_tile_min_batch > 0 && batch >= pp::g_tile_min_batch && (size_t)pk->N * 2 <= 48 * 1024) {
         // tensor-core tile path, 128 batch rows at a time
         pp::TileArgs t{};
         t.row_ptr = L->d_row_ptr; t.col_ptr = L->d_col_ptr; t.tile_col = L->d_tile_col;
         t.scatter_idx = L->d_scatter; t.bias_piv = L->d_bias; t.status = L->d_status;
+        t.tiles_sw = static_cast<const unsigned char*>(L->d_tiles_rm); t.x_sw = static_cast<const unsigned char*>(L->d_x_piv);
         t.ldy = pk->M; t.act = (int)act;
         for (int b0 = 0; b0 < batch; b0 += pp::kTileBatch) {
             t.batch = batch - b0 < pp::kTileBatch ? batch - b0 : pp::kTileBatch;
             t.y = static_cast<float*>(y) + (size_t)b0 * pk->M;
             const char* xc = static_cast<const char*>(x) + (size_t)b0 * pk->N * 2;
-            if (pp::launch_tile(L->tile_plan, t, xc, pk->N, pk->N, L->d_gather, pk->Npad, L->d_x_piv, pk->Mb, stream) != cudaSuccess)
+            if (pp::launch_tile(t, xc, pk->N, pk->N, L->d_gather, pk->Npad, pk->Mb, stream) != cudaSuccess)
                 return PP_ERR_CUDA;
         }
         return PP_OK;

@@ -75,7 +75,7 @@ struct pp_packed {
     std::vector<int32_t> gather_idx, scatter_idx;
     std::vector<float> bias_piv;
     std::vector<unsigned char> values;                       // fragment-ordered tile values
-    std::vector<unsigned char> tiles_rm;                     // fp16, B = 64 only: sorted tiles, row-major (tensor-core path)
+    std::vector<unsigned char> tiles_rm;                     // fp16, B = 64 only: sorted tiles as swizzled 8 KiB images (tensor-core path)
     std::vector<pp::WorkItem> items;
     // plan of the persistent streaming kernel
     std::vector<int32_t> strip_start;   // [S+1] fragment position of each strip

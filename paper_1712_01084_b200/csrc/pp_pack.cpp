@@ -7,6 +7,7 @@
 #include <numeric>
 
 #include "pp_internal.h"
+#include "pp_tile.cuh"
 
 namespace pp {
 int g_use_stream = 1;      // 0: the API never picks the persistent kernel
@@ -326,10 +327,10 @@ pp_status_t pp_pack_create(pp_packed_t** out, int M, int N, int B, const int32_t
             }
         }
 
-        if (wdtype == PP_F16 && B == 64) {       // row-major copy of the sorted tiles for the tensor-core path
-            p->tiles_rm.resize((size_t)T * B * B * 2);
+        if (wdtype == PP_F16 && B == 64) {       // second copy of the sorted tiles for the tensor-core path:
+            p->tiles_rm.resize((size_t)T * B * B * 2);   // each tile as its swizzled shared-memory image
             for (int64_t s2 = 0; s2 < T; ++s2)
-                std::memcpy(&p->tiles_rm[(size_t)s2 * B * B * 2], src + (size_t)order[(size_t)s2] * B * B * 2, (size_t)B * B * 2);
+                pp::swizzle_tile_64x64(src + (size_t)order[(size_t)s2] * B * B * 2, &p->tiles_rm[(size_t)s2 * B * B * 2]);
         }
 
         p->gather_idx.resize((size_t)Npad);

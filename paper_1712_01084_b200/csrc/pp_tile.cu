@@ -5,19 +5,20 @@
 // block-row's kept tiles: the batch chunk (128 rows of the permuted input) is the M side, the
 // tile's 64 output rows the N side, the tile's 64 columns the K side (4 instructions of K = 16).
 //   * Listing 1's group fetch is a pre-pass (gather_x_kernel): x_piv[b][j] = x[b][gather_idx[j]],
-//     one CTA per batch row, through shared memory so that both sides are coalesced;
-//   * warp 0 streams (X segment, W tile) pairs into a ring of shared-memory stages with TMA
-//     (cp.async.bulk.tensor, 128-byte swizzle, no multicast), signalling mbarriers;
+//     one CTA per batch row through shared memory, written as one 16 KiB block per tile-column that
+//     already has the 128-byte-swizzled shared-memory image the tensor core wants; the packer stores
+//     every weight tile as such an image (8 KiB) too;
+//   * warp 0 streams (X block, W tile) pairs into a ring of shared-memory stages with two bulk
+//     asynchronous copies per tile (cp.async.bulk, one request each, no multicast), signalling
+//     mbarriers (2-D tensor-map loads of 128-byte rows were request-rate bound: 60 us vs the
+//     same data as two contiguous copies);
 //   * warp 1 issues tcgen05.mma (kind::f16, accumulator in tensor memory) from shared-memory matrix
 //     descriptors and frees each stage with tcgen05.commit;
 //   * warps 2..5 read the accumulator with tcgen05.ld and run the fused epilogue: bias, activation,
 //     store through the row index array (Listing 1's last step).
 // Every wait on an mbarrier is bounded; on a time-out the kernel raises the layer's status word,
 // stops issuing work, lets its outstanding copies land, frees its tensor memory and returns.
-#include <cuda.h>
 #include <cuda_fp16.h>
-
-#include <new>
 
 #include "pp_gemv.cuh"
 #include "pp_tile.cuh"
@@ -60,9 +61,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile
     return false;
 }
 
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 :: "r"(smem_u32(dst)), "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar)) : "memory");
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes, 8-row groups
@@ -100,7 +101,7 @@ struct TileSmem {
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
-tile_f16_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, const TileArgs a) {
+tile_f16_kernel(const TileArgs a) {
     extern __shared__ unsigned char smem_raw[];
     // stage buffers need 1024-byte alignment for the 128-byte swizzle
     unsigned char* stages = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -130,13 +131,18 @@ tile_f16_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
         // ---------------- TMA producer (one lane)
         if (lane == 0) {
             int issued = 0;
+            const int cbase = __ldg(a.col_ptr + br);
+            const int rot = k > 0 ? (int)(((long long)br * k) / gridDim.x) : 0;
             for (int t = 0; t < k; ++t) {
                 const int s = t % kStages;
                 if (t >= kStages && !mbar_wait(&sm->empty[s], ((t / kStages) & 1) ^ 1, abort_flag)) break;
-                const int col = __ldg(a.tile_col + __ldg(a.col_ptr + br) + t);
+                // block-rows start at different tiles of their lists, so that CTAs running side by side
+                // do not all ask the L2 for the same X segment at the same moment
+                const int tt = (t + rot) % k;
+                const int col = __ldg(a.tile_col + cbase + tt);
                 mbar_expect_tx(&sm->full[s], kStageBytes);
-                tma_load_2d(stages + s * kStageBytes, &map_x, col * 64, 0, &sm->full[s]);
-                tma_load_2d(stages + s * kStageBytes + kXBytes, &map_w, 0, (t0 + t) * 64, &sm->full[s]);
+                bulk_load(stages + s * kStageBytes, a.x_sw + (size_t)col * kXBytes, kXBytes, &sm->full[s]);
+                bulk_load(stages + s * kStageBytes + kXBytes, a.tiles_sw + (size_t)(t0 + tt) * kWBytes, kWBytes, &sm->full[s]);
                 issued = t + 1;
             }
             if (*abort_flag) {
@@ -210,75 +216,41 @@ tile_f16_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
     }
 }
 
+// Byte offset of element (row r, column c) inside a 128-byte-swizzled block of 128-byte rows:
+// the 16-byte chunk index is XOR-ed with the row index modulo 8.
+__host__ __device__ __forceinline__ uint32_t sw128_offset(int r, int c) {
+    return (uint32_t)r * 128u + (uint32_t)(((c >> 3) ^ (r & 7)) << 4) + (uint32_t)(c & 7) * 2u;
+}
+
 // x_piv[b][j] = x[b][gather_idx[j]] for the rows of one batch chunk; rows past the batch and padding
-// columns are zero.  One CTA per row: the row goes to shared memory coalesced and leaves permuted.
+// columns are zero.  One CTA per row: the row goes to shared memory coalesced and leaves permuted, into
+// the swizzled 16 KiB block of its tile-column (row b of the block).
 __global__ void gather_x_kernel(const __half* __restrict__ x, int ldx, int n, const int32_t* __restrict__ gather_idx,
-                                int n_pad, __half* __restrict__ x_piv, int batch) {
+                                int n_pad, unsigned char* __restrict__ x_sw, int batch) {
     extern __shared__ __half row[];
     const int b = blockIdx.x;
-    __half* out = x_piv + (size_t)b * n_pad;
-    if (b >= batch) {
-        for (int j = threadIdx.x; j < n_pad; j += blockDim.x) out[j] = __float2half(0.0f);
-        return;
-    }
-    for (int j = threadIdx.x; j < n; j += blockDim.x) row[j] = x[(size_t)b * ldx + j];
+    if (b < batch)
+        for (int j = threadIdx.x; j < n; j += blockDim.x) row[j] = x[(size_t)b * ldx + j];
     __syncthreads();
     for (int j = threadIdx.x; j < n_pad; j += blockDim.x) {
-        const int idx = __ldg(gather_idx + j);
-        out[j] = idx >= 0 ? row[idx] : __float2half(0.0f);
+        const int idx = b < batch ? __ldg(gather_idx + j) : -1;
+        const __half v = idx >= 0 ? row[idx] : __float2half(0.0f);
+        *reinterpret_cast<__half*>(x_sw + (size_t)(j >> 6) * kXBytes + sw128_offset(b, j & 63)) = v;
     }
-}
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qr;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
-            qr == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
-    return fn;
-}
-
-bool encode_2d(CUtensorMap* map, void* base, uint64_t cols, uint64_t rows, uint32_t box_cols, uint32_t box_rows) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * 2};
-    const cuuint32_t box[2] = {box_cols, box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
-           CUDA_SUCCESS;
 }
 
 }  // namespace
 
-struct TilePlan {
-    CUtensorMap map_x, map_w;
-    bool has_w;
-};
-
-TilePlan* tile_plan_create(void* d_tiles_rm, int64_t T, void* d_x_piv, int n_pad) {
-    TilePlan* p = new (std::nothrow) TilePlan();
-    if (!p) return nullptr;
-    p->has_w = T > 0;
-    bool ok = encode_2d(&p->map_x, d_x_piv, (uint64_t)n_pad, kTileBatch, 64, kTileBatch);
-    if (ok && T > 0) ok = encode_2d(&p->map_w, d_tiles_rm, 64, (uint64_t)T * 64, 64, 64);
-    if (ok && T == 0) p->map_w = p->map_x;      // never dereferenced: no block-row has a tile
-    if (!ok) { delete p; return nullptr; }
-    return p;
+void swizzle_tile_64x64(const void* row_major, void* out) {
+    const unsigned char* src = static_cast<const unsigned char*>(row_major);
+    unsigned char* dst = static_cast<unsigned char*>(out);
+    for (int r = 0; r < 64; ++r)
+        for (int ch = 0; ch < 8; ++ch)
+            for (int k = 0; k < 16; ++k) dst[r * 128 + ((ch ^ (r & 7)) << 4) + k] = src[r * 128 + ch * 16 + k];
 }
 
-void tile_plan_destroy(TilePlan* p) { delete p; }
-
-cudaError_t launch_tile(const TilePlan* plan, const TileArgs& a, const void* x, int ldx, int n, const int32_t* gather_idx,
-                        int n_pad, void* d_x_piv, int Mb, cudaStream_t stream) {
+cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const int32_t* gather_idx, int n_pad, int Mb,
+                        cudaStream_t stream) {
     if (a.batch < 1 || a.batch > kTileBatch) return cudaErrorInvalidValue;
     static bool configured = false;
     const size_t smem = (size_t)kStages * kStageBytes + sizeof(TileSmem) + 1024;
@@ -287,12 +259,12 @@ cudaError_t launch_tile(const TilePlan* plan, const TileArgs& a, const void* x, 
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    if ((size_t)n * 2 > 200 * 1024) return cudaErrorInvalidValue;
+    if ((size_t)n * 2 > 48 * 1024) return cudaErrorInvalidValue;
     gather_x_kernel<<<kTileBatch, 256, (size_t)n * 2, stream>>>(static_cast<const __half*>(x), ldx, n, gather_idx, n_pad,
-                                                              static_cast<__half*>(d_x_piv), a.batch);
+                                                              const_cast<unsigned char*>(a.x_sw), a.batch);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    tile_f16_kernel<<<Mb, kThreads, smem, stream>>>(plan->map_x, plan->map_w, a);
+    tile_f16_kernel<<<Mb, kThreads, smem, stream>>>(a);
     return cudaGetLastError();
 }
 

@@ -14,6 +14,8 @@ struct TileArgs {
     const int32_t* tile_col;     // tile-column index of every kept tile
     const int32_t* scatter_idx;  // pivoted row -> original row, -1 = padding
     const float* bias_piv;
+    const unsigned char* tiles_sw;   // sorted kept tiles, each an 8 KiB swizzled shared-memory image
+    const unsigned char* x_sw;       // [N_pad / 64] blocks of 16 KiB: 128 batch rows x 64 columns, swizzled (scratch)
     float* y;                    // [batch][ldy], first row of this chunk
     int* status;                 // raised to 1 when a bounded wait gave up
     int ldy;
@@ -21,15 +23,11 @@ struct TileArgs {
     int act;
 };
 
-struct TilePlan;                 // tensor maps of one layer (host object)
+// Host: the shared-memory image (128-byte swizzle) of one 64 x 64 row-major fp16 tile, 8 KiB.
+void swizzle_tile_64x64(const void* row_major, void* out);
 
-// d_tiles_rm: sorted kept tiles, each 64 x 64 row-major fp16; d_x_piv: [kTileBatch][n_pad] fp16 scratch.
-// Returns NULL when the driver's tensor-map encoder is unavailable or refuses the shapes.
-TilePlan* tile_plan_create(void* d_tiles_rm, int64_t T, void* d_x_piv, int n_pad);
-void tile_plan_destroy(TilePlan* p);
-
-// Enqueue the gather pre-pass and the tile kernel for one batch chunk.
-cudaError_t launch_tile(const TilePlan* plan, const TileArgs& a, const void* x, int ldx, int n, const int32_t* gather_idx,
-                        int n_pad, void* d_x_piv, int Mb, cudaStream_t stream);
+// Enqueue the gather pre-pass (x -> a.x_sw) and the tile kernel for one batch chunk.
+cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const int32_t* gather_idx, int n_pad, int Mb,
+                        cudaStream_t stream);
 
 }  // namespace pp

@@ -71,9 +71,7 @@ def _run_and_check(pb, lay, x, act, what=""):
 @pytest.mark.parametrize("persistent", [1, 0])
 def test_small_layers(pb, dtype, B, batch, persistent):
     """Ragged M and N, unbalanced block-rows, one block-row without tiles, several tiles and a ragged tail;
-    through the persistent kernel (batch <= 8) and through the chunked kernel."""
-    if persistent and batch > 8:
-        pytest.skip("batch > 8 always takes the chunked kernel")
+    through the persistent kernel (in groups of 8 columns) and through the chunked kernel."""
     pb.pp_set_tuning(5, persistent)
     try:
         lay = _rand_layer(100 + B + batch, 5 * B - 3, 9 * B - 7, B, dtype, density=0.45, empty_rows=(2,))
