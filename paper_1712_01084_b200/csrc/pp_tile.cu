@@ -26,7 +26,8 @@
 namespace pp {
 namespace {
 
-constexpr int kStages = 6;
+constexpr int kStages = 8;
+constexpr int kProducers = 4;      // lanes of warp 0 that issue bulk copies (kStages is a multiple of it)
 constexpr int kXBytes = kTileBatch * 64 * 2;     // 128 x 64 fp16 = 16 KiB
 constexpr int kWBytes = 64 * 64 * 2;             // 64 x 64 fp16 = 8 KiB
 constexpr int kStageBytes = kXBytes + kWBytes;
@@ -128,12 +129,13 @@ tile_f16_kernel(const TileArgs a) {
     volatile int* abort_flag = &sm->abort_flag;
 
     if (warp == 0) {
-        // ---------------- TMA producer (one lane)
-        if (lane == 0) {
-            int issued = 0;
+        // ---------------- producers: kProducers lanes, lane p feeds tiles p, p + kProducers, ...
+        // (one thread issues a bulk copy every ~0.15 us at best, which alone would cap the CTA)
+        if (lane < kProducers) {
+            int last = -1;
             const int cbase = __ldg(a.col_ptr + br);
             const int rot = k > 0 ? (int)(((long long)br * k) / gridDim.x) : 0;
-            for (int t = 0; t < k; ++t) {
+            for (int t = lane; t < k; t += kProducers) {
                 const int s = t % kStages;
                 if (t >= kStages && !mbar_wait(&sm->empty[s], ((t / kStages) & 1) ^ 1, abort_flag)) break;
                 // block-rows start at different tiles of their lists, so that CTAs running side by side
@@ -143,11 +145,11 @@ tile_f16_kernel(const TileArgs a) {
                 mbar_expect_tx(&sm->full[s], kStageBytes);
                 bulk_load(stages + s * kStageBytes, a.x_sw + (size_t)col * kXBytes, kXBytes, &sm->full[s]);
                 bulk_load(stages + s * kStageBytes + kXBytes, a.tiles_sw + (size_t)(t0 + tt) * kWBytes, kWBytes, &sm->full[s]);
-                issued = t + 1;
+                last = t;
             }
             if (*abort_flag) {
-                // let the copies still in flight land before shared memory goes away
-                for (int t = issued > kStages ? issued - kStages : 0; t < issued; ++t)
+                // let this lane's copies still in flight land before shared memory goes away
+                for (int t = last; t >= 0 && t > last - kStages; t -= kProducers)
                     for (int i = 0; i < kPollLimit && !mbar_try_wait(&sm->full[t % kStages], (t / kStages) & 1); ++i) {}
             }
         }
@@ -229,13 +231,32 @@ __global__ void gather_x_kernel(const __half* __restrict__ x, int ldx, int n, co
                                 int n_pad, unsigned char* __restrict__ x_sw, int batch) {
     extern __shared__ __half row[];
     const int b = blockIdx.x;
-    if (b < batch)
-        for (int j = threadIdx.x; j < n; j += blockDim.x) row[j] = x[(size_t)b * ldx + j];
+    if (b < batch) {
+        // 16-byte copies where the row allows it (base and pitch 16-byte aligned), element copies otherwise
+        const __half* src = x + (size_t)b * ldx;
+        const bool vec = ((reinterpret_cast<uintptr_t>(src) & 15u) == 0);
+        const int n8 = vec ? n / 8 : 0;
+        for (int i = threadIdx.x; i < n8; i += blockDim.x)
+            reinterpret_cast<uint4*>(row)[i] = __ldg(reinterpret_cast<const uint4*>(src) + i);
+        for (int j = n8 * 8 + threadIdx.x; j < n; j += blockDim.x) row[j] = src[j];
+    }
     __syncthreads();
-    for (int j = threadIdx.x; j < n_pad; j += blockDim.x) {
-        const int idx = b < batch ? __ldg(gather_idx + j) : -1;
-        const __half v = idx >= 0 ? row[idx] : __float2half(0.0f);
-        *reinterpret_cast<__half*>(x_sw + (size_t)(j >> 6) * kXBytes + sw128_offset(b, j & 63)) = v;
+    // 8 independent index loads per thread before the first use, so their latencies overlap
+    for (int j0 = threadIdx.x; j0 < n_pad; j0 += 8 * blockDim.x) {
+        int idx[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int j = j0 + q * blockDim.x;
+            idx[q] = (b < batch && j < n_pad) ? __ldg(gather_idx + j) : -1;
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const int j = j0 + q * blockDim.x;
+            if (j < n_pad) {
+                const __half v = idx[q] >= 0 ? row[idx[q]] : __float2half(0.0f);
+                *reinterpret_cast<__half*>(x_sw + (size_t)(j >> 6) * kXBytes + sw128_offset(b, j & 63)) = v;
+            }
+        }
     }
 }
 
@@ -260,7 +281,7 @@ cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const 
         configured = true;
     }
     if ((size_t)n * 2 > 48 * 1024) return cudaErrorInvalidValue;
-    gather_x_kernel<<<kTileBatch, 256, (size_t)n * 2, stream>>>(static_cast<const __half*>(x), ldx, n, gather_idx, n_pad,
+    gather_x_kernel<<<kTileBatch, 1024, ((size_t)n * 2 + 15) / 16 * 16, stream>>>(static_cast<const __half*>(x), ldx, n, gather_idx, n_pad,
                                                               const_cast<unsigned char*>(a.x_sw), a.batch);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
