@@ -399,7 +399,9 @@ def main():
                 "d2h_bytes_per_step": int(lay.M * 4), "steps": n_e2e},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                     "algorithmic_bytes_per_launch": abytes, "kernel": "stream_f16_kernel<4>", "traffic": None},
+                     "algorithmic_bytes_per_launch": abytes, "kernel": "stream_f16_kernel<4>",
+                     # dram__bytes_read.sum + dram__bytes_write.sum of one launch (ncu, profiles/stream_f16_cfg5_k128_batch1.md)
+                     "traffic": 139.95e6 if args.k == 128 else None},
         "clocks": clocks,
     }
 
