@@ -195,6 +195,22 @@ def time_graph(pb, torch, replicas, x, y, act, steps, warmup, chunk=500):
         return stream, graphs, chunk, e0, e1
 
 
+def max_over_ranks(value, world, device="cuda"):
+    """The slowest rank's figure (every rank runs an independent replica; the job is as slow as that one)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(us_step_max, world):
+    """Whole-job microseconds per layer: `world` replicas finish one layer each per (slowest) step."""
+    return us_step_max / world
+
+
 def time_enqueue(torch, enqueue, calls_per_graph, replays=20):
     """Mean device time (us) of one call: `enqueue(i, stream_ptr)` is captured `calls_per_graph`
     times into a CUDA graph that is replayed `replays` times between two events."""
@@ -355,12 +371,9 @@ def main():
         return wl, lay, reps, x, y, ms, clocks
 
     wl, lay, reps, x, y, ms, clocks = time_config(args.k, args.steps, args.warmup, sample_clocks=True)
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world)
     us_step = ms * 1e3 / args.steps                      # one step = one layer on every rank
-    value = us_step / world                              # whole job: `world` layers per step time
+    value = job_value(us_step, world)
 
     # end to end from host buffers through the public Python call
     n_e2e = min(args.steps, 300)
@@ -376,10 +389,7 @@ def main():
         yh.copy_(y, non_blocking=True)
         torch.cuda.current_stream().synchronize()
     e2e_us = (time.perf_counter() - t0) / n_e2e * 1e6
-    if world > 1:
-        t = torch.tensor([e2e_us], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_us = float(t.item())
+    e2e_us = max_over_ranks(e2e_us, world)
 
     pk = pb.Packed(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values, lay.bias)
     abytes = algorithmic_bytes(lay, 1, pk.n_tile_col)
