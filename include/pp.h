@@ -154,10 +154,12 @@ pp_status_t pp_forward(pp_layer_t* layer, const void* x, void* y, int batch,
                        pp_act_t act, void* cuda_stream);
 
 /* ------------------------------------------------------------------------- *
- * Chain of layers with folded permutations (Section 4.2.1): between two
- * consecutive layers the activations stay in the producer's pivoted order and
- * the consumer gathers through the folded map q (pp_fold_perm); only the first
- * gather and the last scatter touch original order.  Layer l's output feeds
+ * Chain of layers with folded permutations (Section 4.2.1): the row permutation
+ * of a layer and the column permutation of the next one are folded into one
+ * static map (pp_fold_perm), which the producer applies when it stores: its
+ * output lands directly in the consumer's pivoted column order and the consumer
+ * reads it without any index array; only the first gather and the last scatter
+ * touch original order.  Layer l's output feeds
  * layer l+1 rounded (to nearest even) to layer l+1's element type.
  * layers[l+1].N must equal layers[l].M.  The chain references its layers: they
  * must outlive it.  Intermediate buffers are sized for max_batch at create.
@@ -235,10 +237,13 @@ pp_status_t pp_forward_noalloc(const pp_packed_t* p, const void* device_image,
  *        over `key 2` CTAs (at least `key 3` fragments each) whose boundaries move onto a strip boundary when
  *        closer to it than this percentage of a CTA's share
  * key 5: 0 = never use the persistent kernel, 1 = use it when batch <= 8 and x fits shared memory (default 1)
- * key 6: asynchronous 512-byte weight copies each warp of the persistent kernel keeps in flight: 4 (default) or 8
+ * key 6: asynchronous 512-byte weight copies each warp of the persistent kernel keeps in flight: 4, 6 or 8;
+ *        0 (default) = 4 when two CTAs fit an SM, else the deepest ring that fits
  * key 7: batch 1 in the persistent kernel: 1 (default) reads x through the index array inside the multiply
  *        loop, 0 permutes x into pivoted order in shared memory first (what batch 2..8 always do)
  * key 8: 1 (default) launches the persistent kernel with programmatic stream serialization, 0 plainly
+ * key 10: 1 (default) permutes multi-column inputs in a pre-pass kernel when the layer kernel cannot hold x
+ *         twice in shared memory; 0 leaves the gather to the layer kernel; 2 always uses the pre-pass
  * key 9: smallest batch for which fp16 layers with B = 64 take the tensor-core tile path (default 64; 0 = never) */
 pp_status_t pp_set_tuning(int key, int value);
 

@@ -35,6 +35,7 @@ struct pp_layer {
     int* d_counters = nullptr;     // chunked kernel: [Mb]
     float* d_spartials = nullptr;  // persistent kernel: [stream_slots][rows per strip][kStreamMaxBatch]
     int* d_scounters = nullptr;    // persistent kernel: [S]
+    unsigned char* d_xstage = nullptr;   // [kMaxGroupBatch][N_pad] input in pivoted order (pre-pass output)
     int n_items = 0;
     int max_item_tiles = 0;
     int stream_grid = 0;
@@ -64,8 +65,9 @@ struct pp_lstm {
 struct pp_chain {
     std::vector<pp_layer*> layers;
     std::vector<pp_act_t> acts;
-    std::vector<int32_t*> d_q;     // folded gather map of layer l (l >= 1); entry 0 unused
-    std::vector<void*> d_inter;    // output of layer l in pivoted order, element type of layer l+1
+    std::vector<int32_t*> d_q;     // entry l (l >= 1): folded map of the link l-1 -> l, as a STORE map of layer l-1:
+                                   // pivoted row of layer l-1 -> pivoted column of layer l (-1: padding row)
+    std::vector<void*> d_inter;    // output of layer l in layer l+1's pivoted column order, element type of layer l+1
     int max_batch = 0;
 };
 
@@ -95,7 +97,7 @@ size_t round256(size_t n) { return (n + 255) / 256 * 256; }
 struct LayerLayout {
     size_t off[10];       // cta_desc, strip_start, strip_info, scatter, bias, gather, tile_col, items, xoff, values
     size_t arena_bytes;
-    size_t soff[4];       // partials, counters, spartials, scounters
+    size_t soff[5];       // partials, counters, spartials, scounters, pivoted-x staging
     size_t scratch_bytes;
 };
 
@@ -111,10 +113,11 @@ LayerLayout layer_layout(const pp_packed* pk) {
     size_t pos = 0;
     for (int i = 0; i < 10; ++i) { lo.off[i] = pos; pos += round256(sz[i]); }
     lo.arena_bytes = pos ? pos : 256;
-    const size_t ssz[4] = {(size_t)pk->n_slots * pk->B * pp::kMaxGroupBatch * 4, (size_t)pk->Mb * 4,
-                           (size_t)pk->stream_slots * g.rg_rows * pp::kStreamMaxBatch * 4, (S ? S : 1) * 4};
+    const size_t ssz[5] = {(size_t)pk->n_slots * pk->B * pp::kMaxGroupBatch * 4, (size_t)pk->Mb * 4,
+                           (size_t)pk->stream_slots * g.rg_rows * pp::kStreamMaxBatch * 4, (S ? S : 1) * 4,
+                           (size_t)pp::kMaxGroupBatch * pk->Npad * esz};
     pos = 0;
-    for (int i = 0; i < 4; ++i) { lo.soff[i] = pos; pos += round256(ssz[i]); }
+    for (int i = 0; i < 5; ++i) { lo.soff[i] = pos; pos += round256(ssz[i]); }
     lo.scratch_bytes = pos;
     return lo;
 }
@@ -144,6 +147,7 @@ bool alloc_layer(pp_layer* L, const LayerLayout& lo) {
     L->d_counters = reinterpret_cast<int*>(sc + lo.soff[1]);
     L->d_spartials = reinterpret_cast<float*>(sc + lo.soff[2]);
     L->d_scounters = reinterpret_cast<int*>(sc + lo.soff[3]);
+    L->d_xstage = sc + lo.soff[4];
     return true;
 }
 
@@ -181,7 +185,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 // Enqueue one layer in groups of batch columns.
 // Persistent kernel for up to kStreamMaxBatch columns; PP_ERR_UNSUPPORTED when x does not fit shared memory.
 pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_len, int x_elt, void* y, int ldy,
-                       int out_mode, int batch, pp_act_t act, cudaStream_t stream, int x_limit) {
+                       int out_mode, int batch, pp_act_t act, cudaStream_t stream, int x_limit, const int32_t* scatter) {
     const pp_packed* pk = L->pk;
     int stage_mode = -1;
     const bool rows_aligned = aligned16(x) && (batch == 1 || ((size_t)ldx * x_elt) % 16 == 0);
@@ -195,7 +199,7 @@ pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ld
     s.stage_mode = stage_mode;
     s.values = L->d_values; s.xoff = L->d_xoff; s.strip_start = L->d_strip_start;
     s.cta_desc = L->d_cta_desc; s.strip_info = L->d_strip_info;
-    s.gather_idx = gather; s.scatter_idx = L->d_scatter; s.bias_piv = L->d_bias;
+    s.gather_idx = gather; s.scatter_idx = scatter; s.bias_piv = L->d_bias;
     s.x = x; s.y = y; s.partials = L->d_spartials; s.counters = L->d_scounters;
     s.ldx = ldx; s.ldy = ldy; s.x_limit = x_limit; s.n_pad = pk->Npad; s.x_len = x_len; s.max_rows = L->stream_max_rows; s.batch = batch;
     s.act = (int)act; s.out_mode = out_mode;
@@ -209,20 +213,45 @@ pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ld
 // at 8 columns the persistent kernel holds 16 KiB of x per column in shared memory, runs one CTA
 // per SM and measured 60 us per pass against 85 us for one chunked pass over 16 columns).
 pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_len, int x_elt, void* y, int ldy,
-                      int out_mode, int batch, pp_act_t act, cudaStream_t stream, int x_limit = -1) {
+                      int out_mode, int batch, pp_act_t act, cudaStream_t stream, int x_limit = -1,
+                      const int32_t* scatter = nullptr) {
     const pp_packed* pk = L->pk;
     if (x_limit < 0) x_limit = pk->N;      // without a gather map: columns at or beyond x_limit read 0
-    const int y_elt = out_mode == pp::OUT_PIVOTED_F16 ? 2 : 4;
+    if (!scatter) scatter = L->d_scatter;  // a chain passes the map into its consumer's column order instead
+    const int y_elt = (out_mode == pp::OUT_PIVOTED_F16 || out_mode == pp::OUT_SCATTER_F16) ? 2 : 4;
     const int chunk_group = pp::gemv_group_batch(pk->wdtype);
     const int stream_passes = (batch + pp::kStreamMaxBatch - 1) / pp::kStreamMaxBatch;
     const int chunk_passes = (batch + chunk_group - 1) / chunk_group;
+    // Several batch columns with a gather map: unless the persistent kernel can hold x twice (as
+    // given and permuted) in shared memory, permute x once in a pre-pass and let the layer kernel
+    // read the pivoted rows without any index array.
+    if (gather && batch > 1 && pp::g_prepass) {
+        const bool stream_path = pp::g_use_stream && stream_passes <= chunk_passes;
+        const int nb = batch < pp::kStreamMaxBatch ? batch : pp::kStreamMaxBatch;
+        const bool fits = stream_path && aligned16(x) && ((size_t)ldx * x_elt) % 16 == 0 &&
+                          pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, nb, 1) <= 113 * 1024;
+        if (!fits || pp::g_prepass == 2) {
+            const int group = stream_path ? pp::kStreamMaxBatch : chunk_group;
+            for (int b0 = 0; b0 < batch; b0 += group) {
+                const int gb = batch - b0 < group ? batch - b0 : group;
+                if (pp::launch_pivot_x(pk->wdtype, static_cast<const char*>(x) + (size_t)b0 * ldx * x_elt, ldx, x_len, gather,
+                                       pk->Npad, L->d_xstage, gb, stream) != cudaSuccess)
+                    return PP_ERR_CUDA;
+                const pp_status_t st = run_layer(L, nullptr, L->d_xstage, pk->Npad, pk->Npad, x_elt,
+                                                 static_cast<char*>(y) + (size_t)b0 * ldy * y_elt, ldy, out_mode, gb, act,
+                                                 stream, pk->Npad, scatter);
+                if (st != PP_OK) return st;
+            }
+            return PP_OK;
+        }
+    }
     if (pp::g_use_stream && stream_passes <= chunk_passes) {
         bool done = true;
         for (int b0 = 0; b0 < batch; b0 += pp::kStreamMaxBatch) {
             const int nb = batch - b0 < pp::kStreamMaxBatch ? batch - b0 : pp::kStreamMaxBatch;
             const pp_status_t st = run_stream(L, gather, static_cast<const char*>(x) + (size_t)b0 * ldx * x_elt, ldx, x_len,
                                               x_elt, static_cast<char*>(y) + (size_t)b0 * ldy * y_elt, ldy, out_mode, nb, act,
-                                              stream, x_limit);
+                                              stream, x_limit, scatter);
             if (st == PP_ERR_UNSUPPORTED && b0 == 0) { done = false; break; }   // x too large to stage: chunked kernel
             if (st != PP_OK) return st;
         }
@@ -230,7 +259,7 @@ pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx
     }
     pp::GemvArgs a{};
     a.values = L->d_values; a.items = L->d_items; a.tile_col = L->d_tile_col;
-    a.gather_idx = gather; a.scatter_idx = L->d_scatter; a.bias_piv = L->d_bias;
+    a.gather_idx = gather; a.scatter_idx = scatter; a.bias_piv = L->d_bias;
     a.partials = L->d_partials; a.counters = L->d_counters;
     a.ldx = ldx; a.ldy = ldy; a.x_limit = x_limit; a.act = (int)act; a.out_mode = out_mode;
     const int group = chunk_group;
@@ -387,9 +416,17 @@ pp_status_t pp_chain_create(pp_chain_t** out, pp_layer_t* const* layers, const p
         std::vector<int32_t> q((size_t)Bk->Npad);
         st = pp_fold_perm(A->row_perm.data(), A->M, A->Mpad, Bk->col_perm.data(), Bk->N, Bk->Npad, q.data());
         if (st != PP_OK) { ok = false; break; }
-        ok = upload(&C->d_q[(size_t)l], q.data(), q.size() * 4);
+        // q gathers (consumer column j <- producer row q[j]); the chain applies it on the store side:
+        // producer row i -> consumer column j with q[j] == i.  The consumer then reads its input in
+        // its own pivoted order with no index array at all; its padding columns stay zero.
+        std::vector<int32_t> store((size_t)A->Mpad, -1);
+        for (int j = 0; j < Bk->Npad; ++j)
+            if (q[(size_t)j] >= 0) store[(size_t)q[(size_t)j]] = j;
+        ok = upload(&C->d_q[(size_t)l], store.data(), store.size() * 4);
         const size_t elt = Bk->wdtype == PP_F16 ? 2 : 4;
-        ok = ok && cudaMalloc(&C->d_inter[(size_t)l - 1], (size_t)max_batch * A->Mpad * elt) == cudaSuccess;
+        const size_t ibytes = (size_t)max_batch * Bk->Npad * elt;
+        ok = ok && cudaMalloc(&C->d_inter[(size_t)l - 1], ibytes) == cudaSuccess &&
+             cudaMemset(C->d_inter[(size_t)l - 1], 0, ibytes) == cudaSuccess;
         if (!ok) st = PP_ERR_ALLOC;
     }
     if (!ok) {
@@ -419,16 +456,21 @@ pp_status_t pp_chain_forward(pp_chain_t* C, const void* x, void* y, int batch, v
         pp_layer* L = C->layers[(size_t)l];
         const pp_packed* pk = L->pk;
         const int x_elt = pk->wdtype == PP_F16 ? 2 : 4;
-        const int32_t* gather = l == 0 ? L->d_gather : C->d_q[(size_t)l];
-        const int ldx = l == 0 ? pk->N : C->layers[(size_t)l - 1]->pk->Mpad;
-        const int x_len = ldx;      // the folded map names positions of the producer's padded pivoted output
+        // layer 0 gathers through its own column index array; every later layer finds its input
+        // already in its pivoted column order (written there by its producer's epilogue)
+        const int32_t* gather = l == 0 ? L->d_gather : nullptr;
+        const int ldx = l == 0 ? pk->N : pk->Npad;
+        const int x_len = ldx;
+        const int x_limit = l == 0 ? pk->N : pk->Npad;
         pp_status_t st;
         if (l == n - 1) {
-            st = run_layer(L, gather, cur, ldx, x_len, x_elt, y, pk->M, pp::OUT_SCATTER_F32, batch, C->acts[(size_t)l], stream);
+            st = run_layer(L, gather, cur, ldx, x_len, x_elt, y, pk->M, pp::OUT_SCATTER_F32, batch, C->acts[(size_t)l], stream,
+                           x_limit);
         } else {
-            const bool next_f16 = C->layers[(size_t)l + 1]->pk->wdtype == PP_F16;
-            st = run_layer(L, gather, cur, ldx, x_len, x_elt, C->d_inter[(size_t)l], pk->Mpad,
-                           next_f16 ? pp::OUT_PIVOTED_F16 : pp::OUT_PIVOTED_F32, batch, C->acts[(size_t)l], stream);
+            const pp_packed* nx = C->layers[(size_t)l + 1]->pk;
+            st = run_layer(L, gather, cur, ldx, x_len, x_elt, C->d_inter[(size_t)l], nx->Npad,
+                           nx->wdtype == PP_F16 ? pp::OUT_SCATTER_F16 : pp::OUT_SCATTER_F32, batch, C->acts[(size_t)l], stream,
+                           x_limit, C->d_q[(size_t)l + 1]);
             cur = C->d_inter[(size_t)l];
         }
         if (st != PP_OK) return st;

@@ -81,9 +81,12 @@ __device__ __forceinline__ void reduce_and_store(const GemvArgs& a, const WorkIt
         const int i = it.br * B + r;
         v += __ldg(a.bias_piv + i);
         if (a.act == PP_ACT_RELU) v = fmaxf(v, 0.0f);
-        if (a.out_mode == OUT_SCATTER_F32) {
+        if (a.out_mode == OUT_SCATTER_F32 || a.out_mode == OUT_SCATTER_F16) {
             const int dst = __ldg(a.scatter_idx + i);
-            if (dst >= 0) static_cast<float*>(a.y)[(size_t)b * a.ldy + dst] = v;
+            if (dst >= 0) {
+                if (a.out_mode == OUT_SCATTER_F32) static_cast<float*>(a.y)[(size_t)b * a.ldy + dst] = v;
+                else static_cast<__half*>(a.y)[(size_t)b * a.ldy + dst] = __float2half_rn(v);
+            }
         } else if (a.out_mode == OUT_PIVOTED_F32) {
             static_cast<float*>(a.y)[(size_t)b * a.ldy + i] = v;
         } else {

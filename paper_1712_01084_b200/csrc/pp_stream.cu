@@ -242,9 +242,12 @@ __device__ __forceinline__ void finalize(const StreamArgs& a, const CtaDesc& d, 
         const int lr = ls * RG + r;
         v += L.rowbias[lr];
         if (a.act == PP_ACT_RELU) v = fmaxf(v, 0.0f);
-        if (a.out_mode == OUT_SCATTER_F32) {
+        if (a.out_mode == OUT_SCATTER_F32 || a.out_mode == OUT_SCATTER_F16) {
             const int dst = L.rowdst[lr];
-            if (dst >= 0) static_cast<float*>(a.y)[(size_t)b * a.ldy + dst] = v;
+            if (dst >= 0) {
+                if (a.out_mode == OUT_SCATTER_F32) static_cast<float*>(a.y)[(size_t)b * a.ldy + dst] = v;
+                else static_cast<__half*>(a.y)[(size_t)b * a.ldy + dst] = __float2half_rn(v);
+            }
         } else {
             const int i = d.s_first * RG + lr;
             if (a.out_mode == OUT_PIVOTED_F32) static_cast<float*>(a.y)[(size_t)b * a.ldy + i] = v;
@@ -567,19 +570,41 @@ int xs_stride_for(pp_dtype_t dt, int n_pad) { return dt == PP_F16 ? n_pad + 8 : 
 
 }  // namespace
 
-int g_stream_depth = 4;   // ring slots per warp (4, 6 or 8)
+int g_stream_depth = 0;   // ring slots per warp: 4, 6 or 8; 0 = chosen per launch
 int g_stream_pdl = 1;     // launch with programmatic stream serialization (prologue overlaps the previous kernel)
 
+namespace {
+size_t smem_bytes_at(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int depth);
+}
+
+// Weight copies each warp keeps in flight.  Two CTAs share an SM when a CTA needs at most half of
+// its shared memory: then 4 per warp (64 KiB in flight per SM).  A CTA that has the SM to itself
+// takes the deepest ring that still fits.
+int stream_pick_depth(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode) {
+    if (g_stream_depth) return g_stream_depth;
+    if (smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, 4) <= 113 * 1024) return 4;
+    for (int d : {8, 6})
+        if (smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, d) <= kStreamSmemLimit) return d;
+    return 4;
+}
+
 size_t stream_smem_bytes(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode) {
+    return smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode,
+                         stream_pick_depth(dt, B, n_pad, x_len, max_rows, batch, stage_mode));
+}
+
+namespace {
+size_t smem_bytes_at(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int depth) {
     const int rg = frag_geom(dt, B).rg_rows;
     const int esz = dt == PP_F16 ? 2 : 4;
     size_t bytes = (size_t)kHeaderBytes + (size_t)max_rows * 8 + (size_t)kStreamSegSlots * rg * batch * 4 +
-                   (size_t)kStreamWarps * g_stream_depth * 512;
+                   (size_t)kStreamWarps * depth * 512;
     if (stage_mode != 3) bytes += xs_bytes(batch, xs_stride_for(dt, n_pad), esz);
     if (stage_mode == 1 || stage_mode == 3)
         bytes += (size_t)n_pad * 4 + 16 + (size_t)batch * ((x_len + 15) / 16 * 16) * esz;
     return bytes;
 }
+}  // namespace
 
 cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a_in, const CtaDesc* host_table, int grid,
                           cudaStream_t stream) {
@@ -593,15 +618,21 @@ cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a_in, const Ct
     a.max_rows = (a.max_rows + 3) / 4 * 4;
     if (grid <= kParamCtas)
         for (int c = 0; c < grid; ++c) P.table[c] = host_table[c];
-    const size_t smem = stream_smem_bytes(dt, B, a.n_pad, a.x_len, a.max_rows, a.batch, a.stage_mode);
-    const bool deep = g_stream_depth == 8;
+    const int depth = stream_pick_depth(dt, B, a.n_pad, a.x_len, a.max_rows, a.batch, a.stage_mode);
+    const size_t smem = smem_bytes_at(dt, B, a.n_pad, a.x_len, a.max_rows, a.batch, a.stage_mode, depth);
     if (dt == PP_F16) {
-        if (g_stream_depth == 6) return launch_one<stream_f16_kernel<6>>(P, grid, smem, stream);
-        return deep ? launch_one<stream_f16_kernel<8>>(P, grid, smem, stream)
-                    : launch_one<stream_f16_kernel<4>>(P, grid, smem, stream);
+        if (depth == 8) return launch_one<stream_f16_kernel<8>>(P, grid, smem, stream);
+        if (depth == 6) return launch_one<stream_f16_kernel<6>>(P, grid, smem, stream);
+        return launch_one<stream_f16_kernel<4>>(P, grid, smem, stream);
     }
-    if (B < 32) return deep ? launch_f32<16, 8>(P, grid, smem, stream) : launch_f32<16, 4>(P, grid, smem, stream);
-    return deep ? launch_f32<32, 8>(P, grid, smem, stream) : launch_f32<32, 4>(P, grid, smem, stream);
+    if (B < 32) {
+        if (depth == 8) return launch_f32<16, 8>(P, grid, smem, stream);
+        if (depth == 6) return launch_f32<16, 6>(P, grid, smem, stream);
+        return launch_f32<16, 4>(P, grid, smem, stream);
+    }
+    if (depth == 8) return launch_f32<32, 8>(P, grid, smem, stream);
+    if (depth == 6) return launch_f32<32, 6>(P, grid, smem, stream);
+    return launch_f32<32, 4>(P, grid, smem, stream);
 }
 
 }  // namespace pp

@@ -39,9 +39,9 @@ struct StreamArgs {
 // Shared memory the kernel needs for this (dtype, n_pad, batch); the caller falls back to the
 // chunked kernel when it exceeds kStreamSmemLimit.
 size_t stream_smem_bytes(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode);
-extern int g_stream_depth;   // weight-ring slots per warp: 4, 6 or 8
+extern int g_stream_depth;   // weight-ring slots per warp: 4, 6 or 8; 0 = chosen per launch
 extern int g_stream_pdl;     // 1: launch with programmatic stream serialization
-constexpr size_t kStreamSmemLimit = 200 * 1024;
+constexpr size_t kStreamSmemLimit = 224 * 1024;
 
 // host_table: the plan's CTA ranges in host memory (grid entries); small plans travel to the
 // kernel inside its parameters so that no CTA starts with a dependent global load.

@@ -95,7 +95,7 @@ def test_persistent_kernel_batch1_variants(pb, dtype, B, direct, depth):
         for act in (0, 1):
             _run_and_check(pb, lay, x, act, f"direct={direct} depth={depth} B={B}")
     finally:
-        pb.pp_set_tuning(7, 1); pb.pp_set_tuning(6, 4)
+        pb.pp_set_tuning(7, 1); pb.pp_set_tuning(6, 0)
 
 
 @pytest.mark.parametrize("dtype", [np.float32, np.float16])
@@ -283,6 +283,35 @@ def test_config5_small_batch_sampled_rows(pb, batch):
     y_ref, a = po.dense_forward_rows(W, None, wl.x.astype(np.float64), 0, rows)
     _check(y[:, rows], y_ref, a, np.float16, "config 5 batch 16 sampled")
     L.close()
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float16])
+@pytest.mark.parametrize("prepass", [0, 2])
+def test_input_permutation_prepass(pb, dtype, prepass):
+    """Multi-column inputs permuted by the pre-pass kernel (forced) or inside the layer kernels, for the
+    persistent kernel (batch <= 8), the chunked kernel (batch 20, fp16) and a folded chain."""
+    pb.pp_set_tuning(10, prepass)
+    try:
+        lay = _rand_layer(31, 6 * 32 - 5, 10 * 32 - 3, 32, dtype, density=0.5, empty_rows=(3,))
+        for batch in (2, 8, 20):
+            x = np.random.default_rng(batch).uniform(-1, 1, (batch, lay.N)).astype(dtype)
+            _run_and_check(pb, lay, x, 1, f"prepass={prepass} batch={batch}")
+        dims = [150, 100, 70]
+        lays = []
+        for l in range(2):
+            ll = _rand_layer(400 + l, dims[l + 1], dims[l], 16, dtype, density=0.6, integer=True)
+            ll.tile_values = (np.sign(ll.tile_values) * (np.abs(ll.tile_values) > 3)).astype(dtype)
+            ll.act = 1 if l == 0 else 0
+            lays.append(ll)
+        x = np.random.default_rng(2).integers(-1, 2, (5, dims[0])).astype(dtype)
+        L = [pb.Layer.from_synth(l) for l in lays]
+        chain = pb.Chain(L, [l.act for l in lays], max_batch=8)
+        y = pb.pp_chain_forward(chain, _dev(x)).cpu().numpy()
+        res = po.chain_forward(lays, x.astype(np.float64))
+        assert np.array_equal(y.astype(np.float64), res[-1][1])
+        chain.close()
+    finally:
+        pb.pp_set_tuning(10, 1)
 
 
 # ------------------------------------------------------------------ tensor-core tile path (batch >= 64)
