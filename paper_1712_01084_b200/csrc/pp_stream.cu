@@ -221,6 +221,24 @@ __device__ __forceinline__ void finish_stage(const StreamArgs& a, const SmemLayo
     __syncthreads();
 }
 
+// Which warps will park a partial sum for each of this CTA's strips (their ranges intersect the strip
+// inside the CTA).  Runs right after the staging barrier, off the kernel's tail; the barrier that ends
+// the streaming phase publishes the result.
+__device__ __forceinline__ void plan_parks(const CtaDesc& d, const SmemLayout& L) {
+    for (int ls = threadIdx.x; ls < d.s_count; ls += kThreads) {
+        const int lo = max(L.sstart[ls], d.p_begin), hi = min(L.sstart[ls + 1], d.p_end);
+        int w_lo = 1, w_hi = 0;
+        if (lo < hi) {
+            w_lo = w_hi = 0;
+            for (int w = 1; w < kStreamWarps; ++w) {
+                if (L.wb[w] <= lo) w_lo = w;
+                if (L.wb[w] <= hi - 1) w_hi = w;
+            }
+        }
+        L.wlohi[ls] = w_lo | (w_hi << 8);
+    }
+}
+
 constexpr unsigned kEmptySlot = 0xffffffffu;   // exchange slots rest at this NaN pattern
 
 // Everything after the last barrier of the streaming phase: per-strip sums, cross-CTA reduction,
@@ -254,22 +272,6 @@ __device__ __forceinline__ void finalize(const StreamArgs& a, const CtaDesc& d, 
             else static_cast<__half*>(a.y)[(size_t)b * a.ldy + i] = __float2half_rn(v);
         }
     };
-
-    // which warps parked a partial for each strip (their ranges intersect the strip inside this CTA);
-    // L.wb holds the warps' range starts (written in the prologue)
-    for (int ls = tid; ls < d.s_count; ls += kThreads) {
-        const int lo = max(L.sstart[ls], d.p_begin), hi = min(L.sstart[ls + 1], d.p_end);
-        int w_lo = 1, w_hi = 0;
-        if (lo < hi) {
-            w_lo = w_hi = 0;
-            for (int w = 1; w < kStreamWarps; ++w) {
-                if (L.wb[w] <= lo) w_lo = w;
-                if (L.wb[w] <= hi - 1) w_hi = w;
-            }
-        }
-        L.wlohi[ls] = w_lo | (w_hi << 8);
-    }
-    __syncthreads();
 
     const int n_out = d.s_count * per_strip;
     for (int e = tid; e < n_out; e += kThreads) {
@@ -396,6 +398,7 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
 
     // 3. pivoted x in shared memory
     finish_stage<__half, U>(a, L);
+    plan_parks(d, L);
 
     // 4. stream this warp's share
     float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -472,6 +475,7 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const __grid_co
     asm volatile("griddepcontrol.wait;" ::: "memory");
     issue_x<float>(a, L);
     finish_stage<float, U>(a, L);
+    plan_parks(d, L);
 
     float acc[NB][2];
 #pragma unroll
@@ -577,20 +581,20 @@ namespace {
 size_t smem_bytes_at(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int depth);
 }
 
-// Weight copies each warp keeps in flight.  Two CTAs share an SM when a CTA needs at most half of
-// its shared memory: then 4 per warp (64 KiB in flight per SM).  A CTA that has the SM to itself
-// takes the deepest ring that still fits.
-int stream_pick_depth(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode) {
+// Weight copies each warp keeps in flight.  Two CTAs share an SM when the grid is larger than the SM
+// count and a CTA needs at most half of the SM's shared memory: then 4 per warp (64 KiB in flight per
+// SM).  A CTA that has the SM to itself takes the deepest ring that still fits.
+int stream_pick_depth(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int grid) {
     if (g_stream_depth) return g_stream_depth;
-    if (smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, 4) <= 113 * 1024) return 4;
+    if (grid > 148 && smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, 4) <= 113 * 1024) return 4;
     for (int d : {8, 6})
         if (smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, d) <= kStreamSmemLimit) return d;
     return 4;
 }
 
 size_t stream_smem_bytes(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode) {
-    return smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode,
-                         stream_pick_depth(dt, B, n_pad, x_len, max_rows, batch, stage_mode));
+    // sized for the shallowest ring a launch may pick (a launch with the SM to itself takes a deeper one if it fits)
+    return smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, g_stream_depth ? g_stream_depth : 4);
 }
 
 namespace {
@@ -618,7 +622,7 @@ cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a_in, const Ct
     a.max_rows = (a.max_rows + 3) / 4 * 4;
     if (grid <= kParamCtas)
         for (int c = 0; c < grid; ++c) P.table[c] = host_table[c];
-    const int depth = stream_pick_depth(dt, B, a.n_pad, a.x_len, a.max_rows, a.batch, a.stage_mode);
+    const int depth = stream_pick_depth(dt, B, a.n_pad, a.x_len, a.max_rows, a.batch, a.stage_mode, grid);
     const size_t smem = smem_bytes_at(dt, B, a.n_pad, a.x_len, a.max_rows, a.batch, a.stage_mode, depth);
     if (dt == PP_F16) {
         if (depth == 8) return launch_one<stream_f16_kernel<8>>(P, grid, smem, stream);
