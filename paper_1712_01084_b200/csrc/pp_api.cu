@@ -24,6 +24,7 @@ struct pp_layer {
     pp::WorkItem* d_items = nullptr;
     int32_t* d_tile_col = nullptr;
     int32_t* d_gather = nullptr;
+    uint16_t* d_gather16 = nullptr;  // 16-bit form of d_gather (NULL when N_pad >= 65536)
     int32_t* d_scatter = nullptr;
     float* d_bias = nullptr;
     int32_t* d_xoff = nullptr;
@@ -95,7 +96,7 @@ size_t round256(size_t n) { return (n + 255) / 256 * 256; }
 
 // Section sizes of the arena and the scratch allocation, in a fixed order.
 struct LayerLayout {
-    size_t off[10];       // cta_desc, strip_start, strip_info, scatter, bias, gather, tile_col, items, xoff, values
+    size_t off[11];       // cta_desc, strip_start, strip_info, scatter, bias, gather, tile_col, items, xoff, values, gather16
     size_t arena_bytes;
     size_t soff[5];       // partials, counters, spartials, scounters, pivoted-x staging
     size_t scratch_bytes;
@@ -106,12 +107,13 @@ LayerLayout layer_layout(const pp_packed* pk) {
     const size_t esz = pk->wdtype == PP_F16 ? 2 : 4;
     const size_t S = pk->strip_info.size();
     const size_t F = (size_t)pk->T * g.n_rg * g.fpt;
-    const size_t sz[10] = {pk->cta_desc.size() * sizeof(pp::CtaDesc), (S + 1) * 4, S * sizeof(pp::StripInfo),
+    const size_t sz[11] = {pk->cta_desc.size() * sizeof(pp::CtaDesc), (S + 1) * 4, S * sizeof(pp::StripInfo),
                            (size_t)pk->Mpad * 4, (size_t)pk->Mpad * 4, (size_t)pk->Npad * 4, pk->tile_col.size() * 4,
-                           pk->items.size() * sizeof(pp::WorkItem), F * 4, (size_t)pk->T * pk->B * pk->B * esz};
+                           pk->items.size() * sizeof(pp::WorkItem), F * 4, (size_t)pk->T * pk->B * pk->B * esz,
+                           pk->gather16.size() * 2};
     LayerLayout lo;
     size_t pos = 0;
-    for (int i = 0; i < 10; ++i) { lo.off[i] = pos; pos += round256(sz[i]); }
+    for (int i = 0; i < 11; ++i) { lo.off[i] = pos; pos += round256(sz[i]); }
     lo.arena_bytes = pos ? pos : 256;
     const size_t ssz[5] = {(size_t)pk->n_slots * pk->B * pp::kMaxGroupBatch * 4, (size_t)pk->Mb * 4,
                            (size_t)pk->stream_slots * g.rg_rows * pp::kStreamMaxBatch * 4, (S ? S : 1) * 4,
@@ -124,6 +126,7 @@ LayerLayout layer_layout(const pp_packed* pk) {
 
 // Allocate both device blocks and point the views into them.
 bool alloc_layer(pp_layer* L, const LayerLayout& lo) {
+    const bool pk_has16 = !L->pk->gather16.empty();
     if (cudaMalloc(reinterpret_cast<void**>(&L->d_arena), lo.arena_bytes) != cudaSuccess) return false;
     if (cudaMalloc(reinterpret_cast<void**>(&L->d_scratch), lo.scratch_bytes) != cudaSuccess) return false;
     if (cudaMemset(L->d_scratch, 0, lo.scratch_bytes) != cudaSuccess) return false;
@@ -142,6 +145,7 @@ bool alloc_layer(pp_layer* L, const LayerLayout& lo) {
     L->d_items = reinterpret_cast<pp::WorkItem*>(a + lo.off[7]);
     L->d_xoff = reinterpret_cast<int32_t*>(a + lo.off[8]);
     L->d_values = a + lo.off[9];
+    L->d_gather16 = pk_has16 ? reinterpret_cast<uint16_t*>(a + lo.off[10]) : nullptr;
     unsigned char* sc = L->d_scratch;
     L->d_partials = reinterpret_cast<float*>(sc + lo.soff[0]);
     L->d_counters = reinterpret_cast<int*>(sc + lo.soff[1]);
@@ -189,7 +193,8 @@ pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ld
     const pp_packed* pk = L->pk;
     int stage_mode = -1;
     const bool rows_aligned = aligned16(x) && (batch == 1 || ((size_t)ldx * x_elt) % 16 == 0);
-    const int fast = gather ? (batch == 1 && pp::g_stage_direct ? 3 : 1) : 2;
+    const bool has16 = gather && gather == L->d_gather && L->d_gather16;
+    const int fast = gather ? (batch == 1 && pp::g_stage_direct ? (has16 ? 4 : 3) : 1) : 2;
     if (rows_aligned && pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, fast) <= pp::kStreamSmemLimit)
         stage_mode = fast;
     else if (pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, 0) <= pp::kStreamSmemLimit)
@@ -199,7 +204,7 @@ pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ld
     s.stage_mode = stage_mode;
     s.values = L->d_values; s.xoff = L->d_xoff; s.strip_start = L->d_strip_start;
     s.cta_desc = L->d_cta_desc; s.strip_info = L->d_strip_info;
-    s.gather_idx = gather; s.scatter_idx = scatter; s.bias_piv = L->d_bias;
+    s.gather_idx = gather; s.gather16 = L->d_gather16; s.scatter_idx = scatter; s.bias_piv = L->d_bias;
     s.x = x; s.y = y; s.partials = L->d_spartials; s.counters = L->d_scounters;
     s.ldx = ldx; s.ldy = ldy; s.x_limit = x_limit; s.n_pad = pk->Npad; s.x_len = x_len; s.max_rows = L->stream_max_rows; s.batch = batch;
     s.act = (int)act; s.out_mode = out_mode;
@@ -298,14 +303,15 @@ pp_status_t pp_layer_create(pp_layer_t** out, int M, int N, int B, const int32_t
     const LayerLayout lo = layer_layout(pk);
     bool ok = alloc_layer(L, lo);
     if (ok) {
-        const void* src[10] = {pk->cta_desc.data(), pk->strip_start.data(), pk->strip_info.data(),
+        const void* src[11] = {pk->cta_desc.data(), pk->strip_start.data(), pk->strip_info.data(),
                                pk->scatter_idx.data(), pk->bias_piv.data(), pk->gather_idx.data(),
-                               pk->tile_col.data(), pk->items.data(), pk->xoff.data(), pk->values.data()};
-        const size_t n[10] = {pk->cta_desc.size() * sizeof(pp::CtaDesc), pk->strip_start.size() * 4,
+                               pk->tile_col.data(), pk->items.data(), pk->xoff.data(), pk->values.data(), pk->gather16.data()};
+        const size_t n[11] = {pk->cta_desc.size() * sizeof(pp::CtaDesc), pk->strip_start.size() * 4,
                               pk->strip_info.size() * sizeof(pp::StripInfo), pk->scatter_idx.size() * 4,
                               pk->bias_piv.size() * 4, pk->gather_idx.size() * 4, pk->tile_col.size() * 4,
-                              pk->items.size() * sizeof(pp::WorkItem), pk->xoff.size() * 4, pk->values.size()};
-        for (int i = 0; i < 10 && ok; ++i)
+                              pk->items.size() * sizeof(pp::WorkItem), pk->xoff.size() * 4, pk->values.size(),
+                              pk->gather16.size() * 2};
+        for (int i = 0; i < 11 && ok; ++i)
             ok = n[i] == 0 || cudaMemcpy(L->d_arena + lo.off[i], src[i], n[i], cudaMemcpyHostToDevice) == cudaSuccess;
     }
     ok = ok && tile_setup(L, nullptr);

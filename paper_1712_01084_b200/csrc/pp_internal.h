@@ -74,6 +74,7 @@ struct pp_packed {
     std::vector<int32_t> row_perm, col_perm, inv_row_perm;   // copies of the caller's arrays
     std::vector<int32_t> row_ptr, col_ptr, tile_col;         // block-row-compressed index arrays
     std::vector<int32_t> gather_idx, scatter_idx;
+    std::vector<uint16_t> gather16;                          // gather_idx + 1 as 16-bit entries (when N_pad < 65536)
     std::vector<float> bias_piv;
     std::vector<unsigned char> values;                       // fragment-ordered tile values
     std::vector<unsigned char> tiles_rm;                     // fp16, B = 64 only: sorted tiles as swizzled 8 KiB images (tensor-core path)

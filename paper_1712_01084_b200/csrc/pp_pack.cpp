@@ -337,6 +337,10 @@ pp_status_t pp_pack_create(pp_packed_t** out, int M, int N, int B, const int32_t
 
         p->gather_idx.resize((size_t)Npad);
         for (int64_t j = 0; j < Npad; ++j) p->gather_idx[(size_t)j] = col_perm[j] < N ? col_perm[j] : -1;
+        if (Npad < 65536) {
+            p->gather16.resize((size_t)Npad);
+            for (int64_t j = 0; j < Npad; ++j) p->gather16[(size_t)j] = (uint16_t)(p->gather_idx[(size_t)j] + 1);
+        }
         p->scatter_idx.resize((size_t)Mpad);
         p->bias_piv.assign((size_t)Mpad, 0.0f);
         for (int64_t i = 0; i < Mpad; ++i) {

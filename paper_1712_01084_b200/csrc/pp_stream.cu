@@ -111,9 +111,9 @@ __device__ __forceinline__ SmemLayout carve(unsigned char* base, int rg, int U, 
     L.ring = reinterpret_cast<uint4*>(L.segp + kStreamSegSlots * rg * a.batch);
     unsigned char* p = reinterpret_cast<unsigned char*>(L.ring + kStreamWarps * U * 32);
     L.xs = p;
-    if (a.stage_mode != 3) p += xs_bytes(a.batch, a.xs_stride, esz);
+    if (a.stage_mode < 3) p += xs_bytes(a.batch, a.xs_stride, esz);
     L.idxs = reinterpret_cast<int*>(p);
-    L.raw = p + (size_t)a.n_pad * 4 + 16;     // 16 spare bytes in front: raw[-1] is the zero that index -1 reads
+    L.raw = p + (size_t)a.n_pad * (a.stage_mode == 4 ? 2 : 4) + 16;     // 16 spare bytes in front: raw[-1] is the zero that index -1 reads
     return L;
 }
 
@@ -142,7 +142,20 @@ __device__ __forceinline__ void issue_static(const StreamArgs& a, const CtaDesc&
     }
     if (a.stage_mode == 1 || a.stage_mode == 3)
         for (int i = tid; i < a.n_pad / 4; i += kThreads) cp_async_16(L.idxs + 4 * i, a.gather_idx + 4 * i);
+    if (a.stage_mode == 4)      // 16-bit table: entry = index + 1, 0 = the zero in front of the copied x
+        for (int i = tid; i < a.n_pad / 8; i += kThreads)
+            cp_async_16(reinterpret_cast<uint16_t*>(L.idxs) + 8 * i, a.gather16 + 8 * i);
     asm volatile("cp.async.commit_group;" ::: "memory");
+}
+
+// Before griddepcontrol.wait: touch the pages of x and y with L2 prefetches so that their address
+// translations are already cached when the copy of x and the stores to y are issued.  (A prefetch
+// reads no value into the SM; the data itself is read and written only after the wait.)
+__device__ __forceinline__ void warm_translations(const StreamArgs& a) {
+    if (threadIdx.x == 0) {
+        asm volatile("prefetch.global.L2 [%0];" :: "l"(a.x));
+        asm volatile("prefetch.global.L2 [%0];" :: "l"(a.y));
+    }
 }
 
 // Phase 1b (after griddepcontrol.wait): Listing 1's group fetch, for the whole layer input.
@@ -154,7 +167,6 @@ template <typename T>
 __device__ __forceinline__ void issue_x(const StreamArgs& a, const SmemLayout& L) {
     constexpr int EPC = 16 / (int)sizeof(T);
     const int tid = threadIdx.x;
-    if (tid == 0) asm volatile("prefetch.global.L2 [%0];" :: "l"(a.y));   // warm the translation of the output page
     if (a.stage_mode != 0) {
         const bool via_raw = a.stage_mode != 2;
         const T* x = static_cast<const T*>(a.x);
@@ -184,7 +196,7 @@ __device__ __forceinline__ void finish_stage(const StreamArgs& a, const SmemLayo
         const int dst_stride = via_raw ? a.raw_stride : a.xs_stride;
         const int n_src = via_raw ? a.x_len : a.x_limit;
         const int n_dst = via_raw ? a.x_len : a.n_pad;
-        if (a.stage_mode == 3 && tid == 0) dst[-1] = T(0.0f);
+        if (a.stage_mode >= 3 && tid == 0) dst[-1] = T(0.0f);
         const int done = n_src / EPC * EPC;
         for (int b = 0; b < a.batch; ++b)
             for (int j = done + tid; j < n_dst; j += kThreads)
@@ -391,6 +403,7 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
     ring.prologue(wbeg, wend);
     XoffWindow xw;
     xw.init(a.xoff, wbeg, wend, lane);
+    warm_translations(a);
 
     // 2. everything before this kernel in the stream is complete from here on: fetch x
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -413,7 +426,7 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
         while (ls + 1 < d.s_count && L.sstart[ls + 1] <= wbeg) ++ls;
         int seg_end = min(wend, L.sstart[ls + 1]);
         const bool has_x = g < a.batch;
-        const bool direct = a.stage_mode == 3;
+        const bool direct = a.stage_mode >= 3, idx16 = a.stage_mode == 4;
         const unsigned short* rawu = static_cast<const unsigned short*>(L.raw);
         const __half* xrow = xs + g * a.xs_stride + 2 * t;
         for (int base = wbeg; base < wend; base += U) {
@@ -431,8 +444,17 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
                     uint32_t b0 = 0u, b1 = 0u;
                     if (direct) {            // batch 1: read x through the index array (index -1 reads raw[-1] = 0)
                         if (g == 0) {
-                            const int2 i0 = *reinterpret_cast<const int2*>(L.idxs + xoff + 2 * t);
-                            const int2 i1 = *reinterpret_cast<const int2*>(L.idxs + xoff + 2 * t + 8);
+                            int2 i0, i1;
+                            if (idx16) {
+                                const uint16_t* t16 = reinterpret_cast<const uint16_t*>(L.idxs) + xoff + 2 * t;
+                                const uint32_t p0 = *reinterpret_cast<const uint32_t*>(t16);
+                                const uint32_t p1 = *reinterpret_cast<const uint32_t*>(t16 + 8);
+                                i0 = make_int2((int)(p0 & 0xffffu) - 1, (int)(p0 >> 16) - 1);
+                                i1 = make_int2((int)(p1 & 0xffffu) - 1, (int)(p1 >> 16) - 1);
+                            } else {
+                                i0 = *reinterpret_cast<const int2*>(L.idxs + xoff + 2 * t);
+                                i1 = *reinterpret_cast<const int2*>(L.idxs + xoff + 2 * t + 8);
+                            }
                             b0 = (uint32_t)rawu[i0.x] | ((uint32_t)rawu[i0.y] << 16);
                             b1 = (uint32_t)rawu[i1.x] | ((uint32_t)rawu[i1.y] << 16);
                         }
@@ -472,6 +494,7 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const __grid_co
     ring.prologue(wbeg, wend);
     XoffWindow xw;
     xw.init(a.xoff, wbeg, wend, lane);
+    warm_translations(a);
     asm volatile("griddepcontrol.wait;" ::: "memory");
     issue_x<float>(a, L);
     finish_stage<float, U>(a, L);
@@ -494,7 +517,7 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const __grid_co
         while (ls + 1 < d.s_count && L.sstart[ls + 1] <= wbeg) ++ls;
         int seg_end = min(wend, L.sstart[ls + 1]);
         const float* xlane = xs + (lane / RG) * 4;
-        const bool direct = a.stage_mode == 3;
+        const bool direct = a.stage_mode >= 3, idx16 = a.stage_mode == 4;
         const float* rawf = static_cast<const float*>(L.raw);
         for (int base = wbeg; base < wend; base += U) {
 #pragma unroll
@@ -512,7 +535,13 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const __grid_co
                     const float w0 = __uint_as_float(wa.x), w1 = __uint_as_float(wa.y);
                     const float w2 = __uint_as_float(wa.z), w3 = __uint_as_float(wa.w);
                     if (direct) {            // batch 1: read x through the index array (index -1 reads raw[-1] = 0)
-                        const int4 ii = *reinterpret_cast<const int4*>(L.idxs + xoff + (lane / RG) * 4);
+                        int4 ii;
+                        if (idx16) {
+                            const uint2 pp2 = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(L.idxs) + xoff + (lane / RG) * 4);
+                            ii = make_int4((int)(pp2.x & 0xffffu) - 1, (int)(pp2.x >> 16) - 1, (int)(pp2.y & 0xffffu) - 1, (int)(pp2.y >> 16) - 1);
+                        } else {
+                            ii = *reinterpret_cast<const int4*>(L.idxs + xoff + (lane / RG) * 4);
+                        }
                         acc[0][0] = fmaf(w0, rawf[ii.x], acc[0][0]);
                         acc[0][1] = fmaf(w1, rawf[ii.y], acc[0][1]);
                         acc[0][0] = fmaf(w2, rawf[ii.z], acc[0][0]);
@@ -586,7 +615,9 @@ size_t smem_bytes_at(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, i
 // SM).  A CTA that has the SM to itself takes the deepest ring that still fits.
 int stream_pick_depth(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int grid) {
     if (g_stream_depth) return g_stream_depth;
-    if (grid > 148 && smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, 4) <= 113 * 1024) return 4;
+    if (grid > 148 && smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, 4) <= 113 * 1024) {
+        return 4;                 // two CTAs per SM: deeper rings measured no faster
+    }
     for (int d : {8, 6})
         if (smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, d) <= kStreamSmemLimit) return d;
     return 4;
@@ -603,9 +634,9 @@ size_t smem_bytes_at(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, i
     const int esz = dt == PP_F16 ? 2 : 4;
     size_t bytes = (size_t)kHeaderBytes + (size_t)max_rows * 8 + (size_t)kStreamSegSlots * rg * batch * 4 +
                    (size_t)kStreamWarps * depth * 512;
-    if (stage_mode != 3) bytes += xs_bytes(batch, xs_stride_for(dt, n_pad), esz);
-    if (stage_mode == 1 || stage_mode == 3)
-        bytes += (size_t)n_pad * 4 + 16 + (size_t)batch * ((x_len + 15) / 16 * 16) * esz;
+    if (stage_mode < 3) bytes += xs_bytes(batch, xs_stride_for(dt, n_pad), esz);
+    if (stage_mode == 1 || stage_mode >= 3)
+        bytes += (size_t)n_pad * (stage_mode == 4 ? 2 : 4) + 16 + (size_t)batch * ((x_len + 15) / 16 * 16) * esz;
     return bytes;
 }
 }  // namespace
@@ -616,7 +647,9 @@ cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a_in, const Ct
     StreamLaunch P;
     P.a = a_in;
     StreamArgs& a = P.a;
-    if (a.batch < 1 || a.batch > kStreamMaxBatch || (a.stage_mode == 3 && a.batch != 1)) return cudaErrorInvalidValue;
+    if (a.batch < 1 || a.batch > kStreamMaxBatch || (a.stage_mode >= 3 && a.batch != 1) ||
+        (a.stage_mode == 4 && !a.gather16))
+        return cudaErrorInvalidValue;
     a.xs_stride = xs_stride_for(dt, a.n_pad);
     a.raw_stride = (a.x_len + 15) / 16 * 16;
     a.max_rows = (a.max_rows + 3) / 4 * 4;

@@ -13,6 +13,7 @@ struct StreamArgs {
     const CtaDesc* cta_desc;     // [grid]
     const StripInfo* strip_info; // [S]
     const int32_t* gather_idx;   // pivoted column -> index into x, -1 = reads 0; NULL = identity
+    const uint16_t* gather16;    // staging mode 4: the same map as 16-bit entries index + 1 (0 = reads 0)
     const int32_t* scatter_idx;  // pivoted row -> original row, -1 = padding
     const float* bias_piv;
     const void* x;               // [batch][ldx]
@@ -33,7 +34,8 @@ struct StreamArgs {
                                  // memory, permute there (needs 16-byte aligned rows); 2: x is already
                                  // in pivoted order (gather_idx == NULL), copy it (same alignment rule);
                                  // 3: batch 1 only: copy x and gather_idx as in 1 and read x through the
-                                 // index array inside the multiply loop (no permutation pass)
+                                 // index array inside the multiply loop (no permutation pass);
+                                 // 4: as 3 with the 16-bit index table (half the shared memory)
 };
 
 // Shared memory the kernel needs for this (dtype, n_pad, batch); the caller falls back to the
