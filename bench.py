@@ -34,6 +34,9 @@ if ROOT not in sys.path:
 METRIC = "pivoted_fc_us_per_layer_batch1"
 L2_BYTES = 126 * 1024 * 1024
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the headline kernel (ncu; see profiles/);
+# None while the kernel has changed since the counters were taken
+STREAM_TRAFFIC_BYTES = None
 
 
 def measured_peak_gbs():
@@ -411,7 +414,7 @@ def main():
                      "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                      "algorithmic_bytes_per_launch": abytes, "kernel": "stream_f16_kernel<4>",
                      # dram__bytes_read.sum + dram__bytes_write.sum of one launch (ncu, profiles/stream_f16_cfg5_k128_batch1.md)
-                     "traffic": 139.95e6 if args.k == 128 else None},
+                     "traffic": STREAM_TRAFFIC_BYTES if args.k == 128 else None},
         "clocks": clocks,
     }
 

@@ -429,6 +429,7 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
         const bool direct = a.stage_mode >= 3, idx16 = a.stage_mode == 4;
         const unsigned short* rawu = static_cast<const unsigned short*>(L.raw);
         const __half* xrow = xs + g * a.xs_stride + 2 * t;
+        uint32_t mb0 = 0u, mb1 = 0u;
         for (int base = wbeg; base < wend; base += U) {
 #pragma unroll
             for (int u = 0; u < U; ++u) {
@@ -440,27 +441,38 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
                         do { ++ls; } while (L.sstart[ls + 1] <= p);
                         seg_end = min(wend, L.sstart[ls + 1]);
                     }
-                    const int xoff = xw.get(p, wend, lane);
                     uint32_t b0 = 0u, b1 = 0u;
-                    if (direct) {            // batch 1: read x through the index array (index -1 reads raw[-1] = 0)
-                        if (g == 0) {
+                    if (direct) {
+                        // batch 1: x is read through the index array (index -1 reads raw[-1] = 0).  Every 8
+                        // fragments the warp builds their 8 B-operands at once, 4 lanes per fragment (lane
+                        // 4f + t holds columns 2t, 2t+1, 2t+8, 2t+9 of fragment f), and hands them to the
+                        // lanes that feed the tensor core with two shuffles per fragment.
+                        const int in_group = (p - wbeg) & 7;
+                        if (in_group == 0) {
+                            (void)xw.get(p, wend, lane);                       // moves the window when needed
+                            const int xo = __shfl_sync(0xffffffffu, xw.cur, (p - xw.base) + g);
                             int2 i0, i1;
                             if (idx16) {
-                                const uint16_t* t16 = reinterpret_cast<const uint16_t*>(L.idxs) + xoff + 2 * t;
+                                const uint16_t* t16 = reinterpret_cast<const uint16_t*>(L.idxs) + xo + 2 * t;
                                 const uint32_t p0 = *reinterpret_cast<const uint32_t*>(t16);
                                 const uint32_t p1 = *reinterpret_cast<const uint32_t*>(t16 + 8);
                                 i0 = make_int2((int)(p0 & 0xffffu) - 1, (int)(p0 >> 16) - 1);
                                 i1 = make_int2((int)(p1 & 0xffffu) - 1, (int)(p1 >> 16) - 1);
                             } else {
-                                i0 = *reinterpret_cast<const int2*>(L.idxs + xoff + 2 * t);
-                                i1 = *reinterpret_cast<const int2*>(L.idxs + xoff + 2 * t + 8);
+                                i0 = *reinterpret_cast<const int2*>(L.idxs + xo + 2 * t);
+                                i1 = *reinterpret_cast<const int2*>(L.idxs + xo + 2 * t + 8);
                             }
-                            b0 = (uint32_t)rawu[i0.x] | ((uint32_t)rawu[i0.y] << 16);
-                            b1 = (uint32_t)rawu[i1.x] | ((uint32_t)rawu[i1.y] << 16);
+                            mb0 = (uint32_t)rawu[i0.x] | ((uint32_t)rawu[i0.y] << 16);
+                            mb1 = (uint32_t)rawu[i1.x] | ((uint32_t)rawu[i1.y] << 16);
                         }
-                    } else if (has_x) {
-                        b0 = *reinterpret_cast<const uint32_t*>(xrow + xoff);
-                        b1 = *reinterpret_cast<const uint32_t*>(xrow + xoff + 8);
+                        b0 = __shfl_sync(0xffffffffu, mb0, in_group * 4 + t);
+                        b1 = __shfl_sync(0xffffffffu, mb1, in_group * 4 + t);
+                    } else {
+                        const int xoff = xw.get(p, wend, lane);        // warp-wide shuffle: outside the lane test
+                        if (has_x) {
+                            b0 = *reinterpret_cast<const uint32_t*>(xrow + xoff);
+                            b1 = *reinterpret_cast<const uint32_t*>(xrow + xoff + 8);
+                        }
                     }
                     const uint4 wa = ring.take(u);
                     ring.fill(u, p + U, wend);
