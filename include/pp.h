@@ -186,12 +186,21 @@ pp_status_t pp_chain_forward(pp_chain_t* chain, const void* x, void* y, int batc
  * h      device, [H], element type of the layer: in h_0, out h_T (h is stored
  *        rounded to that type after every step, because it is a layer input)
  * c      device, float[H]: in c_0, out c_T
- * Enqueues 1 + 2*steps kernels on the stream; no synchronisation. */
+ * Enqueues work on the stream without synchronising.  fp16 gate layers whose
+ * weights fit the shared memory of the whole GPU (one CTA per SM, H <= 2048)
+ * run all steps in ONE cooperative kernel that keeps the weights on chip and
+ * meets at one grid barrier per step (1 preparation kernel + 1 memset + 1
+ * kernel; tuning key 11 = 0 switches this off); every other layer takes 1 + 2*steps
+ * kernels.  The barrier's waits are bounded: when one gives up the kernel ends,
+ * the outputs are invalid and pp_lstm_status reports PP_ERR_TIMEOUT.
+ * pp_lstm_status synchronises with the device, writes PP_OK or PP_ERR_TIMEOUT
+ * to *status and clears the flag. */
 typedef struct pp_lstm pp_lstm_t;
 pp_status_t pp_lstm_create(pp_lstm_t** out, pp_layer_t* gates, int I, int H, int max_steps);
 pp_status_t pp_lstm_destroy(pp_lstm_t* lstm);
 pp_status_t pp_lstm_forward(pp_lstm_t* lstm, const void* x_seq, void* h, float* c, int steps,
                             void* cuda_stream);
+pp_status_t pp_lstm_status(pp_lstm_t* lstm, pp_status_t* status);
 
 /* ------------------------------------------------------------------------- *
  * Forward call that allocates nothing (the paper has no counterpart; this is a
@@ -244,7 +253,8 @@ pp_status_t pp_forward_noalloc(const pp_packed_t* p, const void* device_image,
  * key 8: 1 (default) launches the persistent kernel with programmatic stream serialization, 0 plainly
  * key 10: 1 (default) permutes multi-column inputs in a pre-pass kernel when the layer kernel cannot hold x
  *         twice in shared memory; 0 leaves the gather to the layer kernel; 2 always uses the pre-pass
- * key 9: smallest batch for which fp16 layers with B = 64 take the tensor-core tile path (default 64; 0 = never) */
+ * key 9: smallest batch for which fp16 layers with B = 64 take the tensor-core tile path (default 64; 0 = never)
+ * key 11: 1 (default) lets pp_lstm_forward run all steps in one cooperative kernel when the layer qualifies, 0 never */
 pp_status_t pp_set_tuning(int key, int value);
 
 #ifdef __cplusplus

@@ -179,11 +179,12 @@ def _sigmoid(v):
     return 1.0 / (1.0 + np.exp(-v))
 
 
-def lstm_step(W, x_t, h_prev, c_prev, threads: int = 1):
-    """One cell update; returns (pre-activations g [4H], |W||z| [4H], c_t, h_t)."""
+def lstm_step(W, x_t, h_prev, c_prev, threads: int = 1, bias=None):
+    """One cell update; returns (pre-activations g [4H], |W||z| [4H], c_t, h_t).
+    A layer bias, when given, is part of g = W z + b like in any other layer (Eq. 2)."""
     H = h_prev.size
     z = np.concatenate([np.asarray(x_t, dtype=np.float64).ravel(), h_prev])
-    _, g, a = dense_forward(W, None, z[None, :], 0, threads)
+    _, g, a = dense_forward(W, bias, z[None, :], 0, threads)
     g = g[0]
     i, f, gg, o = g[0:H], g[H:2 * H], g[2 * H:3 * H], g[3 * H:4 * H]
     c = _sigmoid(f) * c_prev + _sigmoid(i) * np.tanh(gg)
@@ -192,7 +193,7 @@ def lstm_step(W, x_t, h_prev, c_prev, threads: int = 1):
 
 
 def lstm_forward(W, x_seq, H: int, h_round: Optional[str] = None, threads: int = 1,
-                 h0=None, c0=None):
+                 h0=None, c0=None, bias=None):
     """Free-running recurrence over x_seq [steps][I].  ``h_round`` rounds h_t to
     the layer's input storage type after every step (c stays fp64 here; the
     comparison tolerance covers the fp32 cell state of the device path)."""
@@ -200,7 +201,7 @@ def lstm_forward(W, x_seq, H: int, h_round: Optional[str] = None, threads: int =
     c = np.zeros(H) if c0 is None else np.asarray(c0, dtype=np.float64).copy()
     hs = []
     for t in range(x_seq.shape[0]):
-        _, _, c, h = lstm_step(W, x_seq[t], h, c, threads)
+        _, _, c, h = lstm_step(W, x_seq[t], h, c, threads, bias)
         h = _round_to(h, h_round)
         hs.append(h.copy())
     return h, c, np.stack(hs) if hs else np.zeros((0, H))

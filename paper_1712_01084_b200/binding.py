@@ -67,6 +67,7 @@ def lib() -> ctypes.CDLL:
         "pp_lstm_create": (ci, [ctypes.POINTER(vp), vp, ci, ci, ci]),
         "pp_lstm_destroy": (ci, [vp]),
         "pp_lstm_forward": (ci, [vp, vp, vp, vp, ci, vp]),
+        "pp_lstm_status": (ci, [vp, ctypes.POINTER(ci)]),
         "pp_pack_device_image_bytes": (ci, [vp, i64p]),
         "pp_pack_device_image": (ci, [vp, vp, c64]),
         "pp_forward_noalloc": (ci, [vp, vp, vp, vp, ci, ci, vp]),
@@ -341,6 +342,12 @@ class Lstm:
 
     def forward(self, x_seq, h, c, stream=None):
         return pp_lstm_forward(self, x_seq, h, c, stream=stream)
+
+    def status(self) -> int:
+        """0, or the code of a bounded device-side wait that gave up (synchronises; clears the flag)."""
+        out = ctypes.c_int(0)
+        _check(lib().pp_lstm_status(self._h, ctypes.byref(out)), "pp_lstm_status")
+        return out.value
 
     def close(self):
         if self._h:

@@ -60,7 +60,12 @@ struct pp_lstm {
     int32_t* d_inv_row = nullptr;
     int32_t* d_inv_col = nullptr;
     void* d_z = nullptr;           // [max_steps + 1][N_pad] inputs of every step in pivoted order
-    float* d_g = nullptr;          // [M_pad] gate pre-activations in pivoted order
+    float* d_g = nullptr;          // [M_pad] gate pre-activations in pivoted order; the persistent cell uses the
+                                   // allocation as [2][M_pad] 8-byte packets
+    unsigned int* d_sync = nullptr;   // persistent cell: [1] status word
+    int persist_grid = 0;          // CTAs of the persistent cell (0: layer does not qualify)
+    int persist_strips = 0;        // strips per CTA
+    size_t persist_smem = 0;
 };
 
 struct pp_chain {
@@ -71,6 +76,39 @@ struct pp_chain {
     std::vector<void*> d_inter;    // output of layer l in layer l+1's pivoted column order, element type of layer l+1
     int max_batch = 0;
 };
+
+namespace {
+
+// Persistent cell: fp16 gate layers whose strips, dealt out 1, 2, 4, 8 or 16 to a CTA, fit the shared
+// memory of at most one CTA per SM -- and a grid that size can be resident at once (cooperative launch).
+void lstm_plan_persistent(pp_lstm* R) {
+    const pp_packed* pk = R->gates->pk;
+    R->persist_grid = 0;
+    if (pk->wdtype != PP_F16 || R->H > 4 * 512 || pk->Npad % 8 != 0) return;
+    const int S = (int)pk->strip_start.size() - 1;
+    int dev = 0, sms = 0, coop = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop) {
+        cudaGetLastError();
+        return;
+    }
+    for (int ns = 1; ns <= 16; ns *= 2) {
+        const int grid = (S + ns - 1) / ns;
+        if (grid > sms) continue;
+        int max_frags = 0;
+        for (int c = 0; c < grid; ++c) {
+            const int s0 = c * ns, s1 = std::min(S, s0 + ns);
+            max_frags = std::max(max_frags, pk->strip_start[(size_t)s1] - pk->strip_start[(size_t)s0]);
+        }
+        const size_t smem = pp::lstm_persist_smem(max_frags, pk->Npad, pk->Mpad);
+        if (smem == 0) return;       // more strips per CTA only need more
+        R->persist_grid = grid; R->persist_strips = ns; R->persist_smem = smem;
+        return;
+    }
+}
+
+}  // namespace
 
 namespace {
 
@@ -484,6 +522,16 @@ pp_status_t pp_chain_forward(pp_chain_t* C, const void* x, void* y, int batch, v
     return PP_OK;
 }
 
+pp_status_t pp_lstm_status(pp_lstm_t* R, pp_status_t* status) {
+    if (!R || !status) return PP_ERR_INVALID_ARG;
+    unsigned int flag = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return PP_ERR_CUDA;
+    if (cudaMemcpy(&flag, R->d_sync + 1, sizeof(flag), cudaMemcpyDeviceToHost) != cudaSuccess) return PP_ERR_CUDA;
+    *status = flag ? PP_ERR_TIMEOUT : PP_OK;
+    if (flag && cudaMemset(R->d_sync + 1, 0, sizeof(flag)) != cudaSuccess) return PP_ERR_CUDA;
+    return PP_OK;
+}
+
 pp_status_t pp_lstm_create(pp_lstm_t** out, pp_layer_t* gates, int I, int H, int max_steps) {
     if (!out) return PP_ERR_INVALID_ARG;
     *out = nullptr;
@@ -499,7 +547,10 @@ pp_status_t pp_lstm_create(pp_lstm_t** out, pp_layer_t* gates, int I, int H, int
     const bool ok = upload(&R->d_inv_row, pk->inv_row_perm.data(), pk->inv_row_perm.size() * 4) &&
                     upload(&R->d_inv_col, inv_col.data(), inv_col.size() * 4) &&
                     cudaMalloc(&R->d_z, (size_t)(max_steps + 1) * pk->Npad * elt) == cudaSuccess &&
-                    cudaMalloc(reinterpret_cast<void**>(&R->d_g), (size_t)pk->Mpad * 4) == cudaSuccess;
+                    cudaMalloc(reinterpret_cast<void**>(&R->d_g), 2 * (size_t)pk->Mpad * 8) == cudaSuccess &&
+                    cudaMalloc(reinterpret_cast<void**>(&R->d_sync), 2 * sizeof(unsigned int)) == cudaSuccess &&
+                    cudaMemset(R->d_sync, 0, 2 * sizeof(unsigned int)) == cudaSuccess;
+    if (ok) lstm_plan_persistent(R);
     if (!ok) {
         const cudaError_t e = cudaGetLastError();
         pp_lstm_destroy(R);
@@ -511,7 +562,7 @@ pp_status_t pp_lstm_create(pp_lstm_t** out, pp_layer_t* gates, int I, int H, int
 
 pp_status_t pp_lstm_destroy(pp_lstm_t* R) {
     if (!R) return PP_OK;
-    cudaFree(R->d_inv_row); cudaFree(R->d_inv_col); cudaFree(R->d_z); cudaFree(R->d_g);
+    cudaFree(R->d_inv_row); cudaFree(R->d_inv_col); cudaFree(R->d_z); cudaFree(R->d_g); cudaFree(R->d_sync);
     delete R;
     return PP_OK;
 }
@@ -528,6 +579,17 @@ pp_status_t pp_lstm_forward(pp_lstm_t* R, const void* x_seq, void* h, float* c, 
     a.z = R->d_z; a.x_seq = x_seq; a.h = h; a.c = c; a.g_piv = R->d_g;
     a.I = R->I; a.H = R->H; a.n_pad = pk->Npad; a.steps = steps; a.f16 = pk->wdtype == PP_F16;
     if (pp::launch_lstm_prepare(a, stream) != cudaSuccess) return PP_ERR_CUDA;
+    if (pp::g_lstm_persist && R->persist_grid > 0) {
+        // all steps in one cooperative kernel; no packet of an earlier call may be mistaken for a new one
+        if (cudaMemsetAsync(R->d_g, 0, 2 * (size_t)pk->Mpad * 8, stream) != cudaSuccess) return PP_ERR_CUDA;
+        pp::LstmPersistArgs q{};
+        q.values = L->d_values; q.xoff = L->d_xoff; q.strip_start = L->d_strip_start; q.bias_piv = L->d_bias;
+        q.inv_row = R->d_inv_row; q.inv_col = R->d_inv_col; q.z = R->d_z; q.g_pk = reinterpret_cast<uint2*>(R->d_g);
+        q.status = reinterpret_cast<int*>(R->d_sync + 1); q.h = h; q.c = c;
+        q.I = R->I; q.H = R->H; q.n_pad = pk->Npad; q.m_pad = pk->Mpad; q.steps = steps;
+        q.n_strips = (int)pk->strip_start.size() - 1; q.strips_per_cta = R->persist_strips;
+        return pp::launch_lstm_persist(q, R->persist_grid, R->persist_smem, stream) == cudaSuccess ? PP_OK : PP_ERR_CUDA;
+    }
     for (int t = 0; t < steps; ++t) {
         const char* zt = static_cast<const char*>(R->d_z) + (size_t)t * pk->Npad * elt;
         // the input is already in pivoted order: no gather map, every pivoted column is real

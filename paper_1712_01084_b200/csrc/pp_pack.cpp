@@ -13,6 +13,7 @@ namespace pp {
 int g_use_stream = 1;      // 0: the API never picks the persistent kernel
 int g_tile_min_batch = 64;
 int g_prepass = 1;
+int g_lstm_persist = 1;
 int g_stage_direct = 1;    // 0: batch 1 also materialises the pivoted x in shared memory
 extern int g_stream_depth; // weight-ring slots per warp of the persistent kernel (pp_stream.cu)
 extern int g_stream_pdl;   // programmatic dependent launch of the persistent kernel (pp_stream.cu)
@@ -246,6 +247,7 @@ pp_status_t pp_set_tuning(int key, int value) {
     if (key == 8 && (value == 0 || value == 1)) { pp::g_stream_pdl = value; return PP_OK; }
     if (key == 9 && value >= 0) { pp::g_tile_min_batch = value; return PP_OK; }
     if (key == 10 && value >= 0 && value <= 2) { pp::g_prepass = value; return PP_OK; }
+    if (key == 11 && (value == 0 || value == 1)) { pp::g_lstm_persist = value; return PP_OK; }
     return PP_ERR_INVALID_ARG;
 }
 

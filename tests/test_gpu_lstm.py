@@ -37,8 +37,17 @@ def _step_bounds(a, c_prev, c, h, H):
     return dc, dh
 
 
+@pytest.fixture(params=[1, 0], ids=["persistent", "per-step"])
+def cell_mode(pb, request):
+    """Both ways pp_lstm_forward can run a qualifying fp16 layer: one cooperative kernel with the
+    weights resident in shared memory, or two kernels per step."""
+    pb.pp_set_tuning(11, request.param)
+    yield request.param
+    pb.pp_set_tuning(11, 1)
+
+
 @pytest.mark.parametrize("scale", [1 / 16, 1.0])
-def test_lstm_teacher_forced_steps(pb, scale):
+def test_lstm_teacher_forced_steps(pb, scale, cell_mode):
     steps = 12 if scale < 1 else 6
     wl = synth.config4(steps=steps, scale=scale)
     lay, H, I = wl.layers[0], wl.extra["H"], wl.extra["I"]
@@ -65,7 +74,7 @@ def test_lstm_teacher_forced_steps(pb, scale):
     cell.close(); L.close()
 
 
-def test_lstm_free_running_256_steps(pb):
+def test_lstm_free_running_256_steps(pb, cell_mode):
     wl = synth.config4(steps=256)
     lay, H, I = wl.layers[0], wl.extra["H"], wl.extra["I"]
     L = pb.Layer.from_synth(lay)
@@ -82,6 +91,29 @@ def test_lstm_free_running_256_steps(pb):
     h2 = torch.zeros_like(h); c2 = torch.zeros_like(c)
     pb.pp_lstm_forward(cell, torch.from_numpy(wl.x).cuda(), h2, c2)
     assert torch.equal(h, h2) and torch.equal(c, c2)
+    assert cell.status() == 0
+    cell.close(); L.close()
+
+
+@pytest.mark.parametrize("H,I,B,density", [(40, 56, 16, 1.0), (604, 420, 32, 0.4), (1208, 200, 64, 0.3)])
+def test_lstm_ragged_strip_counts_and_bias(pb, H, I, B, density, cell_mode):
+    """Strip counts that do not divide by the strips a CTA of the persistent cell holds (151 strips
+    dealt out in twos, 302 in fours), block-rows of unequal length, and a layer bias inside g."""
+    lay, rng = synth.make_layer(4100 + H, 4 * H, I + H, B, wdtype="f16", tiles="uniform", density=density,
+                                bias_std=0.3)
+    L = pb.Layer.from_synth(lay)
+    steps = 7
+    cell = pb.Lstm(L, I, H, max_steps=steps)
+    x_seq = rng.uniform(-1, 1, (steps, I)).astype(np.float16)
+    h0 = rng.uniform(-1, 1, H).astype(np.float16)
+    c0 = rng.uniform(-1, 1, H).astype(np.float32)
+    h = torch.from_numpy(h0).cuda(); c = torch.from_numpy(c0).cuda()
+    pb.pp_lstm_forward(cell, torch.from_numpy(x_seq).cuda(), h, c)
+    hr, cr, _ = po.lstm_forward(_dense(lay), x_seq.astype(np.float64), H, h_round="f16", threads=4,
+                                h0=h0, c0=c0, bias=lay.bias.astype(np.float64))
+    assert np.max(np.abs(h.cpu().numpy().astype(np.float64) - hr)) < 4e-3
+    assert np.max(np.abs(c.cpu().numpy().astype(np.float64) - cr)) < 4e-3
+    assert cell.status() == 0
     cell.close(); L.close()
 
 
