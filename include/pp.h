@@ -96,15 +96,21 @@ pp_status_t pp_pack_destroy(pp_packed_t* p);
  * (padded), [4]=number of work items, [5]=bytes of packed values,
  * [6]=max tiles in one work item, [7]=number of partial-sum slots,
  * [8]=S strips (row-groups of block-rows), [9]=F fragments (512-byte units of values),
- * [10]=CTAs of the persistent kernel's plan, [11]=its cross-CTA partial-sum slots. */
-pp_status_t pp_pack_info(const pp_packed_t* p, int64_t out[12]);
+ * [10]=CTAs of the persistent kernel's plan, [11]=its cross-CTA partial-sum slots,
+ * [12]=steps of the clustered tile kernel's plan (0 unless fp16 with B = 64). */
+pp_status_t pp_pack_info(const pp_packed_t* p, int64_t out[13]);
 
 /* Copy one packed array to host memory `dst` of capacity `bytes`.
  * which: 0 row_ptr(int32[Mb+1]) 1 col_ptr(int32[Mb+1]) 2 tile_col(int32[])
  *        3 gather_idx(int32[N_pad]) 4 scatter_idx(int32[M_pad]) 5 bias_piv(float[M_pad])
  *        6 values (bytes) 7 work items (int32[n_items][8]) 8 inv_row_perm(int32[M_pad])
  *        9 strip_start(int32[S+1]) 10 xoff(int32[F]) 11 CTA ranges (int32[G][4] =
- *        p_begin,p_end,s_first,s_count) 12 strip info (int32[S][4] = first_cta,nparts,slot_base,0) */
+ *        p_begin,p_end,s_first,s_count) 12 strip info (int32[S][4] = first_cta,nparts,slot_base,0)
+ *        13 steps of the clustered tile kernel (int32[steps][8] = tile-column, sorted-tile index for each
+ *        of the group's 4 block-rows or -1, tiles in the step, position of the step's first tile in the
+ *        step-ordered tile images, 0; groups of 4 block-rows one after the other, tile-columns ascending
+ *        inside a group) 14 its step boundaries (int32[ceil(Mb/4)][5]: CTA r of a group's cluster owns
+ *        steps [b[r], b[r+1])) 15 position of every sorted tile in the step-ordered images (int32[T]) */
 pp_status_t pp_pack_get(const pp_packed_t* p, int which, void* dst, int64_t bytes);
 
 /* Inverse of the value re-ordering: writes the sorted tile list (int32[T][2])
@@ -254,6 +260,9 @@ pp_status_t pp_forward_noalloc(const pp_packed_t* p, const void* device_image,
  * key 10: 1 (default) permutes multi-column inputs in a pre-pass kernel when the layer kernel cannot hold x
  *         twice in shared memory; 0 leaves the gather to the layer kernel; 2 always uses the pre-pass
  * key 9: smallest batch for which fp16 layers with B = 64 take the tensor-core tile path (default 64; 0 = never)
+ * key 12: tensor-core kernel of batched fp16 B = 64 layers: 0 one block-row per CTA; 2 the clustered kernel (4
+ *         block-rows per cluster of 4 CTAs share every X block); 1 (default) the clustered kernel when the
+ *         groups' tile-columns carry at least 3.5 of 4 possible tiles on average, else one block-row per CTA
  * key 11: 1 (default) lets pp_lstm_forward run all steps in one cooperative kernel when the layer qualifies, 0 never */
 pp_status_t pp_set_tuning(int key, int value);
 

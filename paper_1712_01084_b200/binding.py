@@ -123,11 +123,11 @@ class Packed:
         _check(lib().pp_pack_create(ctypes.byref(self._h), *args), "pp_pack_create")
         self.M, self.N, self.B = int(M), int(N), int(B)
         self.wdtype = np.asarray(tile_values).dtype
-        info = (ctypes.c_int64 * 12)()
+        info = (ctypes.c_int64 * 13)()
         _check(lib().pp_pack_info(self._h, info), "pp_pack_info")
         (self.Mb, self.Nb, self.T, self.n_tile_col, self.n_items, self.value_bytes,
          self.max_item_tiles, self.n_slots, self.n_strips, self.n_frags, self.stream_grid,
-         self.stream_slots) = [int(v) for v in info]
+         self.stream_slots, self.n_tile_steps) = [int(v) for v in info]
 
     def get(self, which: str) -> np.ndarray:
         Mpad, Npad = self.Mb * self.B, self.Nb * self.B
@@ -137,11 +137,17 @@ class Packed:
                 "values": (6, np.uint8, self.value_bytes), "items": (7, np.int32, self.n_items * 8),
                 "inv_row_perm": (8, np.int32, Mpad), "strip_start": (9, np.int32, self.n_strips + 1),
                 "xoff": (10, np.int32, self.n_frags), "cta_desc": (11, np.int32, self.stream_grid * 4),
-                "strip_info": (12, np.int32, self.n_strips * 4)}[which]
+                "strip_info": (12, np.int32, self.n_strips * 4),
+                "tile_steps": (13, np.int32, self.n_tile_steps * 8),
+                "tile_pos": (15, np.int32, self.T if self.n_tile_steps else 0),
+                "tile_parts": (14, np.int32, (-(-self.Mb // 4)) * 5 if self.n_tile_steps or
+                               (self.B == 64 and self.wdtype == np.float16) else 0)}[which]
         out = np.empty(spec[2], dtype=spec[1])
         _check(lib().pp_pack_get(self._h, spec[0], out.ctypes.data_as(ctypes.c_void_p), out.nbytes), "pp_pack_get")
-        if which == "items":
+        if which in ("items", "tile_steps"):
             return out.reshape(-1, 8)
+        if which == "tile_parts":
+            return out.reshape(-1, 5)
         return out.reshape(-1, 4) if which in ("cta_desc", "strip_info") else out
 
     def unpack(self):

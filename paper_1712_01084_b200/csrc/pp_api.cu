@@ -48,6 +48,10 @@ struct pp_layer {
     int32_t* d_row_ptr = nullptr;
     int32_t* d_col_ptr = nullptr;
     void* d_tiles_rm = nullptr;
+    int32_t* d_tile_pos = nullptr;       // sorted-tile index -> position in the step-ordered tile images
+    int32_t* d_tile_parts = nullptr;     // clustered tile kernel: step boundaries per group
+    pp::TileStep* d_tile_steps = nullptr;
+    int n_tile_steps = 0;
     unsigned char* d_tile_scratch = nullptr;
     void* d_x_piv = nullptr;
     int* d_status = nullptr;
@@ -200,21 +204,34 @@ bool tile_setup(pp_layer* L, const pp_layer* from) {
     const pp_packed* pk = L->pk;
     if (pk->wdtype != PP_F16 || pk->B != 64) return true;
     const size_t rp = round256((size_t)(pk->Mb + 1) * 4), tb = (size_t)pk->T * 64 * 64 * 2;
-    L->tile_bytes = 2 * rp + round256(tb);
+    const int groups = (pk->Mb + pp::kTileRows - 1) / pp::kTileRows;
+    const size_t pb = round256((size_t)groups * (pp::kTileRows + 1) * 4);
+    L->n_tile_steps = from ? from->n_tile_steps : (int)pk->tile_steps.size();
+    const size_t sb = round256((size_t)L->n_tile_steps * sizeof(pp::TileStep));
+    const size_t qb = round256((size_t)pk->T * 4);
+    L->tile_bytes = 2 * rp + pb + sb + qb + round256(tb);
     if (cudaMalloc(reinterpret_cast<void**>(&L->d_tile), L->tile_bytes) != cudaSuccess) return false;
     const size_t xb = round256((size_t)pp::kTileBatch * pk->Npad * 2);
     if (cudaMalloc(reinterpret_cast<void**>(&L->d_tile_scratch), xb + 256) != cudaSuccess) return false;
     if (cudaMemset(L->d_tile_scratch, 0, xb + 256) != cudaSuccess) return false;
     L->d_row_ptr = reinterpret_cast<int32_t*>(L->d_tile);
     L->d_col_ptr = reinterpret_cast<int32_t*>(L->d_tile + rp);
-    L->d_tiles_rm = L->d_tile + 2 * rp;
+    L->d_tile_parts = reinterpret_cast<int32_t*>(L->d_tile + 2 * rp);
+    L->d_tile_steps = reinterpret_cast<pp::TileStep*>(L->d_tile + 2 * rp + pb);
+    L->d_tile_pos = reinterpret_cast<int32_t*>(L->d_tile + 2 * rp + pb + sb);
+    L->d_tiles_rm = L->d_tile + 2 * rp + pb + sb + qb;
     L->d_x_piv = L->d_tile_scratch;
     L->d_status = reinterpret_cast<int*>(L->d_tile_scratch + xb);
     if (from) {
-        if (cudaMemcpy(L->d_tile, from->d_tile, L->tile_bytes, cudaMemcpyDeviceToDevice) != cudaSuccess) return false;
+        if (from->tile_bytes != L->tile_bytes ||
+            cudaMemcpy(L->d_tile, from->d_tile, L->tile_bytes, cudaMemcpyDeviceToDevice) != cudaSuccess) return false;
     } else {
         if (cudaMemcpy(L->d_row_ptr, pk->row_ptr.data(), (size_t)(pk->Mb + 1) * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
             cudaMemcpy(L->d_col_ptr, pk->col_ptr.data(), (size_t)(pk->Mb + 1) * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(L->d_tile_parts, pk->tile_parts.data(), pk->tile_parts.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+            (L->n_tile_steps && cudaMemcpy(L->d_tile_steps, pk->tile_steps.data(), (size_t)L->n_tile_steps * sizeof(pp::TileStep),
+                                           cudaMemcpyHostToDevice) != cudaSuccess) ||
+            (pk->T && cudaMemcpy(L->d_tile_pos, pk->tile_pos.data(), (size_t)pk->T * 4, cudaMemcpyHostToDevice) != cudaSuccess) ||
             (tb && cudaMemcpy(L->d_tiles_rm, pk->tiles_rm.data(), tb, cudaMemcpyHostToDevice) != cudaSuccess))   // already swizzled by the packer
             return false;
     }
@@ -422,11 +439,16 @@ pp_status_t pp_forward(pp_layer_t* L, const void* x, void* y, int batch, pp_act_
         t.scatter_idx = L->d_scatter; t.bias_piv = L->d_bias; t.status = L->d_status;
         t.tiles_sw = static_cast<const unsigned char*>(L->d_tiles_rm); t.x_sw = static_cast<const unsigned char*>(L->d_x_piv);
         t.ldy = pk->M; t.act = (int)act;
+        t.steps = L->d_tile_steps; t.parts = L->d_tile_parts; t.Mb = pk->Mb; t.tile_pos = L->d_tile_pos;
+        // The clustered kernel pays an exchange between its CTAs and walks every tile-column some block-row of
+        // a group uses: it wins (measured) once a step carries 3.5 of its 4 possible tiles on average.
+        const bool use_cluster = pp::g_tile_cluster == 2 ||
+                                 (pp::g_tile_cluster == 1 && L->n_tile_steps > 0 && 2 * pk->T >= 7 * (int64_t)L->n_tile_steps);
         for (int b0 = 0; b0 < batch; b0 += pp::kTileBatch) {
             t.batch = batch - b0 < pp::kTileBatch ? batch - b0 : pp::kTileBatch;
             t.y = static_cast<float*>(y) + (size_t)b0 * pk->M;
             const char* xc = static_cast<const char*>(x) + (size_t)b0 * pk->N * 2;
-            if (pp::launch_tile(t, xc, pk->N, pk->N, L->d_gather, pk->Npad, pk->Mb, stream) != cudaSuccess)
+            if (pp::launch_tile(t, xc, pk->N, pk->N, L->d_gather, pk->Npad, pk->Mb, use_cluster, stream) != cudaSuccess)
                 return PP_ERR_CUDA;
         }
         return PP_OK;

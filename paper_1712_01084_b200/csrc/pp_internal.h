@@ -39,6 +39,20 @@ struct StripInfo {
     int32_t pad;
 };
 static_assert(sizeof(CtaDesc) == 16 && sizeof(StripInfo) == 16, "read as 16-byte words");
+// --- clustered tensor-core tile kernel (fp16, B = 64) -------------------------------------------
+// kTileRows consecutive block-rows form a group that one thread-block cluster of kTileRows CTAs
+// computes.  A step is one tile-column some block-row of the group has a tile in; the CTA that owns
+// the step fetches that X block once and multiplies it with the (up to kTileRows) tiles of the step.
+constexpr int kTileRows = 4;
+struct TileStep {
+    int32_t col;                 // tile-column
+    int32_t tile[kTileRows];     // sorted-tile index per block-row of the group, -1: no tile there
+    int32_t ntiles;
+    int32_t pos;                 // position of the step's first tile in the step-ordered tile images
+    int32_t pad;
+};
+static_assert(sizeof(TileStep) == 32, "read as two 16-byte words");
+extern int g_tile_cluster;   // batched fp16 B = 64 layers: 0 one block-row per CTA, 2 the clustered kernel, 1 whichever fits the layer
 constexpr int kStreamWarps = 16;          // warps per CTA
 constexpr int kStreamMaxStrips = 48;      // strips one CTA may list
 constexpr int kStreamSegSlots = kStreamMaxStrips + kStreamWarps;   // (strip, warp) partial slots in shared memory
@@ -78,7 +92,11 @@ struct pp_packed {
     std::vector<uint16_t> gather16;                          // gather_idx + 1 as 16-bit entries (when N_pad < 65536)
     std::vector<float> bias_piv;
     std::vector<unsigned char> values;                       // fragment-ordered tile values
-    std::vector<unsigned char> tiles_rm;                     // fp16, B = 64 only: sorted tiles as swizzled 8 KiB images (tensor-core path)
+    std::vector<unsigned char> tiles_rm;                     // fp16, B = 64 only: tiles as swizzled 8 KiB images in step order
+                                                             // (group, tile-column, block-row) for the tensor-core path
+    std::vector<int32_t> tile_pos;                           // sorted-tile index -> position in tiles_rm
+    std::vector<pp::TileStep> tile_steps;                    // fp16, B = 64 only: steps of all groups, group after group
+    std::vector<int32_t> tile_parts;                         // [groups][kTileRows + 1] step boundaries of the cluster's CTAs
     std::vector<pp::WorkItem> items;
     // plan of the persistent streaming kernel
     std::vector<int32_t> strip_start;   // [S+1] fragment position of each strip

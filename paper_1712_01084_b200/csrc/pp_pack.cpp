@@ -14,6 +14,7 @@ int g_use_stream = 1;      // 0: the API never picks the persistent kernel
 int g_tile_min_batch = 64;
 int g_prepass = 1;
 int g_lstm_persist = 1;
+int g_tile_cluster = 1;
 int g_stage_direct = 1;    // 0: batch 1 also materialises the pivoted x in shared memory
 extern int g_stream_depth; // weight-ring slots per warp of the persistent kernel (pp_stream.cu)
 extern int g_stream_pdl;   // programmatic dependent launch of the persistent kernel (pp_stream.cu)
@@ -235,6 +236,70 @@ const char* pp_status_string(pp_status_t s) {
     return "unknown status";
 }
 
+// Plan of the clustered tile kernel: per group of kTileRows block-rows the union of their tile-columns
+// in ascending order (one step each), cut into kTileRows contiguous parts of about equal bytes
+// (16 KiB for the X block of a step + 8 KiB per tile).
+static void build_tile_steps(pp_packed* p) {
+    constexpr int R = pp::kTileRows;
+    const int G = (p->Mb + R - 1) / R;
+    p->tile_steps.clear();
+    p->tile_parts.assign((size_t)G * (R + 1), 0);
+    for (int g = 0; g < G; ++g) {
+        const size_t first = p->tile_steps.size();
+        std::vector<pp::TileStep> steps;
+        std::vector<int32_t> slot_of_col((size_t)p->Nb, -1);
+        std::vector<int32_t> cols;
+        for (int j = 0; j < R; ++j) {
+            const int br = g * R + j;
+            if (br >= p->Mb) break;
+            const int r0 = p->row_ptr[(size_t)br], k = p->row_ptr[(size_t)br + 1] - r0;
+            for (int t = 0; t < k; ++t) {
+                const int col = p->tile_col[(size_t)p->col_ptr[(size_t)br] + t];
+                if (slot_of_col[(size_t)col] < 0) { slot_of_col[(size_t)col] = 0; cols.push_back(col); }
+            }
+        }
+        std::sort(cols.begin(), cols.end());
+        steps.resize(cols.size());
+        for (size_t i = 0; i < cols.size(); ++i) {
+            slot_of_col[(size_t)cols[i]] = (int32_t)i;
+            steps[i].col = cols[i];
+            for (int j = 0; j < R; ++j) steps[i].tile[j] = -1;
+            steps[i].ntiles = 0; steps[i].pos = 0; steps[i].pad = 0;
+        }
+        for (int j = 0; j < R; ++j) {
+            const int br = g * R + j;
+            if (br >= p->Mb) break;
+            const int r0 = p->row_ptr[(size_t)br], k = p->row_ptr[(size_t)br + 1] - r0;
+            for (int t = 0; t < k; ++t) {
+                pp::TileStep& st = steps[(size_t)slot_of_col[(size_t)p->tile_col[(size_t)p->col_ptr[(size_t)br] + t]]];
+                st.tile[j] = r0 + t;
+                st.ntiles++;
+            }
+        }
+        int64_t total = 0;
+        for (const pp::TileStep& st : steps) total += 2 + st.ntiles;
+        int32_t* parts = &p->tile_parts[(size_t)g * (R + 1)];
+        int64_t run = 0;
+        int part = 1;
+        parts[0] = (int32_t)first;
+        for (size_t i = 0; i < steps.size(); ++i) {
+            // the step goes to the part its centre of mass falls into
+            while (part < R && (run + (2 + steps[i].ntiles) / 2) * R >= total * part) parts[part++] = (int32_t)(first + i);
+            run += 2 + steps[i].ntiles;
+        }
+        while (part <= R) parts[part++] = (int32_t)(first + steps.size());
+        p->tile_steps.insert(p->tile_steps.end(), steps.begin(), steps.end());
+    }
+    // the tiles of a step lie next to each other (block-rows ascending), steps one after the other
+    p->tile_pos.assign((size_t)p->T, 0);
+    int32_t pos = 0;
+    for (pp::TileStep& st : p->tile_steps) {
+        st.pos = pos;
+        for (int j = 0; j < R; ++j)
+            if (st.tile[j] >= 0) p->tile_pos[(size_t)st.tile[j]] = pos++;
+    }
+}
+
 pp_status_t pp_set_tuning(int key, int value) {
     if (key == 0 && value >= 1) { g_target_kib = value; return PP_OK; }
     if (key == 1 && value >= 0) { g_min_items = value; return PP_OK; }
@@ -248,6 +313,7 @@ pp_status_t pp_set_tuning(int key, int value) {
     if (key == 9 && value >= 0) { pp::g_tile_min_batch = value; return PP_OK; }
     if (key == 10 && value >= 0 && value <= 2) { pp::g_prepass = value; return PP_OK; }
     if (key == 11 && (value == 0 || value == 1)) { pp::g_lstm_persist = value; return PP_OK; }
+    if (key == 12 && value >= 0 && value <= 2) { pp::g_tile_cluster = value; return PP_OK; }
     return PP_ERR_INVALID_ARG;
 }
 
@@ -332,9 +398,11 @@ pp_status_t pp_pack_create(pp_packed_t** out, int M, int N, int B, const int32_t
         }
 
         if (wdtype == PP_F16 && B == 64) {       // second copy of the sorted tiles for the tensor-core path:
-            p->tiles_rm.resize((size_t)T * B * B * 2);   // each tile as its swizzled shared-memory image
+            build_tile_steps(p);
+            p->tiles_rm.resize((size_t)T * B * B * 2);   // each tile as its swizzled shared-memory image, in step order
             for (int64_t s2 = 0; s2 < T; ++s2)
-                pp::swizzle_tile_64x64(src + (size_t)order[(size_t)s2] * B * B * 2, &p->tiles_rm[(size_t)s2 * B * B * 2]);
+                pp::swizzle_tile_64x64(src + (size_t)order[(size_t)s2] * B * B * 2,
+                                       &p->tiles_rm[(size_t)p->tile_pos[(size_t)s2] * B * B * 2]);
         }
 
         p->gather_idx.resize((size_t)Npad);
@@ -365,10 +433,11 @@ pp_status_t pp_pack_destroy(pp_packed_t* p) {
     return PP_OK;
 }
 
-pp_status_t pp_pack_info(const pp_packed_t* p, int64_t out[12]) {
+pp_status_t pp_pack_info(const pp_packed_t* p, int64_t out[13]) {
     if (!p || !out) return PP_ERR_INVALID_ARG;
     out[8] = (int64_t)p->strip_start.size() - 1; out[9] = (int64_t)p->xoff.size();
     out[10] = (int64_t)p->cta_desc.size(); out[11] = p->stream_slots;
+    out[12] = (int64_t)p->tile_steps.size();
     out[0] = p->Mb; out[1] = p->Nb; out[2] = p->T; out[3] = (int64_t)p->tile_col.size();
     out[4] = (int64_t)p->items.size(); out[5] = (int64_t)p->values.size();
     out[6] = p->max_item_tiles; out[7] = p->n_slots;
@@ -393,6 +462,9 @@ pp_status_t pp_pack_get(const pp_packed_t* p, int which, void* dst, int64_t byte
         case 10: src = p->xoff.data(); n = p->xoff.size() * 4; break;
         case 11: src = p->cta_desc.data(); n = p->cta_desc.size() * sizeof(pp::CtaDesc); break;
         case 12: src = p->strip_info.data(); n = p->strip_info.size() * sizeof(pp::StripInfo); break;
+        case 13: src = p->tile_steps.data(); n = p->tile_steps.size() * sizeof(pp::TileStep); break;
+        case 14: src = p->tile_parts.data(); n = p->tile_parts.size() * 4; break;
+        case 15: src = p->tile_pos.data(); n = p->tile_pos.size() * 4; break;
         default: return PP_ERR_INVALID_ARG;
     }
     if ((size_t)bytes < n) return PP_ERR_INVALID_ARG;

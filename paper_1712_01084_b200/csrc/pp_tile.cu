@@ -8,14 +8,16 @@
 //     one CTA per batch row through shared memory, written as one 16 KiB block per tile-column that
 //     already has the 128-byte-swizzled shared-memory image the tensor core wants; the packer stores
 //     every weight tile as such an image (8 KiB) too;
-//   * warp 0 streams (X block, W tile) pairs into a ring of shared-memory stages with two bulk
-//     asynchronous copies per tile (cp.async.bulk, one request each, no multicast), signalling
-//     mbarriers (2-D tensor-map loads of 128-byte rows were request-rate bound: 60 us vs the
-//     same data as two contiguous copies);
-//   * warp 1 issues tcgen05.mma (kind::f16, accumulator in tensor memory) from shared-memory matrix
+//   * warps 0..3 (one lane each) stream (X block, W tile) pairs into a ring of shared-memory stages
+//     with two bulk asynchronous copies per tile (cp.async.bulk, one request each, no multicast),
+//     signalling mbarriers (2-D tensor-map loads of 128-byte rows were request-rate bound: 60 us vs
+//     the same data as two contiguous copies);
+//   * warp 4 issues tcgen05.mma (kind::f16, accumulator in tensor memory) from shared-memory matrix
 //     descriptors and frees each stage with tcgen05.commit;
-//   * warps 2..5 read the accumulator with tcgen05.ld and run the fused epilogue: bias, activation,
+//   * warps 5..8 read the accumulator with tcgen05.ld and run the fused epilogue: bias, activation,
 //     store through the row index array (Listing 1's last step).
+// A second kernel (further down) lets a cluster of four CTAs share the X blocks of four block-rows;
+// it wins when most tile-columns of a group carry tiles in all four block-rows.
 // Every wait on an mbarrier is bounded; on a time-out the kernel raises the layer's status word,
 // stops issuing work, lets its outstanding copies land, frees its tensor memory and returns.
 #include <cuda_fp16.h>
@@ -27,12 +29,12 @@ namespace pp {
 namespace {
 
 constexpr int kStages = 8;
-constexpr int kProducers = 4;      // lanes of warp 0 that issue bulk copies (kStages is a multiple of it)
+constexpr int kProducers = 4;      // producer warps (one lane each issues bulk copies; kStages is a multiple of it)
 constexpr int kXBytes = kTileBatch * 64 * 2;     // 128 x 64 fp16 = 16 KiB
 constexpr int kWBytes = 64 * 64 * 2;             // 64 x 64 fp16 = 8 KiB
 constexpr int kStageBytes = kXBytes + kWBytes;
 constexpr int kTmemCols = 64;
-constexpr int kThreads = 192;
+constexpr int kThreads = 32 * (kProducers + 1 + 4);    // producers, MMA issuer, 4 epilogue warps
 constexpr int kPollLimit = 1 << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -99,6 +101,8 @@ struct TileSmem {
     uint64_t acc_full;
     uint32_t tmem_base;
     int abort_flag;
+    float bias[64];           // bias and destination rows of the block-row
+    int dst[64];
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -117,7 +121,7 @@ tile_f16_kernel(const TileArgs a) {
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {
+    if (warp == kProducers) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      :: "r"(smem_u32(&sm->tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -128,14 +132,15 @@ tile_f16_kernel(const TileArgs a) {
     const uint32_t tmem = sm->tmem_base;
     volatile int* abort_flag = &sm->abort_flag;
 
-    if (warp == 0) {
-        // ---------------- producers: kProducers lanes, lane p feeds tiles p, p + kProducers, ...
-        // (one thread issues a bulk copy every ~0.15 us at best, which alone would cap the CTA)
-        if (lane < kProducers) {
+    if (warp < kProducers) {
+        // ---------------- producers: one lane of each of kProducers warps, warp p feeds tiles p, p + kProducers, ...
+        // (a thread is held for a few hundred ns per bulk copy it issues, and the lanes of one warp would
+        // take turns, so the requests come from different warps)
+        if (lane == 0) {
             int last = -1;
             const int cbase = __ldg(a.col_ptr + br);
             const int rot = k > 0 ? (int)(((long long)br * k) / gridDim.x) : 0;
-            for (int t = lane; t < k; t += kProducers) {
+            for (int t = warp; t < k; t += kProducers) {
                 const int s = t % kStages;
                 if (t >= kStages && !mbar_wait(&sm->empty[s], ((t / kStages) & 1) ^ 1, abort_flag)) break;
                 // block-rows start at different tiles of their lists, so that CTAs running side by side
@@ -144,7 +149,7 @@ tile_f16_kernel(const TileArgs a) {
                 const int col = __ldg(a.tile_col + cbase + tt);
                 mbar_expect_tx(&sm->full[s], kStageBytes);
                 bulk_load(stages + s * kStageBytes, a.x_sw + (size_t)col * kXBytes, kXBytes, &sm->full[s]);
-                bulk_load(stages + s * kStageBytes + kXBytes, a.tiles_sw + (size_t)(t0 + tt) * kWBytes, kWBytes, &sm->full[s]);
+                bulk_load(stages + s * kStageBytes + kXBytes, a.tiles_sw + (size_t)__ldg(a.tile_pos + t0 + tt) * kWBytes, kWBytes, &sm->full[s]);
                 last = t;
             }
             if (*abort_flag) {
@@ -153,7 +158,7 @@ tile_f16_kernel(const TileArgs a) {
                     for (int i = 0; i < kPollLimit && !mbar_try_wait(&sm->full[t % kStages], (t / kStages) & 1); ++i) {}
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == kProducers) {
         // ---------------- MMA issuer (one lane)
         if (lane == 0) {
             bool ok = true;
@@ -174,10 +179,17 @@ tile_f16_kernel(const TileArgs a) {
     } else {
         // ---------------- epilogue: 4 warps, warp (w % 4) owns tensor-memory lanes 32 (w % 4) ..
         const int q = warp & 3;
+        const int b = q * 32 + lane;                 // batch row inside the chunk
+        // while the main loop runs: bias and destination rows into shared memory (read by all four warps
+        // after the named barrier below)
+        if (b < 64) {
+            sm->bias[b] = __ldg(a.bias_piv + br * 64 + b);
+            sm->dst[b] = __ldg(a.scatter_idx + br * 64 + b);
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
         // the tensor-memory loads below are warp-wide instructions: the whole warp takes one decision
         const bool ok = __all_sync(0xffffffffu, mbar_wait(&sm->acc_full, 0, abort_flag) && !*abort_flag);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const int b = q * 32 + lane;                 // batch row inside the chunk
         if (ok) {
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
@@ -197,24 +209,280 @@ tile_f16_kernel(const TileArgs a) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) r[j] = 0u;
                 }
-                if (b < a.batch) {
+                // Transpose the 32 x 32 block through shared memory (the stages are idle by now), so that the
+                // lanes of a store run over output rows: 32 scattered words of ONE row of y.  With lanes over
+                // batch rows the words of a store lie a whole row pitch apart and crowd a few L2 slices.
+                float* xpose = reinterpret_cast<float*>(stages) + q * (32 * 33);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int i = br * 64 + c0 + j;
-                        float v = __uint_as_float(r[j]) + __ldg(a.bias_piv + i);
-                        if (a.act == PP_ACT_RELU) v = fmaxf(v, 0.0f);
-                        const int dst = __ldg(a.scatter_idx + i);
-                        if (dst >= 0) a.y[(size_t)b * a.ldy + dst] = v;
-                    }
+                for (int j = 0; j < 32; ++j) xpose[lane * 33 + j] = __uint_as_float(r[j]);
+                __syncwarp();
+                const float bias = sm->bias[c0 + lane];
+                const int dst = sm->dst[c0 + lane];
+#pragma unroll 8
+                for (int rr = 0; rr < 32; ++rr) {
+                    const int bb = q * 32 + rr;
+                    float v = xpose[rr * 33 + lane] + bias;
+                    if (a.act == PP_ACT_RELU) v = fmaxf(v, 0.0f);
+                    if (dst >= 0 && bb < a.batch) a.y[(size_t)bb * a.ldy + dst] = v;
                 }
+                __syncwarp();
             }
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (threadIdx.x == 0 && sm->abort_flag) *a.status = 1;
-    if (warp == 1) {
+    if (warp == kProducers) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Clustered variant.  With one block-row per CTA every CTA pulls the whole permuted input through
+// its L2 port (2 MiB of X for 1 MiB of weights at 8192 columns), every tile costs two copy requests
+// and every MMA re-reads its 128 x 16 slice of X from shared memory for just 64 output columns.
+// Here kTileRows consecutive block-rows form a group computed by a cluster of kTileRows CTAs:
+//   * CTA r owns a contiguous quarter of the group's tile-columns ("steps").  Per step it fetches
+//     the X block ONCE and, with one more request, the tiles all block-rows of the group have in that
+//     column (the packer stores them next to each other); four producer warps issue the requests;
+//   * the block-rows' accumulators sit side by side in tensor memory (4 x 64 columns), so the tiles
+//     of consecutive block-rows are the B operand of ONE instruction with N up to 256;
+//   * at the end the cluster meets at its hardware barrier (everybody's stage buffers are free),
+//     every CTA sends its partial accumulator of block-row j to CTA j with remote shared-memory
+//     stores, the cluster meets again, and CTA j adds the four partials in rank order and runs the
+//     epilogue for block-row j -- no global scratch, no atomics, the same bits on every run.
+constexpr int kCStages = 4;
+constexpr int kCProducers = 4;                                 // producer warps; warp w feeds stage w
+constexpr int kCStageBytes = kXBytes + kTileRows * kWBytes;    // 48 KiB: one X block + up to 4 tiles
+constexpr int kCTmemCols = 64 * kTileRows;
+static_assert(kTileRows * 64 * kTileBatch * 4 + 4 * 32 * 33 * 4 <= kCStages * kCStageBytes, "exchange buffers reuse the stages");
+__device__ __forceinline__ int q_of_warp(int warp) { return warp & 3; }
+constexpr int kCThreads = 32 * (kCProducers + 1 + 4);          // producers, MMA issuer, 4 epilogue warps
+static_assert(kCStages == kCProducers, "one stage per producer warp");
+
+struct ClusterSmem {
+    uint64_t full[kCStages];
+    uint64_t empty[kCStages];
+    uint64_t acc_full;
+    uint32_t tmem_base;
+    int abort_flag;
+    uint32_t acc_mask;        // accumulators that received at least one tile
+    float bias[64];           // bias and destination rows of the block-row this CTA finishes
+    int dst[64];
+};
+
+__device__ __forceinline__ TileStep load_step(const TileStep* p) {
+    const int4 lo = __ldg(reinterpret_cast<const int4*>(p)), hi = __ldg(reinterpret_cast<const int4*>(p) + 1);
+    TileStep s;
+    s.col = lo.x; s.tile[0] = lo.y; s.tile[1] = lo.z; s.tile[2] = lo.w; s.tile[3] = hi.x; s.ntiles = hi.y; s.pos = hi.z;
+    s.pad = 0;
+    return s;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t peer_addr(uint32_t local_addr, uint32_t rank) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    return remote;
+}
+__device__ __forceinline__ void st_peer_v4(uint32_t remote_addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" :: "r"(remote_addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+// tcgen05.mma with M = 128 and N = 64 * n_tiles (instruction descriptor built on the fly)
+__device__ __forceinline__ void umma_f16_n(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, int n_tiles, bool accumulate) {
+    const uint32_t idesc = (1u << 4) | (((uint32_t)(64 * n_tiles) >> 3) << 17) | ((128u >> 4) << 24);
+    asm volatile(
+        "{\n.reg .pred p;\nsetp.ne.u32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
+}
+
+__global__ void __cluster_dims__(kTileRows, 1, 1) __launch_bounds__(kCThreads, 1)
+tile_cluster_f16_kernel(const TileArgs a) {
+    static_assert(kTileRows == 4, "step records carry four tile slots");
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* stages = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    ClusterSmem* sm = reinterpret_cast<ClusterSmem*>(stages + kCStages * kCStageBytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint32_t rank;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    const int grp = blockIdx.x / kTileRows, n_groups = gridDim.x / kTileRows;
+    const int p0 = __ldg(a.parts + grp * (kTileRows + 1) + rank);
+    const int n_steps = __ldg(a.parts + grp * (kTileRows + 1) + rank + 1) - p0;
+    // clusters start at different steps of their ranges, so that the CTAs of equal rank (which walk the
+    // same tile-columns) do not all ask the L2 for the same X block at the same moment
+    const int rot = n_steps > 0 ? (int)(((long long)grp * n_steps) / n_groups) : 0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kCStages; ++s) { mbar_init(&sm->full[s], 1); mbar_init(&sm->empty[s], 1); }
+        mbar_init(&sm->acc_full, 2);          // the tensor core's commit + the issuing thread's own arrival
+        sm->abort_flag = 0;
+        sm->acc_mask = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kCProducers) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     :: "r"(smem_u32(&sm->tmem_base)), "r"(kCTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = sm->tmem_base;
+    volatile int* abort_flag = &sm->abort_flag;
+    // after the main loop the stage buffers hold what the peers send: [sender][16 row quads][128 batch][4]
+    // floats (a warp's remote store is one contiguous 512-byte run), and behind them a 32 x 33
+    // transposition tile per epilogue warp
+    float* recv = reinterpret_cast<float*>(stages);
+    float* xpose = recv + kTileRows * 64 * kTileBatch + q_of_warp(threadIdx.x >> 5) * (32 * 33);
+
+    if (warp < kCProducers) {
+        // ---------------- producers: warp w (one lane) feeds steps w, w + kCProducers, ... into stage w
+        if (lane == 0) {
+            const int s = warp;
+            int last = -1;
+            for (int t = warp; t < n_steps; t += kCProducers) {
+                if (t >= kCStages && !mbar_wait(&sm->empty[s], ((t / kCStages) & 1) ^ 1, abort_flag)) break;
+                const TileStep st = load_step(a.steps + p0 + (t + rot) % n_steps);
+                unsigned char* dst = stages + s * kCStageBytes;
+                mbar_expect_tx(&sm->full[s], (uint32_t)(kXBytes + st.ntiles * kWBytes));
+                bulk_load(dst, a.x_sw + (size_t)st.col * kXBytes, kXBytes, &sm->full[s]);
+                bulk_load(dst + kXBytes, a.tiles_sw + (size_t)st.pos * kWBytes, (uint32_t)(st.ntiles * kWBytes), &sm->full[s]);
+                last = t;
+            }
+            if (*abort_flag && last >= 0) {
+                // let the copies still in flight land before shared memory is reused or goes away
+                for (int i = 0; i < kPollLimit && !mbar_try_wait(&sm->full[s], (last / kCStages) & 1); ++i) {}
+            }
+        }
+    } else if (warp == kCProducers) {
+        // ---------------- MMA issuer (one lane)
+        if (lane == 0) {
+            bool ok = true;
+            uint32_t mask = 0u;
+            for (int t = 0; t < n_steps && ok; ++t) {
+                const int s = t % kCStages;
+                const TileStep st = load_step(a.steps + p0 + (t + rot) % n_steps);
+                ok = mbar_wait(&sm->full[s], (t / kCStages) & 1, abort_flag);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t xa = smem_u32(stages + s * kCStageBytes);
+                // runs of consecutive block-rows that have a tile here and are in the same state (first tile
+                // or not) share one instruction: the tiles are consecutive in the stage, the accumulators in
+                // tensor memory
+                int slot = 0;
+                for (int j = 0; j < kTileRows;) {
+                    if (st.tile[j] < 0) { ++j; continue; }
+                    const bool started = ((mask >> j) & 1u) != 0u;
+                    int n = 1;
+                    while (j + n < kTileRows && st.tile[j + n] >= 0 && (((mask >> (j + n)) & 1u) != 0u) == started) ++n;
+                    const uint32_t wa = xa + kXBytes + slot * kWBytes;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        umma_f16_n(tmem + (uint32_t)(j * 64), smem_desc_sw128(xa + kk * 32), smem_desc_sw128(wa + kk * 32), n,
+                                   started || kk > 0);
+                    mask |= ((1u << n) - 1u) << j;
+                    slot += n;
+                    j += n;
+                }
+                umma_commit(&sm->empty[s]);          // frees the stage once these MMAs have read it
+            }
+            sm->acc_mask = ok ? mask : 0u;
+            if (mask != 0u && ok) umma_commit(&sm->acc_full);   // accumulators complete
+            else mbar_arrive(&sm->acc_full);                    // nothing in flight to wait for (no tile, or giving up)
+            mbar_arrive(&sm->acc_full);                         // releases acc_mask to the epilogue warps
+        }
+    }
+    // ---------------- epilogue warps: warp (w % 4) owns tensor-memory lanes 32 (w % 4) ..
+    const bool epi = warp > kCProducers;
+    const int q = warp & 3, b = q * 32 + lane;
+    const int br = grp * kTileRows + (int)rank;
+    bool ok = true;
+    if (epi) {
+        // while the main loop runs: bias and destination rows of this CTA's block-row into shared memory
+        if (b < 64) {
+            const bool live = br < a.Mb;
+            sm->bias[b] = live ? __ldg(a.bias_piv + br * 64 + b) : 0.0f;
+            sm->dst[b] = live ? __ldg(a.scatter_idx + br * 64 + b) : -1;
+        }
+        ok = __all_sync(0xffffffffu, mbar_wait(&sm->acc_full, 0, abort_flag) && !*abort_flag);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    // Every CTA of the cluster gets here, also one that gave up (the barrier is the hardware's).  Past it
+    // no CTA of the cluster reads or fills its stage buffers any more.
+    cluster_sync_all();
+    if (epi && ok) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t mask = sm->acc_mask;
+        const uint32_t mine = smem_u32(recv) + (uint32_t)(((int)rank * 16) * kTileBatch + b) * 16u;   // [sender = rank][0][b][0]
+#pragma unroll 1
+        for (int j = 0; j < kTileRows; ++j) {
+            const uint32_t dst = peer_addr(mine, (uint32_t)j);
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t r[32];
+                if ((mask >> j) & 1u) {           // warp-uniform
+                    asm volatile(
+                        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                        : "r"(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(j * 64 + c0)));
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = 0u;
+                }
+#pragma unroll
+                for (int i = 0; i < 32; i += 4)
+                    st_peer_v4(dst + (uint32_t)(((c0 + i) >> 2) * kTileBatch) * 16u, r[i], r[i + 1], r[i + 2], r[i + 3]);
+            }
+        }
+    }
+    cluster_sync_all();          // all partials have arrived (release / acquire at cluster scope)
+    if (epi && br < a.Mb && !sm->abort_flag) {
+        // ---------------- block-row `rank` of the group: add the four partials in sender order, epilogue.
+        // Lanes run over the output rows here: one store instruction then writes 32 scattered words of ONE
+        // row of y (lanes over batch rows would write words a whole row pitch apart, which all land in the
+        // same few L2 slices).
+#pragma unroll 1
+        for (int c0 = 0; c0 < 64; c0 += 32) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {            // lanes over batch rows: contiguous, conflict-free reads
+                const float4* src = reinterpret_cast<const float4*>(recv) + ((c0 + i) >> 2) * kTileBatch + b;
+                float4 v = src[0];
+#pragma unroll
+                for (int p = 1; p < kTileRows; ++p) {
+                    const float4 w = src[p * 16 * kTileBatch];
+                    v.x += w.x; v.y += w.y; v.z += w.z; v.w += w.w;
+                }
+                xpose[lane * 33 + i] = v.x; xpose[lane * 33 + i + 1] = v.y;
+                xpose[lane * 33 + i + 2] = v.z; xpose[lane * 33 + i + 3] = v.w;
+            }
+            __syncwarp();
+            const float bias = sm->bias[c0 + lane];
+            const int dst = sm->dst[c0 + lane];
+#pragma unroll 8
+            for (int r = 0; r < 32; ++r) {               // lanes over output rows
+                const int bb = q * 32 + r;
+                float v = xpose[r * 33 + lane] + bias;
+                if (a.act == PP_ACT_RELU) v = fmaxf(v, 0.0f);
+                if (dst >= 0 && bb < a.batch) a.y[(size_t)bb * a.ldy + dst] = v;
+            }
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && sm->abort_flag) *a.status = 1;
+    if (warp == kCProducers) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kCTmemCols) : "memory");
     }
 }
 
@@ -271,7 +539,7 @@ void swizzle_tile_64x64(const void* row_major, void* out) {
 }
 
 cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const int32_t* gather_idx, int n_pad, int Mb,
-                        cudaStream_t stream) {
+                        bool use_cluster, cudaStream_t stream) {
     if (a.batch < 1 || a.batch > kTileBatch) return cudaErrorInvalidValue;
     static bool configured = false;
     const size_t smem = (size_t)kStages * kStageBytes + sizeof(TileSmem) + 1024;
@@ -285,6 +553,18 @@ cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const 
                                                               const_cast<unsigned char*>(a.x_sw), a.batch);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    if (use_cluster && a.steps && a.parts) {
+        static bool configured_c = false;
+        const size_t smem_c = (size_t)kCStages * kCStageBytes + sizeof(ClusterSmem) + 1024;
+        if (!configured_c) {
+            e = cudaFuncSetAttribute(tile_cluster_f16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_c);
+            if (e != cudaSuccess) return e;
+            configured_c = true;
+        }
+        const int groups = (Mb + kTileRows - 1) / kTileRows;
+        tile_cluster_f16_kernel<<<groups * kTileRows, kCThreads, smem_c, stream>>>(a);
+        return cudaGetLastError();
+    }
     tile_f16_kernel<<<Mb, kThreads, smem, stream>>>(a);
     return cudaGetLastError();
 }

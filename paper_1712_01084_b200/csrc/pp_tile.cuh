@@ -14,20 +14,26 @@ struct TileArgs {
     const int32_t* tile_col;     // tile-column index of every kept tile
     const int32_t* scatter_idx;  // pivoted row -> original row, -1 = padding
     const float* bias_piv;
-    const unsigned char* tiles_sw;   // sorted kept tiles, each an 8 KiB swizzled shared-memory image
+    const unsigned char* tiles_sw;   // kept tiles in step order, each an 8 KiB swizzled shared-memory image
+    const int32_t* tile_pos;         // sorted-tile index -> position in tiles_sw
     const unsigned char* x_sw;       // [N_pad / 64] blocks of 16 KiB: 128 batch rows x 64 columns, swizzled (scratch)
     float* y;                    // [batch][ldy], first row of this chunk
     int* status;                 // raised to 1 when a bounded wait gave up
     int ldy;
     int batch;                   // rows of this chunk (1..kTileBatch)
     int act;
+    // clustered kernel only
+    const TileStep* steps;       // steps of all groups
+    const int32_t* parts;        // [groups][kTileRows + 1] step boundaries of each cluster's CTAs
+    int Mb;
 };
 
 // Host: the shared-memory image (128-byte swizzle) of one 64 x 64 row-major fp16 tile, 8 KiB.
 void swizzle_tile_64x64(const void* row_major, void* out);
 
-// Enqueue the gather pre-pass (x -> a.x_sw) and the tile kernel for one batch chunk.
+// Enqueue the gather pre-pass (x -> a.x_sw) and one of the tile kernels for one batch chunk:
+// use_cluster picks the kernel in which a cluster of kTileRows CTAs shares the X blocks of kTileRows block-rows.
 cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const int32_t* gather_idx, int n_pad, int Mb,
-                        cudaStream_t stream);
+                        bool use_cluster, cudaStream_t stream);
 
 }  // namespace pp

@@ -315,8 +315,16 @@ def test_input_permutation_prepass(pb, dtype, prepass):
 
 
 # ------------------------------------------------------------------ tensor-core tile path (batch >= 64)
+@pytest.fixture(params=[2, 0, 1], ids=["clustered", "row-per-cta", "auto"])
+def tile_kernel(pb, request):
+    """Both tensor-core kernels: a cluster of 4 CTAs per 4 block-rows, or one CTA per block-row."""
+    pb.pp_set_tuning(12, request.param)
+    yield request.param
+    pb.pp_set_tuning(12, 1)
+
+
 @pytest.mark.parametrize("batch", [64, 100, 128, 129, 300])
-def test_tile_path_small_layer(pb, batch):
+def test_tile_path_small_layer(pb, batch, tile_kernel):
     """fp16, B = 64: ragged sizes, unbalanced block-rows, one block-row without tiles, batch chunks of 128
     with a ragged last chunk; compared element by element, and bit for bit on integer data."""
     lay = _rand_layer(900 + batch, 5 * 64 - 3, 9 * 64 - 7, 64, np.float16, density=0.45, empty_rows=(2,))
@@ -344,7 +352,40 @@ def test_tile_path_small_layer(pb, batch):
     L.close()
 
 
-def test_config5_batch128_tile_path_sampled_rows(pb):
+def test_tile_path_both_kernels_same_bits_and_repeatable(pb):
+    """Unbalanced groups (a group with an empty block-row, a last group of 2 block-rows, a block-row
+    whose tiles all fall into one CTA's quarter): repeated calls give identical bits, and on integer
+    data the clustered kernel and the one-block-row kernel agree exactly."""
+    lay = _rand_layer(977, 10 * 64 - 9, 23 * 64 - 1, 64, np.float16, density=0.3, empty_rows=(5,), integer=True)
+    x = np.random.default_rng(3).integers(-2, 3, (128, lay.N)).astype(np.float16)
+    L = pb.Layer.from_synth(lay)
+    try:
+        pb.pp_set_tuning(12, 2)
+        y1 = pb.pp_forward(L, _dev(x), 0).cpu().numpy()
+        y1b = pb.pp_forward(L, _dev(x), 0).cpu().numpy()
+        pb.pp_set_tuning(12, 0)
+        y0 = pb.pp_forward(L, _dev(x), 0).cpu().numpy()
+    finally:
+        pb.pp_set_tuning(12, 1)
+    assert L.status() == 0
+    assert np.array_equal(y1, y1b) and np.array_equal(y1, y0)
+    y_ref, _, _ = po.layer_forward(lay, x.astype(np.float64), act=0, threads=8)
+    assert np.array_equal(y1.astype(np.float64), y_ref)
+    L.close()
+    lay = _rand_layer(978, 7 * 64, 12 * 64, 64, np.float16, density=0.6)
+    x = np.random.default_rng(4).uniform(-1, 1, (96, lay.N)).astype(np.float16)
+    L = pb.Layer.from_synth(lay)
+    try:
+        pb.pp_set_tuning(12, 2)
+        ya = pb.pp_forward(L, _dev(x), 1).cpu().numpy()
+        yb = pb.pp_forward(L, _dev(x), 1).cpu().numpy()
+    finally:
+        pb.pp_set_tuning(12, 1)
+    assert np.array_equal(ya, yb)
+    L.close()
+
+
+def test_config5_batch128_tile_path_sampled_rows(pb, tile_kernel):
     """Full size (8192 x 8192, density 25 %), batch 128, in the launch configuration the bench times;
     the oracle evaluates a sample of output rows."""
     wl = synth.config5(k=32, batch=128)

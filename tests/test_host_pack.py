@@ -397,3 +397,57 @@ def test_stream_plan_many_empty_strips_and_no_tiles():
         got = _emulate_stream(pk, x.astype(np.float64), 0, np.float16)
         y, _, a = po.layer_forward(lay, x.astype(np.float64), act=0)
         assert np.all(np.abs(got - y[0]) <= 1e-12 * (a[0] + 1))
+
+
+def test_clustered_tile_plan_covers_every_tile_once():
+    """Plan of the clustered tensor-core kernel (fp16, B = 64): per group of 4 block-rows one step per
+    distinct tile-column in ascending order, every kept tile in exactly one step slot of its own
+    block-row, and four contiguous parts per group that cover the group's steps."""
+    for seed, Mb, Nb, density in ((1, 10, 23, 0.3), (2, 4, 4, 1.0), (3, 3, 7, 0.5), (4, 9, 16, 0.1)):
+        lay, _ = synth.make_layer(seed, Mb * 64 - 5, Nb * 64 - 3, 64, wdtype="f16", tiles="uniform", density=density)
+        pk = pb.Packed(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values, lay.bias)
+        steps, parts = pk.get("tile_steps"), pk.get("tile_parts")
+        row_ptr, col_ptr, tile_col = pk.get("row_ptr"), pk.get("col_ptr"), pk.get("tile_col")
+        G = -(-Mb // 4)
+        assert parts.shape == (G, 5)
+        seen = np.zeros(pk.T, dtype=np.int64)
+        nxt = 0
+        for g in range(G):
+            assert parts[g, 0] == nxt and np.all(np.diff(parts[g]) >= 0)
+            nxt = parts[g, 4]
+            grp = steps[parts[g, 0]:parts[g, 4]]
+            assert np.all(np.diff(grp[:, 0]) > 0)                        # tile-columns ascending, distinct
+            want_cols = set()
+            for j in range(4):
+                br = g * 4 + j
+                k = row_ptr[br + 1] - row_ptr[br] if br < Mb else 0
+                cols = tile_col[col_ptr[br]:col_ptr[br] + k] if br < Mb else []
+                want_cols |= set(int(c) for c in cols)
+                col_of_tile = {int(row_ptr[br] + t): int(cols[t]) for t in range(k)}
+                for st in grp:
+                    if st[1 + j] >= 0:
+                        assert col_of_tile[int(st[1 + j])] == st[0]
+                        seen[st[1 + j]] += 1
+            assert set(int(c) for c in grp[:, 0]) == want_cols
+            assert np.array_equal(grp[:, 5], (grp[:, 1:5] >= 0).sum(axis=1))
+            # parts balanced by bytes: no part exceeds its share by more than one step's worth
+            cost = 2 + grp[:, 5]
+            if len(grp):
+                share = cost.sum() / 4
+                for r in range(4):
+                    assert cost[parts[g, r] - parts[g, 0]:parts[g, r + 1] - parts[g, 0]].sum() <= share + 6
+        assert nxt == len(steps)
+        assert np.all(seen == 1)
+        # step-ordered tile images: the tiles of a step lie next to each other, block-rows ascending,
+        # and the steps follow each other without a gap
+        tile_pos = pk.get("tile_pos")
+        assert sorted(tile_pos.tolist()) == list(range(pk.T))
+        nxt = 0
+        for st in steps:
+            assert st[6] == nxt
+            for j in range(4):
+                if st[1 + j] >= 0:
+                    assert tile_pos[st[1 + j]] == nxt
+                    nxt += 1
+        assert nxt == pk.T
+        pk.close()
