@@ -82,7 +82,9 @@ const char* pp_status_string(pp_status_t s);
  * row_perm      host, int32[M_pad]     col_perm   host, int32[N_pad]
  * tile_list     host, int32[T][2] = (block_row, block_col), any order
  * tile_values   host, [T][B][B] row-major inside a tile, W_piv coordinates,
- *               element type wdtype (PP_F32: float, PP_F16: IEEE binary16 bits)
+ *               element type wdtype (PP_F32: float, PP_F16: IEEE binary16 bits);
+ *               entries on padding rows (row_perm >= M) or padding columns
+ *               (col_perm >= N) are not part of W and are stored as zero
  * bias          host, float[M] in ORIGINAL row order, or NULL
  * ------------------------------------------------------------------------- */
 pp_status_t pp_pack_create(pp_packed_t** out, int M, int N, int B,
@@ -159,6 +161,17 @@ pp_status_t pp_layer_clone(pp_layer_t** out, const pp_layer_t* src);
 pp_status_t pp_forward(pp_layer_t* layer, const void* x, void* y, int batch,
                        pp_act_t act, void* cuda_stream);
 
+/* Output permutation elimination (Section 4.2.2): the same product, but the result stays in
+ * the layer's pivoted row order -- the last index array of Listing 1 is dropped and the host
+ * relabels the coordinates when it interprets the result (an argmax, a softmax).
+ * y_piv  device, float [batch][M_pad] (M_pad = M rounded up to a multiple of B), 16-byte
+ *        aligned: y_piv[b][i] = act(W x + b)[map[i]]; padding positions (map[i] < 0) hold 0
+ * pp_layer_output_map writes that map to HOST memory map[M_pad]: the original output row of
+ * every pivoted position, -1 for padding.  Other arguments and errors as pp_forward. */
+pp_status_t pp_forward_pivoted(pp_layer_t* layer, const void* x, float* y_piv, int batch,
+                               pp_act_t act, void* cuda_stream);
+pp_status_t pp_layer_output_map(const pp_layer_t* layer, int32_t* map);
+
 /* ------------------------------------------------------------------------- *
  * Chain of layers with folded permutations (Section 4.2.1): the row permutation
  * of a layer and the column permutation of the next one are folded into one
@@ -169,10 +182,25 @@ pp_status_t pp_forward(pp_layer_t* layer, const void* x, void* y, int batch,
  * layer l+1 rounded (to nearest even) to layer l+1's element type.
  * layers[l+1].N must equal layers[l].M.  The chain references its layers: they
  * must outlive it.  Intermediate buffers are sized for max_batch at create.
- * x: device [batch][N_0] (dtype of layer 0); y: device float [batch][M_last]. */
+ * x: device [batch][N_0] (dtype of layer 0); y: device float [batch][M_last].
+ *
+ * Cross-layer permutation elimination (Section 4.2.3): a link whose folded map is the
+ * identity (the consumer's column permutation equals the producer's row permutation on the
+ * real rows, equal padded lengths) uses no index array at all: the producer stores its
+ * pivoted rows as they are.  pp_chain_link_info writes identity[l] = 1 for every layer
+ * l >= 1 whose incoming link is of that kind (identity[0] = 0) to HOST memory
+ * identity[n_layers]; tuning key 13 = 0 sends such links through the map as well.
+ *
+ * Output permutation elimination (Section 4.2.2): after pp_chain_set_output_pivoted(chain, 1)
+ * pp_chain_forward leaves y in the last layer's pivoted row order, float
+ * [batch][M_pad_last], padding positions 0; pp_chain_output_map gives the relabelling
+ * (as pp_layer_output_map of the last layer).  Errors: PP_ERR_INVALID_ARG. */
 pp_status_t pp_chain_create(pp_chain_t** out, pp_layer_t* const* layers,
                             const pp_act_t* acts, int n_layers, int max_batch);
 pp_status_t pp_chain_destroy(pp_chain_t* chain);
+pp_status_t pp_chain_set_output_pivoted(pp_chain_t* chain, int enable);
+pp_status_t pp_chain_output_map(const pp_chain_t* chain, int32_t* map);
+pp_status_t pp_chain_link_info(const pp_chain_t* chain, int32_t* identity);
 pp_status_t pp_chain_forward(pp_chain_t* chain, const void* x, void* y, int batch,
                              void* cuda_stream);
 
@@ -263,6 +291,8 @@ pp_status_t pp_forward_noalloc(const pp_packed_t* p, const void* device_image,
  * key 12: tensor-core kernel of batched fp16 B = 64 layers: 0 one block-row per CTA; 2 the clustered kernel (4
  *         block-rows per cluster of 4 CTAs share every X block); 1 (default) the clustered kernel when the
  *         groups' tile-columns carry at least 3.5 of 4 possible tiles on average, else one block-row per CTA
+ * key 13: 1 (default) chain links whose folded map is the identity store pivoted rows without an index array,
+ *         0 sends them through the map like any other link
  * key 11: 1 (default) lets pp_lstm_forward run all steps in one cooperative kernel when the layer qualifies, 0 never */
 pp_status_t pp_set_tuning(int key, int value);
 

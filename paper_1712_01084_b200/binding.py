@@ -63,6 +63,11 @@ def lib() -> ctypes.CDLL:
         "pp_chain_create": (ci, [ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(ci), ci, ci]),
         "pp_chain_destroy": (ci, [vp]),
         "pp_chain_forward": (ci, [vp, vp, vp, ci, vp]),
+        "pp_chain_set_output_pivoted": (ci, [vp, ci]),
+        "pp_chain_output_map": (ci, [vp, i32p]),
+        "pp_chain_link_info": (ci, [vp, i32p]),
+        "pp_forward_pivoted": (ci, [vp, vp, vp, ci, ci, vp]),
+        "pp_layer_output_map": (ci, [vp, i32p]),
         "pp_set_tuning": (ci, [ci, ci]),
         "pp_lstm_create": (ci, [ctypes.POINTER(vp), vp, ci, ci, ci]),
         "pp_lstm_destroy": (ci, [vp]),
@@ -227,6 +232,12 @@ class Layer:
     def forward(self, x, act: int = PP_ACT_IDENTITY, out=None, stream=None):
         return pp_forward(self, x, act, out=out, stream=stream)
 
+    def output_map(self) -> np.ndarray:
+        """Original output row of every pivoted position, -1 for padding (pp_layer_output_map)."""
+        m = np.empty(-(-self.M // self.B) * self.B, dtype=np.int32)
+        _check(lib().pp_layer_output_map(self._h, m.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))), "pp_layer_output_map")
+        return m
+
     def status(self) -> int:
         """PP_OK, or PP_ERR_TIMEOUT when a kernel's bounded wait gave up (synchronises; clears the flag)."""
         st = ctypes.c_int(0)
@@ -276,6 +287,22 @@ def pp_forward(layer: Layer, x, act: int = PP_ACT_IDENTITY, out=None, stream=Non
     return y
 
 
+def pp_forward_pivoted(layer: Layer, x, act: int = PP_ACT_IDENTITY, out=None, stream=None):
+    """y_piv[batch][M_pad] (float32, CUDA): act(W x + b) left in the layer's pivoted row order
+    (pp_forward_pivoted); layer.output_map() relabels the positions."""
+    import torch
+    x2 = _check_x(x, layer.N, layer.wdtype)
+    batch = x2.shape[0]
+    m_pad = -(-layer.M // layer.B) * layer.B
+    y = torch.empty((batch, m_pad), dtype=torch.float32, device=x.device) if out is None else out
+    _require_cuda(y, "out")
+    if y.dtype != torch.float32 or y.numel() != batch * m_pad:
+        raise ValueError("out must be float32 [batch][M_pad]")
+    _check(lib().pp_forward_pivoted(layer._h, ctypes.c_void_p(x2.data_ptr()), ctypes.c_void_p(y.data_ptr()),
+                                    batch, int(act), _stream_ptr(stream)), "pp_forward_pivoted")
+    return y
+
+
 def pp_forward_noalloc(packed: Packed, device_image, x, act: int = PP_ACT_IDENTITY, out=None, stream=None):
     """pp_forward for callers that may not allocate: `device_image` is a CUDA uint8 tensor holding
     packed.device_image(); `out` must be given (this function creates no tensor)."""
@@ -305,9 +332,27 @@ class Chain:
         self._h = ctypes.c_void_p()
         _check(lib().pp_chain_create(ctypes.byref(self._h), arr, acts_arr, n, int(max_batch)), "pp_chain_create")
         self.max_batch = int(max_batch)
+        self.output_pivoted = False
 
     def forward(self, x, out=None, stream=None):
         return pp_chain_forward(self, x, out=out, stream=stream)
+
+    def set_output_pivoted(self, enable: bool = True):
+        """Leave the result in the last layer's pivoted row order (pp_chain_set_output_pivoted)."""
+        _check(lib().pp_chain_set_output_pivoted(self._h, 1 if enable else 0), "pp_chain_set_output_pivoted")
+        self.output_pivoted = bool(enable)
+
+    def output_map(self) -> np.ndarray:
+        last = self.layers[-1]
+        m = np.empty(-(-last.M // last.B) * last.B, dtype=np.int32)
+        _check(lib().pp_chain_output_map(self._h, m.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))), "pp_chain_output_map")
+        return m
+
+    def link_info(self) -> np.ndarray:
+        """identity[l] = 1 when the link into layer l needs no index array (pp_chain_link_info)."""
+        m = np.zeros(len(self.layers), dtype=np.int32)
+        _check(lib().pp_chain_link_info(self._h, m.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))), "pp_chain_link_info")
+        return m
 
     def close(self):
         if self._h:
@@ -330,8 +375,11 @@ def pp_chain_forward(chain: Chain, x, out=None, stream=None):
     first, last = chain.layers[0], chain.layers[-1]
     x2 = _check_x(x, first.N, first.wdtype)
     batch = x2.shape[0]
-    y = torch.empty((batch, last.M), dtype=torch.float32, device=x.device) if out is None else out
+    width = -(-last.M // last.B) * last.B if chain.output_pivoted else last.M
+    y = torch.empty((batch, width), dtype=torch.float32, device=x.device) if out is None else out
     _require_cuda(y, "out")
+    if y.dtype != torch.float32 or y.numel() != batch * width:
+        raise ValueError("out must be float32 [batch][M] ([batch][M_pad] when the output stays pivoted)")
     _check(lib().pp_chain_forward(chain._h, ctypes.c_void_p(x2.data_ptr()), ctypes.c_void_p(y.data_ptr()),
                                   batch, _stream_ptr(stream)), "pp_chain_forward")
     return y

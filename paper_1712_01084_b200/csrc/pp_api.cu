@@ -78,6 +78,8 @@ struct pp_chain {
     std::vector<int32_t*> d_q;     // entry l (l >= 1): folded map of the link l-1 -> l, as a STORE map of layer l-1:
                                    // pivoted row of layer l-1 -> pivoted column of layer l (-1: padding row)
     std::vector<void*> d_inter;    // output of layer l in layer l+1's pivoted column order, element type of layer l+1
+    std::vector<char> identity;    // entry l (l >= 1): the folded map of the link l-1 -> l is the identity (Section 4.2.3)
+    bool out_pivoted = false;      // the last layer leaves its output in pivoted row order (Section 4.2.2)
     int max_batch = 0;
 };
 
@@ -426,19 +428,17 @@ pp_status_t pp_layer_destroy(pp_layer_t* layer) {
     return PP_OK;
 }
 
-pp_status_t pp_forward(pp_layer_t* L, const void* x, void* y, int batch, pp_act_t act, void* cuda_stream) {
-    if (!L || !x || !y || batch < 1 || x == y) return PP_ERR_INVALID_ARG;
-    if (act != PP_ACT_IDENTITY && act != PP_ACT_RELU) return PP_ERR_INVALID_ARG;
-    if (!aligned16(x) || !aligned16(y)) return PP_ERR_INVALID_ARG;
+// One layer forward; pivoted: y is float[batch][M_pad] in pivoted row order (no output index array).
+static pp_status_t forward_impl(pp_layer* L, const void* x, void* y, int batch, pp_act_t act, cudaStream_t stream, bool pivoted) {
     const pp_packed* pk = L->pk;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int ldy = pivoted ? pk->Mpad : pk->M;
     if (L->tile_ok && pp::g_tile_min_batch > 0 && batch >= pp::g_tile_min_batch && (size_t)pk->N * 2 <= 48 * 1024) {
         // tensor-core tile path, 128 batch rows at a time
         pp::TileArgs t{};
         t.row_ptr = L->d_row_ptr; t.col_ptr = L->d_col_ptr; t.tile_col = L->d_tile_col;
         t.scatter_idx = L->d_scatter; t.bias_piv = L->d_bias; t.status = L->d_status;
         t.tiles_sw = static_cast<const unsigned char*>(L->d_tiles_rm); t.x_sw = static_cast<const unsigned char*>(L->d_x_piv);
-        t.ldy = pk->M; t.act = (int)act;
+        t.ldy = ldy; t.act = (int)act; t.pivoted = pivoted ? 1 : 0;
         t.steps = L->d_tile_steps; t.parts = L->d_tile_parts; t.Mb = pk->Mb; t.tile_pos = L->d_tile_pos;
         // The clustered kernel pays an exchange between its CTAs and walks every tile-column some block-row of
         // a group uses: it wins (measured) once a step carries 3.5 of its 4 possible tiles on average.
@@ -446,15 +446,36 @@ pp_status_t pp_forward(pp_layer_t* L, const void* x, void* y, int batch, pp_act_
                                  (pp::g_tile_cluster == 1 && L->n_tile_steps > 0 && 2 * pk->T >= 7 * (int64_t)L->n_tile_steps);
         for (int b0 = 0; b0 < batch; b0 += pp::kTileBatch) {
             t.batch = batch - b0 < pp::kTileBatch ? batch - b0 : pp::kTileBatch;
-            t.y = static_cast<float*>(y) + (size_t)b0 * pk->M;
+            t.y = static_cast<float*>(y) + (size_t)b0 * ldy;
             const char* xc = static_cast<const char*>(x) + (size_t)b0 * pk->N * 2;
             if (pp::launch_tile(t, xc, pk->N, pk->N, L->d_gather, pk->Npad, pk->Mb, use_cluster, stream) != cudaSuccess)
                 return PP_ERR_CUDA;
         }
         return PP_OK;
     }
-    return run_layer(L, L->d_gather, x, pk->N, pk->N, pk->wdtype == PP_F16 ? 2 : 4, y, pk->M, pp::OUT_SCATTER_F32,
-                     batch, act, stream);
+    return run_layer(L, L->d_gather, x, pk->N, pk->N, pk->wdtype == PP_F16 ? 2 : 4, y, ldy,
+                     pivoted ? pp::OUT_PIVOTED_F32 : pp::OUT_SCATTER_F32, batch, act, stream);
+}
+
+pp_status_t pp_forward(pp_layer_t* L, const void* x, void* y, int batch, pp_act_t act, void* cuda_stream) {
+    if (!L || !x || !y || batch < 1 || x == y) return PP_ERR_INVALID_ARG;
+    if (act != PP_ACT_IDENTITY && act != PP_ACT_RELU) return PP_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y)) return PP_ERR_INVALID_ARG;
+    return forward_impl(L, x, y, batch, act, static_cast<cudaStream_t>(cuda_stream), false);
+}
+
+pp_status_t pp_layer_output_map(const pp_layer_t* L, int32_t* map) {
+    if (!L || !map) return PP_ERR_INVALID_ARG;
+    const pp_packed* pk = L->pk;
+    for (int i = 0; i < pk->Mpad; ++i) map[i] = pk->row_perm[(size_t)i] < pk->M ? pk->row_perm[(size_t)i] : -1;
+    return PP_OK;
+}
+
+pp_status_t pp_forward_pivoted(pp_layer_t* L, const void* x, float* y_piv, int batch, pp_act_t act, void* cuda_stream) {
+    if (!L || !x || !y_piv || batch < 1 || x == static_cast<const void*>(y_piv)) return PP_ERR_INVALID_ARG;
+    if (act != PP_ACT_IDENTITY && act != PP_ACT_RELU) return PP_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y_piv)) return PP_ERR_INVALID_ARG;
+    return forward_impl(L, x, y_piv, batch, act, static_cast<cudaStream_t>(cuda_stream), true);
 }
 
 pp_status_t pp_chain_create(pp_chain_t** out, pp_layer_t* const* layers, const pp_act_t* acts, int n_layers,
@@ -474,6 +495,7 @@ pp_status_t pp_chain_create(pp_chain_t** out, pp_layer_t* const* layers, const p
     C->max_batch = max_batch;
     C->d_q.assign((size_t)n_layers, nullptr);
     C->d_inter.assign((size_t)n_layers, nullptr);
+    C->identity.assign((size_t)n_layers, 0);
     bool ok = true;
     pp_status_t st = PP_OK;
     for (int l = 1; l < n_layers && ok; ++l) {
@@ -488,6 +510,12 @@ pp_status_t pp_chain_create(pp_chain_t** out, pp_layer_t* const* layers, const p
         std::vector<int32_t> store((size_t)A->Mpad, -1);
         for (int j = 0; j < Bk->Npad; ++j)
             if (q[(size_t)j] >= 0) store[(size_t)q[(size_t)j]] = j;
+        // Section 4.2.3: when every real producer row already sits at its consumer column (and the two
+        // padded lengths agree), the producer stores its pivoted rows as they are -- no index array on
+        // either side of the link.  Padding rows hold act(0) = 0 and land on padding columns.
+        bool ident = A->Mpad == Bk->Npad;
+        for (int i = 0; i < A->Mpad && ident; ++i) ident = store[(size_t)i] == i || store[(size_t)i] < 0;
+        C->identity[(size_t)l] = ident ? 1 : 0;
         ok = upload(&C->d_q[(size_t)l], store.data(), store.size() * 4);
         const size_t elt = Bk->wdtype == PP_F16 ? 2 : 4;
         const size_t ibytes = (size_t)max_batch * Bk->Npad * elt;
@@ -530,17 +558,43 @@ pp_status_t pp_chain_forward(pp_chain_t* C, const void* x, void* y, int batch, v
         const int x_limit = l == 0 ? pk->N : pk->Npad;
         pp_status_t st;
         if (l == n - 1) {
-            st = run_layer(L, gather, cur, ldx, x_len, x_elt, y, pk->M, pp::OUT_SCATTER_F32, batch, C->acts[(size_t)l], stream,
-                           x_limit);
+            if (C->out_pivoted)
+                st = run_layer(L, gather, cur, ldx, x_len, x_elt, y, pk->Mpad, pp::OUT_PIVOTED_F32, batch, C->acts[(size_t)l],
+                               stream, x_limit);
+            else
+                st = run_layer(L, gather, cur, ldx, x_len, x_elt, y, pk->M, pp::OUT_SCATTER_F32, batch, C->acts[(size_t)l],
+                               stream, x_limit);
         } else {
             const pp_packed* nx = C->layers[(size_t)l + 1]->pk;
-            st = run_layer(L, gather, cur, ldx, x_len, x_elt, C->d_inter[(size_t)l], nx->Npad,
-                           nx->wdtype == PP_F16 ? pp::OUT_SCATTER_F16 : pp::OUT_SCATTER_F32, batch, C->acts[(size_t)l], stream,
-                           x_limit, C->d_q[(size_t)l + 1]);
+            const bool f16 = nx->wdtype == PP_F16;
+            if (C->identity[(size_t)l + 1] && pp::g_link_identity)
+                st = run_layer(L, gather, cur, ldx, x_len, x_elt, C->d_inter[(size_t)l], nx->Npad,
+                               f16 ? pp::OUT_PIVOTED_F16 : pp::OUT_PIVOTED_F32, batch, C->acts[(size_t)l], stream, x_limit);
+            else
+                st = run_layer(L, gather, cur, ldx, x_len, x_elt, C->d_inter[(size_t)l], nx->Npad,
+                               f16 ? pp::OUT_SCATTER_F16 : pp::OUT_SCATTER_F32, batch, C->acts[(size_t)l], stream, x_limit,
+                               C->d_q[(size_t)l + 1]);
             cur = C->d_inter[(size_t)l];
         }
         if (st != PP_OK) return st;
     }
+    return PP_OK;
+}
+
+pp_status_t pp_chain_set_output_pivoted(pp_chain_t* C, int enable) {
+    if (!C || (enable != 0 && enable != 1)) return PP_ERR_INVALID_ARG;
+    C->out_pivoted = enable != 0;
+    return PP_OK;
+}
+
+pp_status_t pp_chain_output_map(const pp_chain_t* C, int32_t* map) {
+    if (!C || !map) return PP_ERR_INVALID_ARG;
+    return pp_layer_output_map(C->layers.back(), map);
+}
+
+pp_status_t pp_chain_link_info(const pp_chain_t* C, int32_t* identity) {
+    if (!C || !identity) return PP_ERR_INVALID_ARG;
+    for (size_t l = 0; l < C->layers.size(); ++l) identity[l] = C->identity[l];
     return PP_OK;
 }
 

@@ -60,6 +60,7 @@ constexpr int kStreamMaxBatch = 8;
 extern int g_use_stream;
 extern int g_tile_min_batch;  // fp16 B = 64 layers take the tensor-core tile path from this batch on (0: never)
 extern int g_prepass;         // 1: permute multi-column inputs in a pre-pass when the kernel cannot do it in shared memory
+extern int g_link_identity;  // 1: chain links whose folded map is the identity store pivoted rows directly (Section 4.2.3)
 extern int g_lstm_persist;  // 1: recurrent cells run all steps in one cooperative kernel when the gate weights fit shared memory
 extern int g_stage_direct;   // batch 1: read x through the index array instead of permuting it first
 

@@ -15,6 +15,7 @@ int g_tile_min_batch = 64;
 int g_prepass = 1;
 int g_lstm_persist = 1;
 int g_tile_cluster = 1;
+int g_link_identity = 1;
 int g_stage_direct = 1;    // 0: batch 1 also materialises the pivoted x in shared memory
 extern int g_stream_depth; // weight-ring slots per warp of the persistent kernel (pp_stream.cu)
 extern int g_stream_pdl;   // programmatic dependent launch of the persistent kernel (pp_stream.cu)
@@ -314,6 +315,7 @@ pp_status_t pp_set_tuning(int key, int value) {
     if (key == 10 && value >= 0 && value <= 2) { pp::g_prepass = value; return PP_OK; }
     if (key == 11 && (value == 0 || value == 1)) { pp::g_lstm_persist = value; return PP_OK; }
     if (key == 12 && value >= 0 && value <= 2) { pp::g_tile_cluster = value; return PP_OK; }
+    if (key == 13 && (value == 0 || value == 1)) { pp::g_link_identity = value; return PP_OK; }
     return PP_ERR_INVALID_ARG;
 }
 
@@ -384,15 +386,23 @@ pp_status_t pp_pack_create(pp_packed_t** out, int M, int N, int B, const int32_t
         const int frags_per_tile = g.n_rg * g.fpt;
         p->values.assign((size_t)T * B * B * esz, 0);
         const unsigned char* src = static_cast<const unsigned char*>(tile_values);
+        // Entries of a tile on padding rows or padding columns are not part of W (Eq. 1 pads in pivoted
+        // space): they are stored as zero, so that padding rows of the pivoted output are exactly 0 and
+        // whatever sits in the padding columns of a pivoted input never contributes.
+        std::vector<unsigned char> clean((size_t)T * B * B * esz);
         for (int br = 0; br < Mb; ++br) {
             const int r0 = p->row_ptr[(size_t)br], k = p->row_ptr[(size_t)br + 1] - r0;
             for (int j = 0; j < k; ++j) {
                 const unsigned char* tile = src + (size_t)order[(size_t)(r0 + j)] * B * B * esz;
+                unsigned char* ctile = &clean[(size_t)(r0 + j) * B * B * esz];
+                const int bc = p->tile_col[(size_t)p->col_ptr[(size_t)br] + j];
                 for (int r = 0; r < B; ++r)
                     for (int c = 0; c < B; ++c) {
+                        const bool real = row_perm[(int64_t)br * B + r] < M && col_perm[(int64_t)bc * B + c] < N;
+                        if (real) std::memcpy(ctile + ((size_t)r * B + c) * esz, tile + ((size_t)r * B + c) * esz, esz);
                         const ElemPos e = elem_pos(wdtype, g, r, c);
                         const size_t frag = (size_t)r0 * frags_per_tile + ((size_t)e.rg * k + j) * g.fpt + e.f;
-                        std::memcpy(&p->values[frag * 512 + e.byte], tile + ((size_t)r * B + c) * esz, esz);
+                        std::memcpy(&p->values[frag * 512 + e.byte], ctile + ((size_t)r * B + c) * esz, esz);
                     }
             }
         }
@@ -401,8 +411,7 @@ pp_status_t pp_pack_create(pp_packed_t** out, int M, int N, int B, const int32_t
             build_tile_steps(p);
             p->tiles_rm.resize((size_t)T * B * B * 2);   // each tile as its swizzled shared-memory image, in step order
             for (int64_t s2 = 0; s2 < T; ++s2)
-                pp::swizzle_tile_64x64(src + (size_t)order[(size_t)s2] * B * B * 2,
-                                       &p->tiles_rm[(size_t)p->tile_pos[(size_t)s2] * B * B * 2]);
+                pp::swizzle_tile_64x64(&clean[(size_t)s2 * B * B * 2], &p->tiles_rm[(size_t)p->tile_pos[(size_t)s2] * B * B * 2]);
         }
 
         p->gather_idx.resize((size_t)Npad);

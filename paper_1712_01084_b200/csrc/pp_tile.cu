@@ -184,7 +184,7 @@ tile_f16_kernel(const TileArgs a) {
         // after the named barrier below)
         if (b < 64) {
             sm->bias[b] = __ldg(a.bias_piv + br * 64 + b);
-            sm->dst[b] = __ldg(a.scatter_idx + br * 64 + b);
+            sm->dst[b] = a.pivoted ? br * 64 + b : __ldg(a.scatter_idx + br * 64 + b);
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         // the tensor-memory loads below are warp-wide instructions: the whole warp takes one decision
@@ -405,7 +405,7 @@ tile_cluster_f16_kernel(const TileArgs a) {
         if (b < 64) {
             const bool live = br < a.Mb;
             sm->bias[b] = live ? __ldg(a.bias_piv + br * 64 + b) : 0.0f;
-            sm->dst[b] = live ? __ldg(a.scatter_idx + br * 64 + b) : -1;
+            sm->dst[b] = live ? (a.pivoted ? br * 64 + b : __ldg(a.scatter_idx + br * 64 + b)) : -1;
         }
         ok = __all_sync(0xffffffffu, mbar_wait(&sm->acc_full, 0, abort_flag) && !*abort_flag);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");

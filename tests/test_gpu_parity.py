@@ -398,3 +398,105 @@ def test_config5_batch128_tile_path_sampled_rows(pb, tile_kernel):
     y_ref, a = po.dense_forward_rows(W, None, wl.x.astype(np.float64), 0, rows)
     _check(y[:, rows], y_ref, a, np.float16, "config 5 batch 128 sampled")
     L.close()
+
+
+# ------------------------------------------------------------------ permutation elimination (Sections 4.2.2, 4.2.3)
+def _check_pivoted(y_piv, y_ref, a_ref, omap, dtype, what):
+    real = omap >= 0
+    assert np.all(y_piv[:, ~real] == 0.0), f"{what}: padding positions must hold 0"
+    _check(y_piv[:, real], y_ref[:, omap[real]], a_ref[:, omap[real]], dtype, what)
+
+
+@pytest.mark.parametrize("dtype,B", [(np.float32, 32), (np.float16, 16), (np.float16, 64)])
+@pytest.mark.parametrize("batch", [1, 5, 40, 130])
+def test_forward_pivoted_output(pb, dtype, B, batch):
+    """Output permutation elimination (Section 4.2.2): the result left in pivoted row order, relabelled by
+    the map the layer hands out, equals the oracle's; batch 130 with fp16, B = 64 runs the tensor-core
+    kernels.  On integer data the relabelled result has the bits of the ordinary call."""
+    lay = _rand_layer(1200 + B + batch, 5 * B - 3, 9 * B - 7, B, dtype, density=0.45, empty_rows=(2,))
+    x = np.random.default_rng(batch).uniform(-1, 1, (batch, lay.N)).astype(dtype)
+    L = pb.Layer.from_synth(lay)
+    omap = L.output_map()
+    assert omap.shape == (5 * B,) and sorted(omap[omap >= 0].tolist()) == list(range(lay.M))
+    assert np.array_equal(omap, np.where(lay.row_perm < lay.M, lay.row_perm, -1))
+    for kern in ((2, 0) if (dtype == np.float16 and B == 64 and batch >= 64) else (1,)):
+        pb.pp_set_tuning(12, kern)
+        try:
+            for act in (0, 1):
+                y_piv = pb.pp_forward_pivoted(L, _dev(x), act).cpu().numpy()
+                y_ref, _, a = po.layer_forward(lay, x.astype(np.float64), act=act, threads=8)
+                _check_pivoted(y_piv, y_ref, a, omap, dtype, f"pivoted {dtype.__name__} B={B} batch={batch} act={act}")
+        finally:
+            pb.pp_set_tuning(12, 1)
+    L.close()
+    lay = _rand_layer(1300 + B + batch, 4 * B - 1, 6 * B - 5, B, dtype, density=0.5, integer=True)
+    x = np.random.default_rng(5).integers(-2, 3, (batch, lay.N)).astype(dtype)
+    L = pb.Layer.from_synth(lay)
+    omap = L.output_map()
+    y = pb.pp_forward(L, _dev(x), 1).cpu().numpy()
+    y_piv = pb.pp_forward_pivoted(L, _dev(x), 1).cpu().numpy()
+    assert np.array_equal(y_piv[:, omap >= 0], y[:, omap[omap >= 0]])
+    assert L.status() == 0
+    L.close()
+
+
+@pytest.mark.parametrize("dtype,B", [(np.float32, 32), (np.float16, 64)])
+def test_chain_identity_links_and_pivoted_output(pb, dtype, B):
+    """Cross-layer permutation elimination (Section 4.2.3): when the consumer's column permutation equals
+    the producer's row permutation the link is detected as the identity and stored without an index
+    array; same bits as the mapped store, oracle parity, and the final output may stay pivoted
+    (Section 4.2.2).  Link 1 is an identity, link 2 is not (different permutations), link 3 is not
+    (different padded lengths would be needed: here it has an unequal permutation too)."""
+    dims = [7 * B - 5, 6 * B, 5 * B, 4 * B - 3]          # M of layers 0 and 1 are multiples of B: no padding rows
+    lays = []
+    for l in range(3):
+        ll = _rand_layer(1400 + l + B, dims[l + 1], dims[l], B, dtype, density=0.6)
+        ll.act = 1 if l < 2 else 0
+        lays.append(ll)
+    lays[1].col_perm = lays[0].row_perm.copy()           # P^{AB} = I for link 0 -> 1
+    x = np.random.default_rng(9).uniform(-1, 1, (6, dims[0])).astype(dtype)
+    L = [pb.Layer.from_synth(l) for l in lays]
+    chain = pb.Chain(L, [l.act for l in lays], max_batch=8)
+    assert chain.link_info().tolist() == [0, 1, 0]
+    res = po.chain_forward(lays, x.astype(np.float64), round_intermediate="f16" if dtype == np.float16 else "f32",
+                           threads=4)
+    y1 = pb.pp_chain_forward(chain, _dev(x)).cpu().numpy()
+    pb.pp_set_tuning(13, 0)
+    try:
+        y0 = pb.pp_chain_forward(chain, _dev(x)).cpu().numpy()
+    finally:
+        pb.pp_set_tuning(13, 1)
+    assert np.array_equal(y1, y0)
+    bound = _chain_bound(lays, res, TOL[np.dtype(dtype)])
+    worst = np.max(np.abs(y1.astype(np.float64) - res[-1][1]) / bound)
+    assert worst <= 1.0, f"chain with an identity link: worst error/bound {worst:.3f}"
+    chain.set_output_pivoted(True)
+    omap = chain.output_map()
+    yp = pb.pp_chain_forward(chain, _dev(x)).cpu().numpy()
+    assert yp.shape == (6, 4 * B)
+    assert np.array_equal(yp[:, omap >= 0], y1[:, omap[omap >= 0]]) and np.all(yp[:, omap < 0] == 0)
+    chain.set_output_pivoted(False)
+    assert np.array_equal(pb.pp_chain_forward(chain, _dev(x)).cpu().numpy(), y1)
+    chain.close()
+    for l in L:
+        l.close()
+
+
+def test_chain_identity_link_with_padding_rows(pb):
+    """An identity link whose producer has padding rows (M not a multiple of B): the padding rows hold
+    act(0) = 0 and land on the consumer's padding columns."""
+    B, dtype = 16, np.float32
+    dims = [5 * B - 2, 4 * B - 5, 3 * B]
+    lays = [_rand_layer(1500 + l, dims[l + 1], dims[l], B, dtype, density=0.7, integer=True) for l in range(2)]
+    lays[0].act, lays[1].act = 1, 0
+    lays[1].col_perm = lays[0].row_perm.copy()
+    x = np.random.default_rng(2).integers(-2, 3, (3, dims[0])).astype(dtype)
+    L = [pb.Layer.from_synth(l) for l in lays]
+    chain = pb.Chain(L, [1, 0], max_batch=4)
+    assert chain.link_info().tolist() == [0, 1]
+    y = pb.pp_chain_forward(chain, _dev(x)).cpu().numpy()
+    res = po.chain_forward(lays, x.astype(np.float64))
+    assert np.array_equal(y.astype(np.float64), res[-1][1])
+    chain.close()
+    for l in L:
+        l.close()
