@@ -248,15 +248,15 @@ def other_workloads(pb, torch, synth):
         if st != 0:
             raise pb.PPError(st, "forward")
 
-    def layer_case(name, wl, batch):
+    def layer_case(name, wl, batch, pivoted=False):
         lay = wl.layers[0]
         L0 = pb.Layer.from_synth(lay)
         wbytes = lay.T * lay.B * lay.B * lay.tile_values.dtype.itemsize
         R = max(2, -(-2 * L2_BYTES // wbytes) + 1)
         reps = [L0] + [L0.clone() for _ in range(R - 1)]
         x = torch.from_numpy(wl.x).cuda()
-        y = torch.empty((batch, lay.M), dtype=torch.float32, device="cuda")
-        fn = pb.lib().pp_forward
+        y = torch.empty((batch, -(-lay.M // lay.B) * lay.B), dtype=torch.float32, device="cuda")
+        fn = pb.lib().pp_forward_pivoted if pivoted else pb.lib().pp_forward
         cold = time_enqueue(torch, lambda i, sp: check(fn(reps[i % R]._h, x.data_ptr(), y.data_ptr(), batch, lay.act, sp)), R * max(1, 64 // R))
         warm = time_enqueue(torch, lambda i, sp: check(fn(L0._h, x.data_ptr(), y.data_ptr(), batch, lay.act, sp)), 64)
         pk = pb.Packed(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values, lay.bias)
@@ -270,6 +270,9 @@ def other_workloads(pb, torch, synth):
     layer_case("cfg2_fc4096_f32_b64_d12.5_batch1", synth.config2(), 1)
     for batch in (16, 128):
         layer_case(f"cfg5_fc8192_f16_b64_k128_batch{batch}", synth.config5(k=128, batch=batch), batch)
+    # the same product with the output left in pivoted row order (output permutation elimination)
+    layer_case("cfg5_fc8192_f16_b64_k128_batch128_pivoted_output", synth.config5(k=128, batch=128), 128, pivoted=True)
+    layer_case("cfg5_fc8192_f16_b64_k32_batch128", synth.config5(k=32, batch=128), 128)
 
     for batch in (1, 8):
         wl = synth.config3(batch=batch)

@@ -11,7 +11,7 @@
 
 namespace pp {
 int g_use_stream = 1;      // 0: the API never picks the persistent kernel
-int g_tile_min_batch = 64;
+int g_tile_min_batch = 9;
 int g_prepass = 1;
 int g_lstm_persist = 1;
 int g_tile_cluster = 1;

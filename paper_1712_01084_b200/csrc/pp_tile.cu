@@ -1,4 +1,4 @@
-// Batched tile path for sm_100a (fp16 layers with B = 64, batch >= 64): every kept tile is a real
+// Batched tile path for sm_100a (fp16 layers with B = 64, batch > 8): every kept tile is a real
 // dense contraction, so it runs on the 5th-generation tensor cores.
 //
 // Per block-row the kernel accumulates  D[128 x 64] += X_piv_seg[128 x 64] * W_tile^T  over the
@@ -492,8 +492,7 @@ __host__ __device__ __forceinline__ uint32_t sw128_offset(int r, int c) {
     return (uint32_t)r * 128u + (uint32_t)(((c >> 3) ^ (r & 7)) << 4) + (uint32_t)(c & 7) * 2u;
 }
 
-// x_piv[b][j] = x[b][gather_idx[j]] for the rows of one batch chunk; rows past the batch and padding
-// columns are zero.  One CTA per row: the row goes to shared memory coalesced and leaves permuted, into
+// x_piv[b][j] = x[b][gather_idx[j]] for the rows of one batch chunk; padding columns are zero.  One CTA per row: the row goes to shared memory coalesced and leaves permuted, into
 // the swizzled 16 KiB block of its tile-column (row b of the block).
 __global__ void gather_x_kernel(const __half* __restrict__ x, int ldx, int n, const int32_t* __restrict__ gather_idx,
                                 int n_pad, unsigned char* __restrict__ x_sw, int batch) {
@@ -549,7 +548,9 @@ cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const 
         configured = true;
     }
     if ((size_t)n * 2 > 48 * 1024) return cudaErrorInvalidValue;
-    gather_x_kernel<<<kTileBatch, 1024, ((size_t)n * 2 + 15) / 16 * 16, stream>>>(static_cast<const __half*>(x), ldx, n, gather_idx, n_pad,
+    // rows past the batch keep whatever an earlier call left there: every row of the product is independent
+    // and the epilogue drops those rows
+    gather_x_kernel<<<a.batch, 1024, ((size_t)n * 2 + 15) / 16 * 16, stream>>>(static_cast<const __half*>(x), ldx, n, gather_idx, n_pad,
                                                               const_cast<unsigned char*>(a.x_sw), a.batch);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
