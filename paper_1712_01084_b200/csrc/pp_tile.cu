@@ -148,8 +148,11 @@ tile_f16_kernel(const TileArgs a) {
                 const int tt = (t + rot) % k;
                 const int col = __ldg(a.tile_col + cbase + tt);
                 mbar_expect_tx(&sm->full[s], kStageBytes);
-                bulk_load(stages + s * kStageBytes, a.x_sw + (size_t)col * kXBytes, kXBytes, &sm->full[s]);
                 bulk_load(stages + s * kStageBytes + kXBytes, a.tiles_sw + (size_t)__ldg(a.tile_pos + t0 + tt) * kWBytes, kWBytes, &sm->full[s]);
+                // the permuted input comes from the gather kernel launched just before: everything up to here
+                // (set-up, the first weight copies) may overlap its tail
+                if (t == warp) asm volatile("griddepcontrol.wait;" ::: "memory");
+                bulk_load(stages + s * kStageBytes, a.x_sw + (size_t)col * kXBytes, kXBytes, &sm->full[s]);
                 last = t;
             }
             if (*abort_flag) {
@@ -190,7 +193,7 @@ tile_f16_kernel(const TileArgs a) {
         // the tensor-memory loads below are warp-wide instructions: the whole warp takes one decision
         const bool ok = __all_sync(0xffffffffu, mbar_wait(&sm->acc_full, 0, abort_flag) && !*abort_flag);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (ok) {
+        if (ok && q * 32 < a.batch) {
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t r[32];
@@ -348,8 +351,11 @@ tile_cluster_f16_kernel(const TileArgs a) {
                 const TileStep st = load_step(a.steps + p0 + (t + rot) % n_steps);
                 unsigned char* dst = stages + s * kCStageBytes;
                 mbar_expect_tx(&sm->full[s], (uint32_t)(kXBytes + st.ntiles * kWBytes));
-                bulk_load(dst, a.x_sw + (size_t)st.col * kXBytes, kXBytes, &sm->full[s]);
                 bulk_load(dst + kXBytes, a.tiles_sw + (size_t)st.pos * kWBytes, (uint32_t)(st.ntiles * kWBytes), &sm->full[s]);
+                // the permuted input comes from the gather kernel launched just before: everything up to here
+                // (set-up, the first weight copies) may overlap its tail
+                if (t == warp) asm volatile("griddepcontrol.wait;" ::: "memory");
+                bulk_load(dst, a.x_sw + (size_t)st.col * kXBytes, kXBytes, &sm->full[s]);
                 last = t;
             }
             if (*abort_flag && last >= 0) {
@@ -415,7 +421,7 @@ tile_cluster_f16_kernel(const TileArgs a) {
     // Every CTA of the cluster gets here, also one that gave up (the barrier is the hardware's).  Past it
     // no CTA of the cluster reads or fills its stage buffers any more.
     cluster_sync_all();
-    if (epi && ok) {
+    if (epi && ok && q * 32 < a.batch) {          // a warp whose 32 batch rows all lie past the batch has nothing to send
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t mask = sm->acc_mask;
         const uint32_t mine = smem_u32(recv) + (uint32_t)(((int)rank * 16) * kTileBatch + b) * 16u;   // [sender = rank][0][b][0]
@@ -447,7 +453,7 @@ tile_cluster_f16_kernel(const TileArgs a) {
         }
     }
     cluster_sync_all();          // all partials have arrived (release / acquire at cluster scope)
-    if (epi && br < a.Mb && !sm->abort_flag) {
+    if (epi && br < a.Mb && !sm->abort_flag && q * 32 < a.batch) {
         // ---------------- block-row `rank` of the group: add the four partials in sender order, epilogue.
         // Lanes run over the output rows here: one store instruction then writes 32 scattered words of ONE
         // row of y (lanes over batch rows would write words a whole row pitch apart, which all land in the
@@ -497,6 +503,7 @@ __host__ __device__ __forceinline__ uint32_t sw128_offset(int r, int c) {
 __global__ void gather_x_kernel(const __half* __restrict__ x, int ldx, int n, const int32_t* __restrict__ gather_idx,
                                 int n_pad, unsigned char* __restrict__ x_sw, int batch) {
     extern __shared__ __half row[];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the tile kernel may set up meanwhile
     const int b = blockIdx.x;
     if (b < batch) {
         // 16-byte copies where the row allows it (base and pitch 16-byte aligned), element copies otherwise
@@ -537,6 +544,23 @@ void swizzle_tile_64x64(const void* row_major, void* out) {
             for (int k = 0; k < 16; ++k) dst[r * 128 + ((ch ^ (r & 7)) << 4) + k] = src[r * 128 + ch * 16 + k];
 }
 
+// Launch with programmatic stream serialization: the kernel may start while the gather kernel before it
+// still runs; its producers wait for that kernel (griddepcontrol.wait) before they touch the permuted input.
+static cudaError_t launch_after_gather(void (*kernel)(const TileArgs), int grid, int threads, size_t smem, const TileArgs& a,
+                                       cudaStream_t stream) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, a);
+}
+
 cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const int32_t* gather_idx, int n_pad, int Mb,
                         bool use_cluster, cudaStream_t stream) {
     if (a.batch < 1 || a.batch > kTileBatch) return cudaErrorInvalidValue;
@@ -563,11 +587,9 @@ cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const 
             configured_c = true;
         }
         const int groups = (Mb + kTileRows - 1) / kTileRows;
-        tile_cluster_f16_kernel<<<groups * kTileRows, kCThreads, smem_c, stream>>>(a);
-        return cudaGetLastError();
+        return launch_after_gather(tile_cluster_f16_kernel, groups * kTileRows, kCThreads, smem_c, a, stream);
     }
-    tile_f16_kernel<<<Mb, kThreads, smem, stream>>>(a);
-    return cudaGetLastError();
+    return launch_after_gather(tile_f16_kernel, Mb, kThreads, smem, a, stream);
 }
 
 }  // namespace pp
