@@ -25,7 +25,10 @@
  * Pinned by tests/test_oracle_pins.py: a 4x4 example worked by hand, the
  * "cab" index-array convention, brute-force P^T W_piv P products on tiny
  * sizes, identity permutations at density 1 against a library matmul, B = 1
- * against an element-wise sparse sum, and Eq. 2 against Eq. 1.
+ * against an element-wise sparse sum, and Eq. 2 against Eq. 1.  The irregular
+ * block form (ppo_reconstruct_blocks, Section 4.1.5) is pinned by a second 4x4
+ * example worked by hand, by explicit permutation-matrix products on random
+ * rectangles and by its agreement with the uniform-tile form.
  */
 #include <math.h>
 #include <stdint.h>
@@ -80,6 +83,37 @@ int ppo_reconstruct(int M, int N, int B, const int32_t* row_perm, const int32_t*
         }
     }
     return PPO_OK;
+}
+
+/* Eq. 1 with the irregular block structure of Section 4.1.5: M_block holds
+ * rectangles of any size.  Block k covers pivoted rows [r0, r0+h) and pivoted
+ * columns [c0, c0+w) (blocks[4k..4k+3] = r0, c0, h, w); its values follow those
+ * of block k-1 in block_values, row-major h x w.  Blocks may share rows (their
+ * products add up) but no element of M_block belongs to two blocks.  Mp, Np are
+ * the lengths of the index arrays (pivoted sizes, >= M, N). */
+int ppo_reconstruct_blocks(int M, int N, int Mp, int Np, const int32_t* row_perm, const int32_t* col_perm,
+                           const int32_t* blocks, int64_t nb, const double* block_values, double* W) {
+    if (M <= 0 || N <= 0 || Mp < M || Np < N || nb < 0) return PPO_BAD_ARG;
+    if (!is_bijection(row_perm, Mp) || !is_bijection(col_perm, Np)) return PPO_BAD_PERM;
+    unsigned char* taken = (unsigned char*)calloc((size_t)Mp * (size_t)Np, 1);
+    memset(W, 0, sizeof(double) * (size_t)M * (size_t)N);
+    int rc = PPO_OK;
+    int64_t v = 0;
+    for (int64_t k = 0; k < nb && rc == PPO_OK; ++k) {
+        int64_t r0 = blocks[4 * k], c0 = blocks[4 * k + 1], h = blocks[4 * k + 2], w = blocks[4 * k + 3];
+        if (r0 < 0 || c0 < 0 || h <= 0 || w <= 0 || r0 + h > Mp || c0 + w > Np) { rc = PPO_BAD_TILE; break; }
+        for (int64_t r = 0; r < h && rc == PPO_OK; ++r) {
+            for (int64_t c = 0; c < w; ++c, ++v) {
+                int64_t i = r0 + r, j = c0 + c;
+                if (taken[i * Np + j]) { rc = PPO_BAD_TILE; break; }
+                taken[i * Np + j] = 1;
+                int64_t I = row_perm[i], J = col_perm[j];
+                if (I < M && J < N) W[I * N + J] = block_values[v];
+            }
+        }
+    }
+    free(taken);
+    return rc;
 }
 
 static double activate(double s, int act) { return (act == 1 && s < 0.0) ? 0.0 : s; }

@@ -48,6 +48,9 @@ def _load():
         _lib.ppo_reconstruct.restype = ctypes.c_int
         _lib.ppo_reconstruct.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, i32p, i32p, i32p,
                                          ctypes.c_int64, f64p, f64p]
+        _lib.ppo_reconstruct_blocks.restype = ctypes.c_int
+        _lib.ppo_reconstruct_blocks.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, i32p, i32p,
+                                                i32p, ctypes.c_int64, f64p, f64p]
         _lib.ppo_dense_forward.restype = None
         _lib.ppo_dense_forward.argtypes = [ctypes.c_int, ctypes.c_int, f64p, f64p, f64p, ctypes.c_int,
                                            ctypes.c_int, f64p, f64p, f64p, ctypes.c_int]
@@ -92,6 +95,26 @@ def reconstruct(M, N, B, row_perm, col_perm, tile_list, tile_values) -> np.ndarr
         raise OracleError("tile_values has the wrong size")
     W = np.empty((M, N), dtype=np.float64)
     rc = lib.ppo_reconstruct(M, N, B, rpp, cpp, tlp, T, tvp, W.ctypes.data_as(ctypes.POINTER(ctypes.c_double)))
+    if rc:
+        raise OracleError(_ERR.get(rc, str(rc)))
+    return W
+
+
+def reconstruct_blocks(M, N, row_perm, col_perm, blocks, block_values) -> np.ndarray:
+    """Dense W of Eq. 1 when M_block holds rectangles of any size (Section 4.1.5).
+    blocks: [nb][4] = (first pivoted row, first pivoted column, height, width);
+    block_values: the blocks' values one after the other, each row-major.
+    The pivoted sizes are the lengths of the index arrays."""
+    lib = _load()
+    rp, rpp = _i32(row_perm)
+    cp, cpp = _i32(col_perm)
+    bl, blp = _i32(np.asarray(blocks).reshape(-1, 4))
+    bv, bvp = _f64(np.asarray(block_values, dtype=np.float64).reshape(-1))
+    if bv.size != int(np.sum(bl[:, 2].astype(np.int64) * bl[:, 3])):
+        raise OracleError("block_values has the wrong size")
+    W = np.empty((M, N), dtype=np.float64)
+    rc = lib.ppo_reconstruct_blocks(M, N, rp.size, cp.size, rpp, cpp, blp, bl.shape[0], bvp,
+                                    W.ctypes.data_as(ctypes.POINTER(ctypes.c_double)))
     if rc:
         raise OracleError(_ERR.get(rc, str(rc)))
     return W

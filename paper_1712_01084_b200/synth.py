@@ -218,6 +218,95 @@ def config5(k: int = 128, batch: int = 1, scale: float = 1.0, **kw) -> Workload:
     return Workload(f"cfg5_fc8192_f16_b64_k{k}", [lay], x)
 
 
+# --------------------------------------------------------------------------- #
+# Irregular block structure (Section 4.1.5): W_piv holds rectangles of any size.
+# --------------------------------------------------------------------------- #
+
+@dataclass
+class BlockLayer:
+    M: int
+    N: int
+    B: int                        # grid the library lays the blocks over; fixes the padded sizes
+    row_perm: np.ndarray          # int32 [ceil(M/B)*B]
+    col_perm: np.ndarray          # int32 [ceil(N/B)*B]
+    blocks: np.ndarray            # int32 [nb, 4] = first pivoted row, first pivoted column, height, width
+    block_values: np.ndarray      # float32 or float16, the blocks one after the other, each row-major
+    bias: Optional[np.ndarray]
+    act: int = ACT_IDENTITY
+    seed: int = 0
+
+    @property
+    def wdtype(self) -> str:
+        return "f16" if self.block_values.dtype == np.float16 else "f32"
+
+    @property
+    def block_bytes(self) -> int:
+        return int(self.block_values.size * self.block_values.dtype.itemsize)
+
+
+def _block_values(rng, blocks, N, wdtype, integer_values):
+    n = int(np.sum(blocks[:, 2].astype(np.int64) * blocks[:, 3])) if len(blocks) else 0
+    if integer_values:
+        v = rng.integers(-4, 5, size=n).astype(np.float32)
+    else:
+        v = (rng.standard_normal(n) / np.sqrt(N)).astype(np.float32)
+    return v.astype(np.float16) if wdtype == "f16" else v
+
+
+def paper_square(size: int, blocks_per_side: int, B: int, *, wdtype: str = "f32", batch: int = 1,
+                 integer_values: bool = False, seed: Optional[int] = None) -> Workload:
+    """The geometry the paper measures (Section 5): a size x size matrix with
+    ``blocks_per_side`` identical square blocks of edge size/blocks_per_side on the
+    diagonal of the pivoted matrix (fill-in = 1/blocks_per_side), random index arrays,
+    x ~ U(-1, 1), no bias."""
+    edge = size // blocks_per_side
+    if edge * blocks_per_side != size:
+        raise ValueError("size must be a multiple of blocks_per_side")
+    seed = _seed(6, 0) + size + blocks_per_side if seed is None else seed
+    rng = np.random.default_rng(seed)
+    pad = -(-size // B) * B
+    row_perm = rng.permutation(pad).astype(np.int32)
+    col_perm = rng.permutation(pad).astype(np.int32)
+    blocks = np.array([[k * edge, k * edge, edge, edge] for k in range(blocks_per_side)], dtype=np.int32)
+    vals = _block_values(rng, blocks, size, wdtype, integer_values)
+    lay = BlockLayer(size, size, B, row_perm, col_perm, blocks, vals, None, ACT_IDENTITY, seed)
+    x = draw_x(rng, batch, size, -1.0, 1.0, wdtype, integer_values)
+    return Workload(f"paper_square_{size}_fill{100.0 / blocks_per_side:g}_{wdtype}_grid{B}", [lay], x)
+
+
+def irregular_blocks(seed: int, M: int, N: int, B: int, *, wdtype: str, n_row_cuts: int, n_col_cuts: int,
+                     keep: float, batch: int = 1, bias_std: Optional[float] = None, act: int = ACT_IDENTITY,
+                     integer_values: bool = False, aligned: bool = False) -> Workload:
+    """Rectangles of mixed sizes: random cut lines split the padded pivoted matrix into a grid of
+    unequal cells and a random fraction ``keep`` of the cells become blocks (so blocks differ in height
+    and width, several share their rows, none overlap).  ``aligned`` puts the cuts on multiples of B."""
+    rng = np.random.default_rng(seed)
+    Mp, Np = -(-M // B) * B, -(-N // B) * B
+    row_perm = rng.permutation(Mp).astype(np.int32)
+    col_perm = rng.permutation(Np).astype(np.int32)
+
+    def cuts(n, length):
+        if aligned:
+            inner = rng.choice(np.arange(1, length // B), size=min(n, length // B - 1), replace=False) * B
+        else:
+            inner = rng.choice(np.arange(1, length), size=min(n, length - 1), replace=False)
+        return np.concatenate([[0], np.sort(inner), [length]]).astype(np.int64)
+
+    rc, cc = cuts(n_row_cuts, Mp), cuts(n_col_cuts, Np)
+    cells = [(i, j) for i in range(len(rc) - 1) for j in range(len(cc) - 1)]
+    chosen = rng.permutation(len(cells))[:max(1, int(round(keep * len(cells))))]
+    blocks = np.array([[rc[cells[c][0]], cc[cells[c][1]], rc[cells[c][0] + 1] - rc[cells[c][0]],
+                        cc[cells[c][1] + 1] - cc[cells[c][1]]] for c in chosen], dtype=np.int32)
+    vals = _block_values(rng, blocks, N, wdtype, integer_values)
+    bias = None
+    if bias_std is not None:
+        bias = rng.integers(-8, 9, size=M).astype(np.float32) if integer_values else \
+            (rng.standard_normal(M) * bias_std).astype(np.float32)
+    lay = BlockLayer(M, N, B, row_perm, col_perm, blocks, vals, bias, act, seed)
+    x = draw_x(rng, batch, N, -1.0, 1.0, wdtype, integer_values)
+    return Workload(f"irregular_{M}x{N}_{wdtype}_grid{B}", [lay], x)
+
+
 # The 4 x 4 example worked by hand (values are part of the test fixtures, not drawn).
 def hand_example() -> Layer:
     return Layer(

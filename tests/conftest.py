@@ -28,3 +28,8 @@ def load_golden(name):
 @pytest.fixture(scope="session")
 def hand4():
     return load_golden("hand_4x4.txt")
+
+
+@pytest.fixture(scope="session")
+def hand_blocks4():
+    return load_golden("hand_blocks_4x4.txt")

@@ -280,3 +280,95 @@ def test_lstm_zero_weights_and_recurrence_wiring():
     h1_unit1 = np.tanh(np.tanh(0.5))
     np.testing.assert_allclose(hs[0, 1], h1_unit1, atol=1e-12)
     np.testing.assert_allclose(hs[1, 0], np.tanh(np.tanh(2.0 * h1_unit1)), atol=1e-12)
+
+
+# ------------------------------------------------ irregular block structure (Section 4.1.5)
+def test_hand_blocks_4x4(hand_blocks4):
+    g = hand_blocks4
+    rp = np.array(g["row_perm"], dtype=np.int32)
+    cp = np.array(g["col_perm"], dtype=np.int32)
+    W = po.reconstruct_blocks(4, 4, rp, cp, np.array(g["blocks"], dtype=np.int32).reshape(-1, 4), g["block_values"])
+    assert np.array_equal(W, np.array(g["W"]).reshape(4, 4))
+    y, s, a = po.dense_forward(W, None, np.array(g["x"]), act=0)
+    assert np.array_equal(y[0], g["Wx"])
+    assert np.array_equal(a[0], g["absW_absx"])
+
+
+def _dense_from_blocks(Mp, Np, blocks, values):
+    """W_piv assembled by array slicing (not by the oracle's element loop)."""
+    Wp = np.zeros((Mp, Np))
+    cover = np.zeros((Mp, Np), dtype=np.int64)
+    off = 0
+    for r0, c0, h, w in blocks:
+        Wp[r0:r0 + h, c0:c0 + w] = np.asarray(values[off:off + h * w], dtype=np.float64).reshape(h, w)
+        cover[r0:r0 + h, c0:c0 + w] += 1
+        off += h * w
+    return Wp, cover
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_blocks_against_permutation_matrices(seed):
+    """Random rectangles (unaligned, several per row): Eq. 1 with explicit 0/1 matrices, W = P_r^T W_piv P_c."""
+    rng = np.random.default_rng(seed)
+    B = int(rng.choice([1, 2, 3, 4]))
+    M, N = int(rng.integers(3, 13)), int(rng.integers(3, 13))
+    wl = synth.irregular_blocks(900 + seed, M, N, B, wdtype="f32", n_row_cuts=3, n_col_cuts=3, keep=0.5,
+                                integer_values=True)
+    lay = wl.layers[0]
+    Mp, Np = lay.row_perm.size, lay.col_perm.size
+    Wp, cover = _dense_from_blocks(Mp, Np, lay.blocks, lay.block_values)
+    assert cover.max() == 1
+    Pr = np.zeros((Mp, Mp)); Pr[np.arange(Mp), lay.row_perm] = 1.0
+    Pc = np.zeros((Np, Np)); Pc[np.arange(Np), lay.col_perm] = 1.0
+    W_full = Pr.T @ Wp @ Pc
+    W = po.reconstruct_blocks(M, N, lay.row_perm, lay.col_perm, lay.blocks, lay.block_values)
+    assert np.array_equal(W, W_full[:M, :N])
+
+
+def test_blocks_equal_tiles_when_uniform():
+    """Blocks that are exactly the tiles of a uniform layer give the same W as the tile form."""
+    lay = synth.config1(scale=0.25).layers[0]
+    B = lay.B
+    blocks = np.array([[br * B, bc * B, B, B] for br, bc in lay.tile_list], dtype=np.int32)
+    W_b = po.reconstruct_blocks(lay.M, lay.N, lay.row_perm, lay.col_perm, blocks, lay.tile_values.reshape(-1))
+    W_t = po.reconstruct(lay.M, lay.N, B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values)
+    assert np.array_equal(W_b, W_t)
+
+
+def test_blocks_split_and_order_invariance():
+    """Cutting a block in two, or listing the blocks in another order, changes nothing."""
+    wl = synth.irregular_blocks(77, 40, 56, 8, wdtype="f32", n_row_cuts=4, n_col_cuts=5, keep=0.6)
+    lay = wl.layers[0]
+    W = po.reconstruct_blocks(lay.M, lay.N, lay.row_perm, lay.col_perm, lay.blocks, lay.block_values)
+    blocks2, vals2 = [], []
+    offs = np.concatenate([[0], np.cumsum(lay.blocks[:, 2].astype(np.int64) * lay.blocks[:, 3])])
+    for k in range(len(lay.blocks) - 1, -1, -1):
+        r0, c0, h, w = (int(v) for v in lay.blocks[k])
+        v = lay.block_values[offs[k]:offs[k + 1]].reshape(h, w)
+        if w >= 2:
+            blocks2 += [[r0, c0, h, w // 2], [r0, c0 + w // 2, h, w - w // 2]]
+            vals2 += [v[:, :w // 2].ravel(), v[:, w // 2:].ravel()]
+        else:
+            blocks2.append([r0, c0, h, w]); vals2.append(v.ravel())
+    W2 = po.reconstruct_blocks(lay.M, lay.N, lay.row_perm, lay.col_perm, np.array(blocks2, dtype=np.int32),
+                               np.concatenate(vals2))
+    assert np.array_equal(W, W2)
+
+
+def test_blocks_rejects_overlap_and_range():
+    rp = np.arange(8, dtype=np.int32)
+    with pytest.raises(po.OracleError):
+        po.reconstruct_blocks(8, 8, rp, rp, [[0, 0, 4, 4], [3, 3, 2, 2]], np.zeros(20))
+    with pytest.raises(po.OracleError):
+        po.reconstruct_blocks(8, 8, rp, rp, [[6, 0, 4, 4]], np.zeros(16))
+
+
+def test_paper_square_geometry():
+    """Section 5's example: size 512 at fill-in 6.25 % is 16 identical 32 x 32 blocks, one per block-row."""
+    lay = synth.paper_square(512, 16, 32).layers[0]
+    assert lay.blocks.shape == (16, 4)
+    assert np.all(lay.blocks[:, 2] == 32) and np.all(lay.blocks[:, 3] == 32)
+    assert len(set(lay.blocks[:, 0])) == 16 and len(set(lay.blocks[:, 1])) == 16
+    W = po.reconstruct_blocks(512, 512, lay.row_perm, lay.col_perm, lay.blocks, lay.block_values)
+    assert np.count_nonzero(W) == 16 * 32 * 32
+    assert np.all(np.count_nonzero(W, axis=1) == 32) and np.all(np.count_nonzero(W, axis=0) == 32)
