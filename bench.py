@@ -274,6 +274,34 @@ def other_workloads(pb, torch, synth):
     layer_case("cfg5_fc8192_f16_b64_k128_batch128_pivoted_output", synth.config5(k=128, batch=128), 128, pivoted=True)
     layer_case("cfg5_fc8192_f16_b64_k32_batch128", synth.config5(k=32, batch=128), 128)
 
+    # The geometry the paper itself measures (Section 5): size x size, 1/fill-in square blocks on the diagonal of
+    # the pivoted matrix, batch 1, here fp32.  Blocks go through pp_layer_create_blocks (grid = block edge clamped
+    # to 16..64).  "warm" repeats one layer as the paper's 2,500-call average does; "cold" rotates copies
+    # that together exceed twice the L2 (given where at most 96 copies do).
+    geo = {}
+    for size in (64, 128, 256, 512, 1024, 2048, 4096):
+        for per_side in (32, 16, 8, 4):
+            edge = size // per_side
+            grid = 16 if edge <= 16 else 32 if edge <= 32 else 64
+            wl = synth.paper_square(size, per_side, grid, wdtype="f32")
+            lay = wl.layers[0]
+            L0 = pb.Layer.from_synth(lay)
+            x = torch.from_numpy(wl.x).cuda()
+            y = torch.empty((1, size), dtype=torch.float32, device="cuda")
+            fn = pb.lib().pp_forward
+            warm = time_enqueue(torch, lambda i, sp: check(fn(L0._h, x.data_ptr(), y.data_ptr(), 1, 0, sp)), 64)
+            row = {"block_edge": edge, "grid": grid, "block_bytes": lay.block_bytes, "us_warm": round(warm, 3)}
+            R = -(-2 * L2_BYTES // max(1, lay.block_bytes)) + 1
+            if R <= 96:
+                reps = [L0] + [L0.clone() for _ in range(R - 1)]
+                cold = time_enqueue(torch, lambda i, sp: check(fn(reps[i % R]._h, x.data_ptr(), y.data_ptr(), 1, 0, sp)), R)
+                row.update({"us_cold": round(cold, 3), "GBps_cold": round(lay.block_bytes / cold / 1e3, 1), "copies": R})
+                for r in reps[1:]:
+                    r.close()
+            L0.close()
+            geo[f"size{size}_fill{100.0 / per_side:g}"] = row
+    out["paper_geometry_f32_batch1"] = geo
+
     for batch in (1, 8):
         wl = synth.config3(batch=batch)
         wbytes = sum(l.T * l.B * l.B * 2 for l in wl.layers)

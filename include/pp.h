@@ -141,6 +141,50 @@ pp_status_t pp_layer_create(pp_layer_t** out, int M, int N, int B,
                             const float* bias);
 pp_status_t pp_layer_destroy(pp_layer_t* layer);
 
+/* ------------------------------------------------------------------------- *
+ * Irregular block structure (Section 4.1.5: blocks of different sizes, given to
+ * the kernel through a table of block shapes; blocks that share rows need one
+ * more reduction step).  W_piv holds n_blocks dense rectangles of any height,
+ * width and position instead of tiles on a B x B grid.  This includes the
+ * geometry the paper measures (Section 5: a size x size matrix with 1/fill-in
+ * square blocks of edge size * fill-in, one per block-row).
+ *
+ * The rectangles are laid over the grid of B x B tiles the kernels work on:
+ * every tile a block touches is kept, tile elements no block covers are zero,
+ * and the products of tiles that share a block-row add up, which is that
+ * reduction step.  So blocks whose edges are multiples of B and that start on
+ * multiples of B cost exactly their own bytes; other shapes are padded to the grid.
+ *
+ * blocks        host, int32[n_blocks][4] = (first pivoted row, first pivoted
+ *               column, height, width); 0 <= row, row + height <= M_pad (same for
+ *               columns); height, width > 0; no element in two blocks
+ * block_values  host, the blocks' values one block after the other, each
+ *               row-major height x width, element type wdtype
+ * M, N, B, row_perm, col_perm, wdtype, bias   as pp_pack_create
+ *
+ * pp_blocks_to_tiles is the host-side conversion on its own: *T_out receives the
+ * number of tiles touched; with tile_list_out == tile_values_out == NULL it only
+ * counts, otherwise it writes the tiles sorted by (block-row, block-column) into
+ * tile_list_out (int32[T][2]) and tile_values_out ([T][B][B], wdtype), which
+ * must hold capacity_tiles >= T tiles.  pp_pack_create_blocks and
+ * pp_layer_create_blocks convert and then behave as pp_pack_create /
+ * pp_layer_create.  Errors: PP_ERR_BAD_TILE for a block outside the padded
+ * matrix, of non-positive size, or overlapping another; else as pp_pack_create.
+ * ------------------------------------------------------------------------- */
+pp_status_t pp_blocks_to_tiles(int M, int N, int B, const int32_t* blocks, int64_t n_blocks,
+                               const void* block_values, pp_dtype_t wdtype, int64_t* T_out,
+                               int32_t* tile_list_out, void* tile_values_out, int64_t capacity_tiles);
+pp_status_t pp_pack_create_blocks(pp_packed_t** out, int M, int N, int B,
+                                  const int32_t* row_perm, const int32_t* col_perm,
+                                  const int32_t* blocks, int64_t n_blocks,
+                                  const void* block_values, pp_dtype_t wdtype,
+                                  const float* bias);
+pp_status_t pp_layer_create_blocks(pp_layer_t** out, int M, int N, int B,
+                                   const int32_t* row_perm, const int32_t* col_perm,
+                                   const int32_t* blocks, int64_t n_blocks,
+                                   const void* block_values, pp_dtype_t wdtype,
+                                   const float* bias);
+
 /* Raised by a kernel whose bounded device-side wait gave up (the call's output is then invalid).
  * Synchronises with the device; *status is PP_OK or PP_ERR_TIMEOUT.  The flag is cleared by the read. */
 pp_status_t pp_layer_status(pp_layer_t* layer, pp_status_t* status);

@@ -51,6 +51,9 @@ def lib() -> ctypes.CDLL:
         "pp_status_string": (ctypes.c_char_p, [ci]),
         "pp_pack_create": (ci, create_args),
         "pp_pack_destroy": (ci, [vp]),
+        "pp_blocks_to_tiles": (ci, [ci, ci, ci, i32p, c64, vp, ci, i64p, i32p, vp, c64]),
+        "pp_pack_create_blocks": (ci, create_args),
+        "pp_layer_create_blocks": (ci, create_args),
         "pp_pack_info": (ci, [vp, i64p]),
         "pp_pack_get": (ci, [vp, ci, vp, c64]),
         "pp_pack_unpack": (ci, [vp, i32p, vp]),
@@ -118,6 +121,50 @@ def _layer_args(M, N, B, row_perm, col_perm, tile_list, tile_values, bias):
     return keep, (int(M), int(N), int(B), rpp, cpp, tlp, T, tv.ctypes.data_as(ctypes.c_void_p), wd, bp)
 
 
+def _block_args(M, N, B, row_perm, col_perm, blocks, block_values, bias):
+    rp, rpp = _i32(row_perm)
+    cp, cpp = _i32(col_perm)
+    bl, blp = _i32(np.asarray(blocks).reshape(-1, 4))
+    bv = np.ascontiguousarray(block_values).reshape(-1)
+    if bv.dtype == np.float16:
+        wd = PP_F16
+    elif bv.dtype == np.float32:
+        wd = PP_F32
+    else:
+        raise TypeError("block_values must be float32 or float16")
+    if bv.size != int(np.sum(bl[:, 2].astype(np.int64) * bl[:, 3])):
+        raise ValueError("block_values must hold sum(height*width) elements")
+    if rp.size != -(-M // B) * B or cp.size != -(-N // B) * B:
+        raise ValueError("row_perm/col_perm must cover the padded ranges")
+    b = None if bias is None else np.ascontiguousarray(bias, dtype=np.float32)
+    if b is not None and b.size != M:
+        raise ValueError("bias must have M entries")
+    bp = None if b is None else b.ctypes.data_as(ctypes.POINTER(ctypes.c_float))
+    keep = (rp, cp, bl, bv, b)
+    return keep, (int(M), int(N), int(B), rpp, cpp, blp, bl.shape[0], bv.ctypes.data_as(ctypes.c_void_p), wd, bp)
+
+
+def pp_blocks_to_tiles(M, N, B, blocks, block_values):
+    """Lay irregular blocks over the B x B tile grid (pp_blocks_to_tiles): (tile_list [T,2], tile_values [T,B,B])."""
+    bl, blp = _i32(np.asarray(blocks).reshape(-1, 4))
+    bv = np.ascontiguousarray(block_values).reshape(-1)
+    wd = PP_F16 if bv.dtype == np.float16 else PP_F32
+    if bv.dtype not in (np.float16, np.float32):
+        raise TypeError("block_values must be float32 or float16")
+    if bv.size != int(np.sum(bl[:, 2].astype(np.int64) * bl[:, 3])):
+        raise ValueError("block_values must hold sum(height*width) elements")
+    T = ctypes.c_int64(0)
+    bvp = bv.ctypes.data_as(ctypes.c_void_p)
+    _check(lib().pp_blocks_to_tiles(int(M), int(N), int(B), blp, bl.shape[0], bvp, wd, ctypes.byref(T), None, None, 0),
+           "pp_blocks_to_tiles")
+    tl = np.zeros((T.value, 2), dtype=np.int32)
+    tv = np.zeros((T.value, B, B), dtype=bv.dtype)
+    _check(lib().pp_blocks_to_tiles(int(M), int(N), int(B), blp, bl.shape[0], bvp, wd, ctypes.byref(T),
+                                    tl.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), tv.ctypes.data_as(ctypes.c_void_p),
+                                    T.value), "pp_blocks_to_tiles")
+    return tl, tv
+
+
 # ---------------------------------------------------------------- host packer
 class Packed:
     """Host-side packed layer (pp_pack_create); needs no GPU."""
@@ -126,8 +173,21 @@ class Packed:
         keep, args = _layer_args(M, N, B, row_perm, col_perm, tile_list, tile_values, bias)
         self._h = ctypes.c_void_p()
         _check(lib().pp_pack_create(ctypes.byref(self._h), *args), "pp_pack_create")
+        self._finish(M, N, B, np.asarray(tile_values).dtype)
+
+    @classmethod
+    def from_blocks(cls, M, N, B, row_perm, col_perm, blocks, block_values, bias=None) -> "Packed":
+        """Packed layer from irregular blocks (pp_pack_create_blocks)."""
+        keep, args = _block_args(M, N, B, row_perm, col_perm, blocks, block_values, bias)
+        self = object.__new__(cls)
+        self._h = ctypes.c_void_p()
+        _check(lib().pp_pack_create_blocks(ctypes.byref(self._h), *args), "pp_pack_create_blocks")
+        self._finish(M, N, B, np.asarray(block_values).dtype)
+        return self
+
+    def _finish(self, M, N, B, wdtype):
         self.M, self.N, self.B = int(M), int(N), int(B)
-        self.wdtype = np.asarray(tile_values).dtype
+        self.wdtype = wdtype
         info = (ctypes.c_int64 * 13)()
         _check(lib().pp_pack_info(self._h, info), "pp_pack_info")
         (self.Mb, self.Nb, self.T, self.n_tile_col, self.n_items, self.value_bytes,
@@ -220,7 +280,20 @@ class Layer:
 
     @classmethod
     def from_synth(cls, lay):
+        if hasattr(lay, "blocks"):
+            return cls.from_blocks(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.blocks, lay.block_values, lay.bias)
         return cls(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values, lay.bias)
+
+    @classmethod
+    def from_blocks(cls, M, N, B, row_perm, col_perm, blocks, block_values, bias=None) -> "Layer":
+        """Layer whose W_piv holds rectangles of any size and position (pp_layer_create_blocks)."""
+        keep, args = _block_args(M, N, B, row_perm, col_perm, blocks, block_values, bias)
+        self = object.__new__(cls)
+        self._h = ctypes.c_void_p()
+        _check(lib().pp_layer_create_blocks(ctypes.byref(self._h), *args), "pp_layer_create_blocks")
+        self.M, self.N, self.B = int(M), int(N), int(B)
+        self.wdtype = np.asarray(block_values).dtype
+        return self
 
     def clone(self) -> "Layer":
         other = object.__new__(Layer)
@@ -258,6 +331,10 @@ class Layer:
 
 def pp_layer_create(M, N, B, row_perm, col_perm, tile_list, tile_values, bias=None) -> Layer:
     return Layer(M, N, B, row_perm, col_perm, tile_list, tile_values, bias)
+
+
+def pp_layer_create_blocks(M, N, B, row_perm, col_perm, blocks, block_values, bias=None) -> Layer:
+    return Layer.from_blocks(M, N, B, row_perm, col_perm, blocks, block_values, bias)
 
 
 def _check_x(x, N, wdtype):

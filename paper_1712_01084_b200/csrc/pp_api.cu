@@ -337,6 +337,11 @@ pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx
 
 }  // namespace
 
+namespace {
+// Uploads a packed layer to the current device; takes ownership of pk (freed on failure).
+pp_status_t layer_from_pack(pp_layer_t** out, pp_packed* pk);
+}
+
 extern "C" {
 
 pp_status_t pp_layer_create(pp_layer_t** out, int M, int N, int B, const int32_t* row_perm,
@@ -347,6 +352,26 @@ pp_status_t pp_layer_create(pp_layer_t** out, int M, int N, int B, const int32_t
     pp_packed* pk = nullptr;
     pp_status_t st = pp_pack_create(&pk, M, N, B, row_perm, col_perm, tile_list, T, tile_values, wdtype, bias);
     if (st != PP_OK) return st;
+    return layer_from_pack(out, pk);
+}
+
+pp_status_t pp_layer_create_blocks(pp_layer_t** out, int M, int N, int B, const int32_t* row_perm,
+                                   const int32_t* col_perm, const int32_t* blocks, int64_t n_blocks,
+                                   const void* block_values, pp_dtype_t wdtype, const float* bias) {
+    if (!out) return PP_ERR_INVALID_ARG;
+    *out = nullptr;
+    pp_packed* pk = nullptr;
+    pp_status_t st = pp_pack_create_blocks(&pk, M, N, B, row_perm, col_perm, blocks, n_blocks, block_values, wdtype, bias);
+    if (st != PP_OK) return st;
+    return layer_from_pack(out, pk);
+}
+
+}  // extern "C"
+
+namespace {
+pp_status_t layer_from_pack(pp_layer_t** out, pp_packed* pk) {
+    const pp_dtype_t wdtype = pk->wdtype;
+    const int B = pk->B;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { pp_pack_destroy(pk); cudaGetLastError(); return PP_ERR_CUDA; }
     pp_layer* L = new (std::nothrow) pp_layer();
@@ -384,6 +409,9 @@ pp_status_t pp_layer_create(pp_layer_t** out, int M, int N, int B, const int32_t
     *out = L;
     return PP_OK;
 }
+}  // namespace
+
+extern "C" {
 
 pp_status_t pp_layer_clone(pp_layer_t** out, const pp_layer_t* src) {
     if (!out) return PP_ERR_INVALID_ARG;

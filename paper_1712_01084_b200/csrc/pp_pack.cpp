@@ -437,6 +437,82 @@ pp_status_t pp_pack_create(pp_packed_t** out, int M, int N, int B, const int32_t
     return PP_OK;
 }
 
+// Irregular block structure (Section 4.1.5): blocks of any size and position are laid over the
+// grid of B x B tiles the kernels work on.  Every tile a block touches is kept; the part of a tile no
+// block covers is zero.  Several blocks may meet in one tile, but no element may belong to two.
+pp_status_t pp_blocks_to_tiles(int M, int N, int B, const int32_t* blocks, int64_t n_blocks,
+                               const void* block_values, pp_dtype_t wdtype, int64_t* T_out,
+                               int32_t* tile_list_out, void* tile_values_out, int64_t capacity_tiles) {
+    if (!T_out || M <= 0 || N <= 0 || B <= 0 || n_blocks < 0) return PP_ERR_INVALID_ARG;
+    if (n_blocks > 0 && (!blocks || !block_values)) return PP_ERR_INVALID_ARG;
+    if (wdtype != PP_F32 && wdtype != PP_F16) return PP_ERR_INVALID_ARG;
+    const int64_t Mb = ((int64_t)M + B - 1) / B, Nb = ((int64_t)N + B - 1) / B;
+    const int64_t Mpad = Mb * B, Npad = Nb * B;
+    const size_t esz = wdtype == PP_F16 ? 2 : 4;
+    try {
+        std::vector<int64_t> keys;
+        for (int64_t k = 0; k < n_blocks; ++k) {
+            const int64_t r0 = blocks[4 * k], c0 = blocks[4 * k + 1], h = blocks[4 * k + 2], w = blocks[4 * k + 3];
+            if (r0 < 0 || c0 < 0 || h <= 0 || w <= 0 || r0 + h > Mpad || c0 + w > Npad) return PP_ERR_BAD_TILE;
+            for (int64_t br = r0 / B; br <= (r0 + h - 1) / B; ++br)
+                for (int64_t bc = c0 / B; bc <= (c0 + w - 1) / B; ++bc) keys.push_back(br * Nb + bc);
+        }
+        std::sort(keys.begin(), keys.end());
+        keys.erase(std::unique(keys.begin(), keys.end()), keys.end());
+        const int64_t T = (int64_t)keys.size();
+        *T_out = T;
+        if (!tile_list_out && !tile_values_out) return PP_OK;          // count only
+        if (!tile_list_out || !tile_values_out || capacity_tiles < T) return PP_ERR_INVALID_ARG;
+        for (int64_t t = 0; t < T; ++t) {
+            tile_list_out[2 * t] = (int32_t)(keys[(size_t)t] / Nb);
+            tile_list_out[2 * t + 1] = (int32_t)(keys[(size_t)t] % Nb);
+        }
+        const size_t tile_elems = (size_t)B * B;
+        unsigned char* dst = static_cast<unsigned char*>(tile_values_out);
+        std::memset(dst, 0, (size_t)T * tile_elems * esz);
+        std::vector<unsigned char> taken((size_t)T * tile_elems, 0);
+        const unsigned char* src = static_cast<const unsigned char*>(block_values);
+        for (int64_t k = 0; k < n_blocks; ++k) {
+            const int64_t r0 = blocks[4 * k], c0 = blocks[4 * k + 1], h = blocks[4 * k + 2], w = blocks[4 * k + 3];
+            for (int64_t r = 0; r < h; ++r) {
+                const int64_t i = r0 + r;
+                for (int64_t c = 0; c < w; ++c, src += esz) {
+                    const int64_t j = c0 + c;
+                    const int64_t key = (i / B) * Nb + j / B;
+                    const size_t t = (size_t)(std::lower_bound(keys.begin(), keys.end(), key) - keys.begin());
+                    const size_t e = t * tile_elems + (size_t)(i % B) * B + (size_t)(j % B);
+                    if (taken[e]) return PP_ERR_BAD_TILE;               // two blocks overlap
+                    taken[e] = 1;
+                    std::memcpy(dst + e * esz, src, esz);
+                }
+            }
+        }
+    } catch (const std::bad_alloc&) {
+        return PP_ERR_ALLOC;
+    }
+    return PP_OK;
+}
+
+pp_status_t pp_pack_create_blocks(pp_packed_t** out, int M, int N, int B, const int32_t* row_perm,
+                                  const int32_t* col_perm, const int32_t* blocks, int64_t n_blocks,
+                                  const void* block_values, pp_dtype_t wdtype, const float* bias) {
+    if (!out) return PP_ERR_INVALID_ARG;
+    *out = nullptr;
+    int64_t T = 0;
+    pp_status_t st = pp_blocks_to_tiles(M, N, B, blocks, n_blocks, block_values, wdtype, &T, nullptr, nullptr, 0);
+    if (st != PP_OK) return st;
+    try {
+        std::vector<int32_t> tile_list((size_t)T * 2 + 2);
+        std::vector<unsigned char> tile_values((size_t)T * B * B * (wdtype == PP_F16 ? 2 : 4) + 16);
+        st = pp_blocks_to_tiles(M, N, B, blocks, n_blocks, block_values, wdtype, &T, tile_list.data(),
+                                tile_values.data(), T);
+        if (st != PP_OK) return st;
+        return pp_pack_create(out, M, N, B, row_perm, col_perm, tile_list.data(), T, tile_values.data(), wdtype, bias);
+    } catch (const std::bad_alloc&) {
+        return PP_ERR_ALLOC;
+    }
+}
+
 pp_status_t pp_pack_destroy(pp_packed_t* p) {
     delete p;
     return PP_OK;

@@ -457,3 +457,65 @@ def test_clustered_tile_plan_covers_every_tile_once():
                     nxt += 1
         assert nxt == pk.T
         pk.close()
+
+
+# ------------------------------------------------ irregular block structure (Section 4.1.5)
+def _numpy_tiles(Mp, Np, B, blocks, values):
+    """The tile form of a set of blocks by array slicing: dense W_piv, then the tiles any block touches."""
+    Wp = np.zeros((Mp, Np), dtype=values.dtype)
+    touched = np.zeros((Mp // B, Np // B), dtype=bool)
+    off = 0
+    for r0, c0, h, w in blocks:
+        Wp[r0:r0 + h, c0:c0 + w] = values[off:off + h * w].reshape(h, w)
+        touched[r0 // B:(r0 + h - 1) // B + 1, c0 // B:(c0 + w - 1) // B + 1] = True
+        off += h * w
+    tl = np.argwhere(touched).astype(np.int32)
+    tv = np.stack([Wp[br * B:(br + 1) * B, bc * B:(bc + 1) * B] for br, bc in tl]) if len(tl) else \
+        np.zeros((0, B, B), dtype=values.dtype)
+    return tl, tv
+
+
+@pytest.mark.parametrize("dtype", ["f32", "f16"])
+@pytest.mark.parametrize("B,aligned", [(16, False), (32, False), (64, True), (16, True)])
+def test_blocks_to_tiles_bit_exact(dtype, B, aligned):
+    wl = synth.irregular_blocks(300 + B, 5 * B - 5, 7 * B - 9, B, wdtype=dtype, n_row_cuts=4, n_col_cuts=5,
+                                keep=0.5, aligned=aligned)
+    lay = wl.layers[0]
+    tl, tv = pb.pp_blocks_to_tiles(lay.M, lay.N, B, lay.blocks, lay.block_values)
+    tl_ref, tv_ref = _numpy_tiles(lay.row_perm.size, lay.col_perm.size, B, lay.blocks, lay.block_values)
+    assert np.array_equal(tl, tl_ref)
+    assert tv.tobytes() == tv_ref.tobytes()
+    if aligned:      # blocks on the grid cost exactly their own bytes
+        assert tv.size == lay.block_values.size
+
+
+def test_blocks_pack_equals_tile_pack():
+    """pp_pack_create_blocks is pp_blocks_to_tiles followed by pp_pack_create."""
+    wl = synth.irregular_blocks(41, 200, 330, 32, wdtype="f16", n_row_cuts=3, n_col_cuts=6, keep=0.6, bias_std=0.1)
+    lay = wl.layers[0]
+    tl, tv = pb.pp_blocks_to_tiles(lay.M, lay.N, lay.B, lay.blocks, lay.block_values)
+    a = pb.Packed.from_blocks(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.blocks, lay.block_values, lay.bias)
+    b = pb.Packed(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, tl, tv, lay.bias)
+    for which in ("row_ptr", "tile_col", "values", "bias_piv", "gather_idx", "scatter_idx"):
+        assert np.array_equal(a.get(which), b.get(which)), which
+    # and the tile form reconstructs the same W as the block form (oracle on both)
+    W_t = po.reconstruct(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, tl, tv)
+    W_b = po.reconstruct_blocks(lay.M, lay.N, lay.row_perm, lay.col_perm, lay.blocks, lay.block_values)
+    assert np.array_equal(W_t, W_b)
+
+
+def test_blocks_error_codes():
+    rp = np.arange(64, dtype=np.int32)
+    v = np.zeros(64 * 64, dtype=np.float32)
+    def status(blocks, vals):
+        try:
+            pb.Packed.from_blocks(64, 64, 16, rp, rp, np.array(blocks, dtype=np.int32), vals)
+        except pb.PPError as e:
+            return e.status
+        return 0
+    assert status([[0, 0, 16, 16]], v[:256]) == 0
+    assert status([[0, 0, 16, 16], [15, 15, 2, 2]], v[:260]) == 3      # overlap in one element
+    assert status([[0, 0, 16, 16], [16, 16, 2, 2]], v[:260]) == 0                       # touching corners is fine
+    assert status([[60, 0, 8, 4]], v[:32]) == 3                         # leaves the padded matrix
+    assert status([[0, 0, 0, 4]], v[:0]) == 3                           # empty block
+    assert status([[-1, 0, 2, 2]], v[:4]) == 3
