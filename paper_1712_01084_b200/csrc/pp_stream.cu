@@ -345,6 +345,10 @@ struct WeightRing {
         if (p < wend) cp_async_16(slot + 32 * u, vals + (size_t)p * 32);
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
+    __device__ __forceinline__ void refill(int u, int p) const {       // p is known to be inside the warp's range
+        cp_async_16(slot + 32 * u, vals + (size_t)p * 32);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
     __device__ __forceinline__ void prologue(int wbeg, int wend) const {
 #pragma unroll
         for (int u = 0; u < U; ++u) fill(u, wbeg + u, wend);
@@ -423,10 +427,56 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
         const unsigned short* rawu = static_cast<const unsigned short*>(L.raw);
         const __half* xrow = xs + g * a.xs_stride + 2 * t;
         uint32_t mb0 = 0u, mb1 = 0u;
-        for (int base = wbeg; base < wend; base += U) {
+        // batch 1: x is read through the index array (index -1 reads raw[-1] = 0).  Every 8 fragments the
+        // warp builds their 8 B-operands at once, 4 lanes per fragment (lane 4f + t holds columns 2t, 2t+1,
+        // 2t+8, 2t+9 of fragment f), and hands them to the lanes that feed the tensor core with two
+        // shuffles per fragment.
+        auto gather8 = [&](int p) {
+            (void)xw.get(p, wend, lane);                       // moves the window when needed
+            const int xo = __shfl_sync(0xffffffffu, xw.cur, (p - xw.base) + g);
+            int2 i0, i1;
+            if (idx16) {
+                const uint16_t* t16 = reinterpret_cast<const uint16_t*>(L.idxs) + xo + 2 * t;
+                const uint32_t p0 = *reinterpret_cast<const uint32_t*>(t16);
+                const uint32_t p1 = *reinterpret_cast<const uint32_t*>(t16 + 8);
+                i0 = make_int2((int)(p0 & 0xffffu) - 1, (int)(p0 >> 16) - 1);
+                i1 = make_int2((int)(p1 & 0xffffu) - 1, (int)(p1 >> 16) - 1);
+            } else {
+                i0 = *reinterpret_cast<const int2*>(L.idxs + xo + 2 * t);
+                i1 = *reinterpret_cast<const int2*>(L.idxs + xo + 2 * t + 8);
+            }
+            mb0 = (uint32_t)rawu[i0.x] | ((uint32_t)rawu[i0.y] << 16);
+            mb1 = (uint32_t)rawu[i1.x] | ((uint32_t)rawu[i1.y] << 16);
+        };
+        // Fragments are taken in groups of GRP; fragment wbeg + i sits in ring slot i % U.  A group of 8
+        // that lies inside one strip, with all its refills inside the warp's range, runs without any
+        // per-fragment test (the common case: a strip is hundreds of fragments long).
+        constexpr int GRP = (8 % U == 0) ? 8 : U;
+        for (int base = wbeg; base < wend; base += GRP) {
+            if (GRP == 8 && base + 8 + U <= wend && base + 8 <= seg_end) {
+                if (direct) gather8(base);
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int p = base + u;
+                for (int j = 0; j < 8; ++j) {
+                    uint32_t b0 = 0u, b1 = 0u;
+                    if (direct) {
+                        b0 = __shfl_sync(0xffffffffu, mb0, j * 4 + t);
+                        b1 = __shfl_sync(0xffffffffu, mb1, j * 4 + t);
+                    } else {
+                        const int xoff = xw.get(base + j, wend, lane);
+                        if (has_x) {
+                            b0 = *reinterpret_cast<const uint32_t*>(xrow + xoff);
+                            b1 = *reinterpret_cast<const uint32_t*>(xrow + xoff + 8);
+                        }
+                    }
+                    const uint4 wa = ring.take(j % U);
+                    ring.refill(j % U, base + j + U);
+                    mma_16x8x16(acc, wa, b0, b1);
+                }
+                continue;
+            }
+#pragma unroll
+            for (int j = 0; j < GRP; ++j) {
+                const int p = base + j;
                 if (p < wend) {
                     if (p == seg_end) {
                         park(ls + warp);
@@ -436,28 +486,8 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
                     }
                     uint32_t b0 = 0u, b1 = 0u;
                     if (direct) {
-                        // batch 1: x is read through the index array (index -1 reads raw[-1] = 0).  Every 8
-                        // fragments the warp builds their 8 B-operands at once, 4 lanes per fragment (lane
-                        // 4f + t holds columns 2t, 2t+1, 2t+8, 2t+9 of fragment f), and hands them to the
-                        // lanes that feed the tensor core with two shuffles per fragment.
                         const int in_group = (p - wbeg) & 7;
-                        if (in_group == 0) {
-                            (void)xw.get(p, wend, lane);                       // moves the window when needed
-                            const int xo = __shfl_sync(0xffffffffu, xw.cur, (p - xw.base) + g);
-                            int2 i0, i1;
-                            if (idx16) {
-                                const uint16_t* t16 = reinterpret_cast<const uint16_t*>(L.idxs) + xo + 2 * t;
-                                const uint32_t p0 = *reinterpret_cast<const uint32_t*>(t16);
-                                const uint32_t p1 = *reinterpret_cast<const uint32_t*>(t16 + 8);
-                                i0 = make_int2((int)(p0 & 0xffffu) - 1, (int)(p0 >> 16) - 1);
-                                i1 = make_int2((int)(p1 & 0xffffu) - 1, (int)(p1 >> 16) - 1);
-                            } else {
-                                i0 = *reinterpret_cast<const int2*>(L.idxs + xo + 2 * t);
-                                i1 = *reinterpret_cast<const int2*>(L.idxs + xo + 2 * t + 8);
-                            }
-                            mb0 = (uint32_t)rawu[i0.x] | ((uint32_t)rawu[i0.y] << 16);
-                            mb1 = (uint32_t)rawu[i1.x] | ((uint32_t)rawu[i1.y] << 16);
-                        }
+                        if (in_group == 0) gather8(p);
                         b0 = __shfl_sync(0xffffffffu, mb0, in_group * 4 + t);
                         b1 = __shfl_sync(0xffffffffu, mb1, in_group * 4 + t);
                     } else {
@@ -467,8 +497,8 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
                             b1 = *reinterpret_cast<const uint32_t*>(xrow + xoff + 8);
                         }
                     }
-                    const uint4 wa = ring.take(u);
-                    ring.fill(u, p + U, wend);
+                    const uint4 wa = ring.take(j % U);
+                    ring.fill(j % U, p + U, wend);
                     mma_16x8x16(acc, wa, b0, b1);
                 }
             }
