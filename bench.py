@@ -239,6 +239,51 @@ def time_enqueue(torch, enqueue, calls_per_graph, replays=20):
     return e0.elapsed_time(e1) * 1e3 / (replays * calls_per_graph)
 
 
+def paper_geometry(pb, torch, synth, sizes=(64, 128, 256, 512, 1024, 2048, 4096), per_sides=(32, 16, 8, 4)):
+    """The geometry the paper itself measures (Section 5): size x size, 1/fill-in square blocks on the diagonal
+    of the pivoted matrix, batch 1, here fp32.  Per case: this library's kernels (blocks through
+    pp_layer_create_blocks, grid = block edge clamped to 16..64) and the paper's own kernel model (one thread
+    group per block, one thread per output row) in its three physical layouts.  "warm" repeats one layer as the
+    paper's 2,500-call average does; "cold" rotates copies that together exceed twice the L2 (given where at
+    most 96 copies do)."""
+    def check(st):
+        if st != 0:
+            raise pb.PPError(st, "forward")
+
+    geo = {}
+    for size in sizes:
+        for per_side in per_sides:
+            edge = size // per_side
+            grid = 16 if edge <= 16 else 32 if edge <= 32 else 64
+            wl = synth.paper_square(size, per_side, grid, wdtype="f32")
+            lay = wl.layers[0]
+            L0 = pb.Layer.from_synth(lay)
+            x = torch.from_numpy(wl.x).cuda()
+            y = torch.empty((1, size), dtype=torch.float32, device="cuda")
+            fn = pb.lib().pp_forward
+            warm = time_enqueue(torch, lambda i, sp: check(fn(L0._h, x.data_ptr(), y.data_ptr(), 1, 0, sp)), 64)
+            row = {"block_edge": edge, "grid": grid, "block_bytes": lay.block_bytes, "us_warm": round(warm, 3)}
+            R = -(-2 * L2_BYTES // max(1, lay.block_bytes)) + 1
+            if R <= 96:
+                reps = [L0] + [L0.clone() for _ in range(R - 1)]
+                cold = time_enqueue(torch, lambda i, sp: check(fn(reps[i % R]._h, x.data_ptr(), y.data_ptr(), 1, 0, sp)), R)
+                row.update({"us_cold": round(cold, 3), "GBps_cold": round(lay.block_bytes / cold / 1e3, 1), "copies": R})
+                for r in reps[1:]:
+                    r.close()
+            L0.close()
+            # the paper's own kernel (one thread group per block, one thread per output row) in its three layouts
+            if edge <= 1024:
+                x1, y1 = x.reshape(-1), y.reshape(-1)
+                fl = pb.lib().pp_listing1_forward
+                for name, layout in (("brc", pb.PP_LAYOUT_BRC), ("bcr", pb.PP_LAYOUT_BCR), ("cbr", pb.PP_LAYOUT_CBR)):
+                    K = pb.Listing1(size, per_side, layout, lay.row_perm, lay.col_perm, lay.block_values)
+                    row[f"listing1_{name}_us_warm"] = round(time_enqueue(
+                        torch, lambda i, sp: check(fl(K._h, x1.data_ptr(), y1.data_ptr(), sp)), 64), 3)
+                    K.close()
+            geo[f"size{size}_fill{100.0 / per_side:g}"] = row
+    return geo
+
+
 def other_workloads(pb, torch, synth):
     """Latency of the other synthetic workloads: cold (calls rotate over copies of the layers that
     together exceed twice the L2) and warm (one copy, weights may sit in L2)."""
@@ -274,33 +319,7 @@ def other_workloads(pb, torch, synth):
     layer_case("cfg5_fc8192_f16_b64_k128_batch128_pivoted_output", synth.config5(k=128, batch=128), 128, pivoted=True)
     layer_case("cfg5_fc8192_f16_b64_k32_batch128", synth.config5(k=32, batch=128), 128)
 
-    # The geometry the paper itself measures (Section 5): size x size, 1/fill-in square blocks on the diagonal of
-    # the pivoted matrix, batch 1, here fp32.  Blocks go through pp_layer_create_blocks (grid = block edge clamped
-    # to 16..64).  "warm" repeats one layer as the paper's 2,500-call average does; "cold" rotates copies
-    # that together exceed twice the L2 (given where at most 96 copies do).
-    geo = {}
-    for size in (64, 128, 256, 512, 1024, 2048, 4096):
-        for per_side in (32, 16, 8, 4):
-            edge = size // per_side
-            grid = 16 if edge <= 16 else 32 if edge <= 32 else 64
-            wl = synth.paper_square(size, per_side, grid, wdtype="f32")
-            lay = wl.layers[0]
-            L0 = pb.Layer.from_synth(lay)
-            x = torch.from_numpy(wl.x).cuda()
-            y = torch.empty((1, size), dtype=torch.float32, device="cuda")
-            fn = pb.lib().pp_forward
-            warm = time_enqueue(torch, lambda i, sp: check(fn(L0._h, x.data_ptr(), y.data_ptr(), 1, 0, sp)), 64)
-            row = {"block_edge": edge, "grid": grid, "block_bytes": lay.block_bytes, "us_warm": round(warm, 3)}
-            R = -(-2 * L2_BYTES // max(1, lay.block_bytes)) + 1
-            if R <= 96:
-                reps = [L0] + [L0.clone() for _ in range(R - 1)]
-                cold = time_enqueue(torch, lambda i, sp: check(fn(reps[i % R]._h, x.data_ptr(), y.data_ptr(), 1, 0, sp)), R)
-                row.update({"us_cold": round(cold, 3), "GBps_cold": round(lay.block_bytes / cold / 1e3, 1), "copies": R})
-                for r in reps[1:]:
-                    r.close()
-            L0.close()
-            geo[f"size{size}_fill{100.0 / per_side:g}"] = row
-    out["paper_geometry_f32_batch1"] = geo
+    out["paper_geometry_f32_batch1"] = paper_geometry(pb, torch, synth)
 
     for batch in (1, 8):
         wl = synth.config3(batch=batch)
@@ -347,6 +366,8 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="skip the density sweep")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
     ap.add_argument("--no-configs", action="store_true", help="skip the other synthetic workloads")
+    ap.add_argument("--geometry", default=None, metavar="SIZE:BLOCKS",
+                    help="only time the paper's square-block geometry for one case (e.g. 2048:4) and print that table")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -362,6 +383,11 @@ def main():
     from paper_1712_01084_b200 import synth
 
     torch.cuda.set_device(local_rank)
+    if args.geometry:
+        size, per_side = (int(v) for v in args.geometry.split(":"))
+        pb.lib()
+        print(json.dumps({"paper_geometry_f32_batch1": paper_geometry(pb, torch, synth, (size,), (per_side,))}))
+        return
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     pb.lib()

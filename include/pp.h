@@ -281,6 +281,36 @@ pp_status_t pp_lstm_forward(pp_lstm_t* lstm, const void* x_seq, void* h, float* 
 pp_status_t pp_lstm_status(pp_lstm_t* lstm, pp_status_t* status);
 
 /* ------------------------------------------------------------------------- *
+ * The paper's own kernel model (Section 4.1.1 and Listing 1), for the layout
+ * study of Section 4.1.1 and as the baseline the other kernels are measured
+ * against: one thread group per block, one thread per output coordinate running
+ * along its row of the block, the block's input slice fetched by the group
+ * through the column index array, the result stored through the row index array.
+ * Geometry of Section 5: a size x size matrix, n_blocks identical square blocks
+ * of edge size / n_blocks, block k on pivoted rows and columns [k*edge, (k+1)*edge).
+ * fp32, one input vector, no bias, no activation.
+ *
+ * layout: physical order of M_block (rightmost axis fastest):
+ *   PP_LAYOUT_BRC block,row,column  PP_LAYOUT_BCR block,column,row  PP_LAYOUT_CBR column,block,row
+ * row_perm, col_perm   host, int32[size], pivoted -> original (no padding)
+ * block_values         host, float[n_blocks][edge][edge], row-major per block
+ * x, y                 device, float[size]; must not alias
+ * pp_listing1_pack writes the values in the chosen layout to host memory out
+ * (n_blocks*edge*edge floats); create uses it before the upload.
+ * Errors: PP_ERR_INVALID_ARG (sizes, NULL, size not a multiple of n_blocks),
+ * PP_ERR_BAD_PERM, PP_ERR_UNSUPPORTED when edge > 1024 (one thread per block row),
+ * PP_ERR_ALLOC, PP_ERR_CUDA.  pp_listing1_forward only enqueues.
+ * ------------------------------------------------------------------------- */
+typedef struct pp_listing1 pp_listing1_t;
+typedef enum { PP_LAYOUT_BRC = 0, PP_LAYOUT_BCR = 1, PP_LAYOUT_CBR = 2 } pp_layout_t;
+pp_status_t pp_listing1_pack(int size, int n_blocks, pp_layout_t layout, const float* block_values, float* out);
+pp_status_t pp_listing1_create(pp_listing1_t** out, int size, int n_blocks, pp_layout_t layout,
+                               const int32_t* row_perm, const int32_t* col_perm,
+                               const float* block_values);
+pp_status_t pp_listing1_destroy(pp_listing1_t* h);
+pp_status_t pp_listing1_forward(pp_listing1_t* h, const float* x, float* y, void* cuda_stream);
+
+/* ------------------------------------------------------------------------- *
  * Forward call that allocates nothing (the paper has no counterpart; this is a
  * packaging of pp_forward's small-batch kernel).
  *

@@ -76,6 +76,10 @@ def lib() -> ctypes.CDLL:
         "pp_lstm_destroy": (ci, [vp]),
         "pp_lstm_forward": (ci, [vp, vp, vp, vp, ci, vp]),
         "pp_lstm_status": (ci, [vp, ctypes.POINTER(ci)]),
+        "pp_listing1_pack": (ci, [ci, ci, ci, fp, fp]),
+        "pp_listing1_create": (ci, [ctypes.POINTER(vp), ci, ci, ci, i32p, i32p, fp]),
+        "pp_listing1_destroy": (ci, [vp]),
+        "pp_listing1_forward": (ci, [vp, vp, vp, vp]),
         "pp_pack_device_image_bytes": (ci, [vp, i64p]),
         "pp_pack_device_image": (ci, [vp, vp, c64]),
         "pp_forward_noalloc": (ci, [vp, vp, vp, vp, ci, ci, vp]),
@@ -506,3 +510,52 @@ def pp_lstm_forward(lstm: Lstm, x_seq, h, c, stream=None):
                                  ctypes.c_void_p(c.data_ptr()), int(x_seq.shape[0]), _stream_ptr(stream)),
            "pp_lstm_forward")
     return h, c
+
+
+# ------------------------------------------------- the paper's kernel model (Listing 1)
+PP_LAYOUT_BRC, PP_LAYOUT_BCR, PP_LAYOUT_CBR = 0, 1, 2
+
+
+def pp_listing1_pack(size, n_blocks, layout, block_values) -> np.ndarray:
+    bv = np.ascontiguousarray(block_values, dtype=np.float32).reshape(-1)
+    out = np.empty_like(bv)
+    fp = ctypes.POINTER(ctypes.c_float)
+    _check(lib().pp_listing1_pack(int(size), int(n_blocks), int(layout), bv.ctypes.data_as(fp), out.ctypes.data_as(fp)),
+           "pp_listing1_pack")
+    return out
+
+
+class Listing1:
+    """The paper's kernel (one thread group per block, one thread per output row) with a chosen
+    physical layout of the blocks (pp_listing1_create / pp_listing1_forward)."""
+
+    def __init__(self, size, n_blocks, layout, row_perm, col_perm, block_values):
+        rp, rpp = _i32(row_perm)
+        cp, cpp = _i32(col_perm)
+        bv = np.ascontiguousarray(block_values, dtype=np.float32).reshape(-1)
+        if size % n_blocks or bv.size != n_blocks * (size // n_blocks) ** 2 or rp.size != size or cp.size != size:
+            raise ValueError("sizes do not describe n_blocks square blocks of edge size/n_blocks")
+        self._h = ctypes.c_void_p()
+        _check(lib().pp_listing1_create(ctypes.byref(self._h), int(size), int(n_blocks), int(layout), rpp, cpp,
+                                        bv.ctypes.data_as(ctypes.POINTER(ctypes.c_float))), "pp_listing1_create")
+        self.size = int(size)
+
+    def forward(self, x, out=None, stream=None):
+        import torch
+        _require_cuda(x, "x")
+        if x.dtype != torch.float32 or x.numel() != self.size:
+            raise ValueError("x must be float32 with `size` elements")
+        y = torch.empty(self.size, dtype=torch.float32, device=x.device) if out is None else out
+        _check(lib().pp_listing1_forward(self._h, x.data_ptr(), y.data_ptr(), _stream_ptr(stream)), "pp_listing1_forward")
+        return y
+
+    def close(self):
+        if self._h:
+            lib().pp_listing1_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -95,3 +95,31 @@ def test_block_layer_in_a_chain(pb):
     bound = e0 @ np.abs(W1).T + 2e-3 * a1 + 1e-4
     assert np.all(np.abs(y.astype(np.float64) - y1) <= bound)
     ch.close(); L0.close(); L1.close()
+
+
+# ------------------------------------------------ the paper's kernel model (Section 4.1.1, Listing 1)
+@pytest.mark.parametrize("layout", [0, 1, 2])
+@pytest.mark.parametrize("size,blocks_per_side", [(512, 16), (1024, 4), (96, 8), (2048, 2), (60, 5)])
+def test_listing1_kernel_layouts(pb, layout, size, blocks_per_side):
+    """One thread group per block, one thread per output row, in the three layouts; same numbers as the oracle."""
+    for integer in (False, True):
+        wl = synth.paper_square(size, blocks_per_side, 1, wdtype="f32", integer_values=integer)
+        lay = wl.layers[0]
+        K = pb.Listing1(size, blocks_per_side, layout, lay.row_perm, lay.col_perm, lay.block_values)
+        y = K.forward(torch.from_numpy(wl.x[0]).cuda()).cpu().numpy()
+        K.close()
+        y_ref, _, a = _reference(lay, wl.x, 0)
+        if integer:
+            assert np.array_equal(y.astype(np.float64), y_ref[0])
+        else:
+            assert np.all(np.abs(y.astype(np.float64) - y_ref[0]) <= 1e-5 * a[0] + 1e-6)
+
+
+def test_listing1_rejects_what_it_cannot_run(pb):
+    rp = np.arange(4096, dtype=np.int32)
+    with pytest.raises(pb.PPError) as e:
+        pb.Listing1(4096, 2, 0, rp, rp, np.zeros(2 * 2048 * 2048, dtype=np.float32))     # 2048 threads per group
+    assert e.value.status == 6
+    with pytest.raises(pb.PPError) as e:
+        pb.Listing1(64, 4, 0, rp[:64][::-1] * 0, rp[:64], np.zeros(4 * 16 * 16, dtype=np.float32))
+    assert e.value.status == 2
