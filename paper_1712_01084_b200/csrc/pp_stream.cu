@@ -278,7 +278,33 @@ __device__ __forceinline__ void finalize(const StreamArgs& a, const CtaDesc& d, 
         }
     };
 
-    const int n_out = d.s_count * per_strip;
+    // One input vector (the common case) needs no index arithmetic beyond a shift: element e is row e of
+    // the CTA's strips.  Kept apart from the general loop so that this path is a short run of code.
+    const bool single = batch == 1;
+    if (single) {
+        for (int e = tid; e < d.s_count * RG; e += kThreads) {
+            const int ls = e / RG, r = e % RG;
+            const int wl = L.wlohi[ls] & 0xff, wh = L.wlohi[ls] >> 8;
+            float v = 0.0f;
+            for (int w = wl; w <= wh; ++w)
+                if (L.wb[w] < L.wb[w + 1]) v += L.segp[(ls + w) * RG + r];
+            const int4 info = L.sinfo[ls];
+            if (info.y == 2) {
+                unsigned* slot = reinterpret_cast<unsigned*>(a.partials + (size_t)info.z * (RG * kStreamMaxBatch) + r);
+                unsigned mine = __float_as_uint(v);
+                if (mine == kEmptySlot) mine = 0x7fc00000u;
+                const unsigned other = atomicExch(slot, mine);
+                if (other == kEmptySlot) continue;
+                v += __uint_as_float(other);
+                *slot = kEmptySlot;
+            } else if (info.y != 1) {
+                a.partials[(size_t)(info.z + (int)blockIdx.x - info.x) * (RG * kStreamMaxBatch) + r] = v;
+                continue;
+            }
+            emit(ls, r, 0, v);
+        }
+    }
+    const int n_out = single ? 0 : d.s_count * per_strip;
     for (int e = tid; e < n_out; e += kThreads) {
         const int ls = e / per_strip, rem = e - ls * per_strip;
         const int r = rem / batch, b = rem - r * batch;
