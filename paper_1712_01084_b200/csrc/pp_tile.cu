@@ -28,14 +28,13 @@
 namespace pp {
 namespace {
 
-constexpr int kStages = 8;
-constexpr int kProducers = 4;      // producer warps (one lane each issues bulk copies; kStages is a multiple of it)
+constexpr int kProducers = 4;      // producer warps (one lane each issues bulk copies; the stage count is a multiple of it)
 constexpr int kXBytes = kTileBatch * 64 * 2;     // 128 x 64 fp16 = 16 KiB
 constexpr int kWBytes = 64 * 64 * 2;             // 64 x 64 fp16 = 8 KiB
-constexpr int kStageBytes = kXBytes + kWBytes;
 constexpr int kTmemCols = 64;
 constexpr int kThreads = 32 * (kProducers + 1 + 4);    // producers, MMA issuer, 4 epilogue warps
 constexpr int kPollLimit = 1 << 22;
+constexpr int kIdxCap = 512;       // tiles of a block-row whose indices are staged in shared memory
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -81,6 +80,10 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     return d;
 }
 
+// The descriptor of the same operand layout `bytes` further on (bytes a multiple of 16; shared-memory
+// addresses stay below 256 KiB, so the 14-bit address field cannot carry into its neighbours).
+__device__ __forceinline__ uint64_t desc_advance(uint64_t d, uint32_t bytes) { return d + (uint64_t)(bytes >> 4); }
+
 // Instruction descriptor: D = f32, A = B = f16, both K-major, N = 64, M = 128.
 constexpr uint32_t kInstrDesc = (1u << 4) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
 
@@ -95,26 +98,49 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
                  :: "r"(smem_u32(bar)) : "memory");
 }
 
+// STAGES stages of (XB bytes of the X block + one tile).  A stage is re-used once per STAGES tiles and a
+// copy takes 1.5-2 us to land, so small batches (which need only the first 8-row groups of the X block)
+// trade the unused part of the X region for more stages in flight.
+template <int STAGES>
 struct TileSmem {
-    uint64_t full[kStages];
-    uint64_t empty[kStages];
+    uint64_t full[STAGES];
+    uint64_t empty[STAGES];
     uint64_t acc_full;
     uint32_t tmem_base;
     int abort_flag;
     float bias[64];           // bias and destination rows of the block-row
     int dst[64];
+    int col[kIdxCap];         // tile-column and image position of the block-row's first kIdxCap tiles
+    int pos[kIdxCap];
 };
 
+template <int STAGES, int XB>
 __global__ void __launch_bounds__(kThreads, 1)
 tile_f16_kernel(const TileArgs a) {
+    constexpr int kStages = STAGES;
+    constexpr int kStageBytes = XB + kWBytes;
+    static_assert(STAGES % kProducers == 0 && XB % 1024 == 0 && XB <= kXBytes, "stage geometry");
     extern __shared__ unsigned char smem_raw[];
     // stage buffers need 1024-byte alignment for the 128-byte swizzle
     unsigned char* stages = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    TileSmem* sm = reinterpret_cast<TileSmem*>(stages + kStages * kStageBytes);
+    // The A operand of every MMA spans 128 rows (16 KiB) from the start of its stage's X region, whatever XB is:
+    // the rows past XB are dead batch rows read from the bytes that follow (the stage's tile, the next stage).
+    // kXBytes - XB spare bytes behind the last stage keep that read inside the allocation.
+    TileSmem<STAGES>* sm = reinterpret_cast<TileSmem<STAGES>*>(stages + kStages * kStageBytes + (kXBytes - XB));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int br = blockIdx.x;
     const int t0 = __ldg(a.row_ptr + br), k = __ldg(a.row_ptr + br + 1) - t0;
 
+    // The block-row's tile list goes to shared memory once, by the whole CTA, while tensor memory is set
+    // up: a producer that fetched each tile's indices from global memory just before its copies spent one
+    // L2 round trip per tile on that and capped the kernel at four tiles per round trip.
+    {
+        const int cbase0 = __ldg(a.col_ptr + br);
+        for (int i = threadIdx.x; i < k && i < kIdxCap; i += kThreads) {
+            sm->col[i] = __ldg(a.tile_col + cbase0 + i);
+            sm->pos[i] = __ldg(a.tile_pos + t0 + i);
+        }
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&sm->full[s], 1); mbar_init(&sm->empty[s], 1); }
         mbar_init(&sm->acc_full, 1);
@@ -138,6 +164,10 @@ tile_f16_kernel(const TileArgs a) {
         // take turns, so the requests come from different warps)
         if (lane == 0) {
             int last = -1;
+            // Only the 8-row groups (1 KiB each) that hold live batch rows are fetched.  The rows of the
+            // stage beyond them keep whatever they held: a row of the A operand only reaches its own row
+            // of the accumulator, and rows past the batch are never stored.
+            const uint32_t xbytes = (uint32_t)((a.batch + 7) / 8) * 1024u;
             const int cbase = __ldg(a.col_ptr + br);
             const int rot = k > 0 ? (int)(((long long)br * k) / gridDim.x) : 0;
             for (int t = warp; t < k; t += kProducers) {
@@ -146,13 +176,14 @@ tile_f16_kernel(const TileArgs a) {
                 // block-rows start at different tiles of their lists, so that CTAs running side by side
                 // do not all ask the L2 for the same X segment at the same moment
                 const int tt = (t + rot) % k;
-                const int col = __ldg(a.tile_col + cbase + tt);
-                mbar_expect_tx(&sm->full[s], kStageBytes);
-                bulk_load(stages + s * kStageBytes + kXBytes, a.tiles_sw + (size_t)__ldg(a.tile_pos + t0 + tt) * kWBytes, kWBytes, &sm->full[s]);
+                const int col = tt < kIdxCap ? sm->col[tt] : __ldg(a.tile_col + cbase + tt);
+                const int pos = tt < kIdxCap ? sm->pos[tt] : __ldg(a.tile_pos + t0 + tt);
+                mbar_expect_tx(&sm->full[s], xbytes + kWBytes);
+                bulk_load(stages + s * kStageBytes + XB, a.tiles_sw + (size_t)pos * kWBytes, kWBytes, &sm->full[s]);
                 // the permuted input comes from the gather kernel launched just before: everything up to here
                 // (set-up, the first weight copies) may overlap its tail
                 if (t == warp) asm volatile("griddepcontrol.wait;" ::: "memory");
-                bulk_load(stages + s * kStageBytes, a.x_sw + (size_t)col * kXBytes, kXBytes, &sm->full[s]);
+                bulk_load(stages + s * kStageBytes, a.x_sw + (size_t)col * kXBytes, xbytes, &sm->full[s]);
                 last = t;
             }
             if (*abort_flag) {
@@ -165,15 +196,16 @@ tile_f16_kernel(const TileArgs a) {
         // ---------------- MMA issuer (one lane)
         if (lane == 0) {
             bool ok = true;
+            const uint64_t desc0 = smem_desc_sw128(smem_u32(stages));
             for (int t = 0; t < k && ok; ++t) {
                 const int s = t % kStages;
                 ok = mbar_wait(&sm->full[s], (t / kStages) & 1, abort_flag);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t xa = smem_u32(stages + s * kStageBytes), wa = xa + kXBytes;
+                const uint64_t xd = desc_advance(desc0, (uint32_t)(s * kStageBytes)), wd = desc_advance(xd, XB);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)
-                    umma_f16(tmem, smem_desc_sw128(xa + kk * 32), smem_desc_sw128(wa + kk * 32), t > 0 || kk > 0);
+                    umma_f16(tmem, desc_advance(xd, kk * 32), desc_advance(wd, kk * 32), t > 0 || kk > 0);
                 umma_commit(&sm->empty[s]);          // frees the stage once these MMAs have read it
             }
             if (k > 0 && ok) umma_commit(&sm->acc_full);   // accumulator complete
@@ -261,6 +293,7 @@ constexpr int kCTmemCols = 64 * kTileRows;
 static_assert(kTileRows * 64 * kTileBatch * 4 + 4 * 32 * 33 * 4 <= kCStages * kCStageBytes, "exchange buffers reuse the stages");
 __device__ __forceinline__ int q_of_warp(int warp) { return warp & 3; }
 constexpr int kCThreads = 32 * (kCProducers + 1 + 4);          // producers, MMA issuer, 4 epilogue warps
+constexpr int kStepCap = 96;                                   // step records of a CTA staged in shared memory
 static_assert(kCStages == kCProducers, "one stage per producer warp");
 
 struct ClusterSmem {
@@ -272,10 +305,18 @@ struct ClusterSmem {
     uint32_t acc_mask;        // accumulators that received at least one tile
     float bias[64];           // bias and destination rows of the block-row this CTA finishes
     int dst[64];
+    int4 steps[kStepCap][2];  // this CTA's first kStepCap step records
 };
+static_assert(sizeof(TileStep) == 2 * sizeof(int4), "a step record is staged as two 16-byte words");
 
 __device__ __forceinline__ TileStep load_step(const TileStep* p) {
     const int4 lo = __ldg(reinterpret_cast<const int4*>(p)), hi = __ldg(reinterpret_cast<const int4*>(p) + 1);
+    TileStep s;
+    s.col = lo.x; s.tile[0] = lo.y; s.tile[1] = lo.z; s.tile[2] = lo.w; s.tile[3] = hi.x; s.ntiles = hi.y; s.pos = hi.z;
+    s.pad = 0;
+    return s;
+}
+__device__ __forceinline__ TileStep unpack_step(const int4 lo, const int4 hi) {
     TileStep s;
     s.col = lo.x; s.tile[0] = lo.y; s.tile[1] = lo.z; s.tile[2] = lo.w; s.tile[3] = hi.x; s.ntiles = hi.y; s.pos = hi.z;
     s.pad = 0;
@@ -318,6 +359,13 @@ tile_cluster_f16_kernel(const TileArgs a) {
     // same tile-columns) do not all ask the L2 for the same X block at the same moment
     const int rot = n_steps > 0 ? (int)(((long long)grp * n_steps) / n_groups) : 0;
 
+    // This CTA's step records go to shared memory once, by all threads, while tensor memory is set up: read
+    // from global memory inside the loops they cost the producers and the MMA issuer one L2 round trip per step.
+    for (int i = threadIdx.x; i < 2 * n_steps && i < 2 * kStepCap; i += kCThreads)
+        sm->steps[i >> 1][i & 1] = __ldg(reinterpret_cast<const int4*>(a.steps + p0) + i);
+    auto step_at = [&](int i) {
+        return i < kStepCap ? unpack_step(sm->steps[i][0], sm->steps[i][1]) : load_step(a.steps + p0 + i);
+    };
     if (threadIdx.x == 0) {
         for (int s = 0; s < kCStages; ++s) { mbar_init(&sm->full[s], 1); mbar_init(&sm->empty[s], 1); }
         mbar_init(&sm->acc_full, 2);          // the tensor core's commit + the issuing thread's own arrival
@@ -346,16 +394,17 @@ tile_cluster_f16_kernel(const TileArgs a) {
         if (lane == 0) {
             const int s = warp;
             int last = -1;
+            const uint32_t xbytes = (uint32_t)((a.batch + 7) / 8) * 1024u;   // live 8-row groups of the X block only
             for (int t = warp; t < n_steps; t += kCProducers) {
                 if (t >= kCStages && !mbar_wait(&sm->empty[s], ((t / kCStages) & 1) ^ 1, abort_flag)) break;
-                const TileStep st = load_step(a.steps + p0 + (t + rot) % n_steps);
+                const TileStep st = step_at((t + rot) % n_steps);
                 unsigned char* dst = stages + s * kCStageBytes;
-                mbar_expect_tx(&sm->full[s], (uint32_t)(kXBytes + st.ntiles * kWBytes));
+                mbar_expect_tx(&sm->full[s], xbytes + (uint32_t)(st.ntiles * kWBytes));
                 bulk_load(dst + kXBytes, a.tiles_sw + (size_t)st.pos * kWBytes, (uint32_t)(st.ntiles * kWBytes), &sm->full[s]);
                 // the permuted input comes from the gather kernel launched just before: everything up to here
                 // (set-up, the first weight copies) may overlap its tail
                 if (t == warp) asm volatile("griddepcontrol.wait;" ::: "memory");
-                bulk_load(dst, a.x_sw + (size_t)st.col * kXBytes, kXBytes, &sm->full[s]);
+                bulk_load(dst, a.x_sw + (size_t)st.col * kXBytes, xbytes, &sm->full[s]);
                 last = t;
             }
             if (*abort_flag && last >= 0) {
@@ -370,7 +419,7 @@ tile_cluster_f16_kernel(const TileArgs a) {
             uint32_t mask = 0u;
             for (int t = 0; t < n_steps && ok; ++t) {
                 const int s = t % kCStages;
-                const TileStep st = load_step(a.steps + p0 + (t + rot) % n_steps);
+                const TileStep st = step_at((t + rot) % n_steps);
                 ok = mbar_wait(&sm->full[s], (t / kCStages) & 1, abort_flag);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -561,16 +610,21 @@ static cudaError_t launch_after_gather(void (*kernel)(const TileArgs), int grid,
     return cudaLaunchKernelEx(&cfg, kernel, a);
 }
 
-cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const int32_t* gather_idx, int n_pad, int Mb,
-                        bool use_cluster, cudaStream_t stream) {
-    if (a.batch < 1 || a.batch > kTileBatch) return cudaErrorInvalidValue;
+template <int STAGES, int XB>
+cudaError_t launch_one_row(const TileArgs& a, int Mb, cudaStream_t stream) {
     static bool configured = false;
-    const size_t smem = (size_t)kStages * kStageBytes + sizeof(TileSmem) + 1024;
+    const size_t smem = (size_t)STAGES * (XB + kWBytes) + (kXBytes - XB) + sizeof(TileSmem<STAGES>) + 1024;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(tile_f16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(tile_f16_kernel<STAGES, XB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         configured = true;
     }
+    return launch_after_gather(tile_f16_kernel<STAGES, XB>, Mb, kThreads, smem, a, stream);
+}
+
+cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const int32_t* gather_idx, int n_pad, int Mb,
+                        bool use_cluster, cudaStream_t stream) {
+    if (a.batch < 1 || a.batch > kTileBatch) return cudaErrorInvalidValue;
     if ((size_t)n * 2 > 48 * 1024) return cudaErrorInvalidValue;
     // rows past the batch keep whatever an earlier call left there: every row of the product is independent
     // and the epilogue drops those rows
@@ -589,7 +643,9 @@ cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const 
         const int groups = (Mb + kTileRows - 1) / kTileRows;
         return launch_after_gather(tile_cluster_f16_kernel, groups * kTileRows, kCThreads, smem_c, a, stream);
     }
-    return launch_after_gather(tile_f16_kernel, Mb, kThreads, smem, a, stream);
+    if (a.batch <= 32) return launch_one_row<16, 4 * 1024>(a, Mb, stream);
+    if (a.batch <= 64) return launch_one_row<12, 8 * 1024>(a, Mb, stream);
+    return launch_one_row<8, kXBytes>(a, Mb, stream);
 }
 
 }  // namespace pp
