@@ -142,7 +142,7 @@ size_t round256(size_t n) { return (n + 255) / 256 * 256; }
 struct LayerLayout {
     size_t off[11];       // cta_desc, strip_start, strip_info, scatter, bias, gather, tile_col, items, xoff, values, gather16
     size_t arena_bytes;
-    size_t soff[5];       // partials, counters, spartials, scounters, pivoted-x staging
+    size_t soff[6];       // partials, counters, spartials, scounters, pivoted-x staging, status word
     size_t scratch_bytes;
 };
 
@@ -159,11 +159,11 @@ LayerLayout layer_layout(const pp_packed* pk) {
     size_t pos = 0;
     for (int i = 0; i < 11; ++i) { lo.off[i] = pos; pos += round256(sz[i]); }
     lo.arena_bytes = pos ? pos : 256;
-    const size_t ssz[5] = {(size_t)pk->n_slots * pk->B * pp::kMaxGroupBatch * 4, (size_t)pk->Mb * 4,
+    const size_t ssz[6] = {(size_t)pk->n_slots * pk->B * pp::kMaxGroupBatch * 4, (size_t)pk->Mb * 4,
                            (size_t)pk->stream_slots * g.rg_rows * pp::kStreamMaxBatch * 4, (S ? S : 1) * 4,
-                           (size_t)pp::kMaxGroupBatch * pk->Npad * esz};
+                           (size_t)pp::kMaxGroupBatch * pk->Npad * esz, 4};
     pos = 0;
-    for (int i = 0; i < 5; ++i) { lo.soff[i] = pos; pos += round256(ssz[i]); }
+    for (int i = 0; i < 6; ++i) { lo.soff[i] = pos; pos += round256(ssz[i]); }
     lo.scratch_bytes = pos;
     return lo;
 }
@@ -196,6 +196,7 @@ bool alloc_layer(pp_layer* L, const LayerLayout& lo) {
     L->d_spartials = reinterpret_cast<float*>(sc + lo.soff[2]);
     L->d_scounters = reinterpret_cast<int*>(sc + lo.soff[3]);
     L->d_xstage = sc + lo.soff[4];
+    L->d_status = reinterpret_cast<int*>(sc + lo.soff[5]);     // zeroed with the scratch block; every kernel of the layer raises this word
     return true;
 }
 
@@ -223,7 +224,6 @@ bool tile_setup(pp_layer* L, const pp_layer* from) {
     L->d_tile_pos = reinterpret_cast<int32_t*>(L->d_tile + 2 * rp + pb + sb);
     L->d_tiles_rm = L->d_tile + 2 * rp + pb + sb + qb;
     L->d_x_piv = L->d_tile_scratch;
-    L->d_status = reinterpret_cast<int*>(L->d_tile_scratch + xb);
     if (from) {
         if (from->tile_bytes != L->tile_bytes ||
             cudaMemcpy(L->d_tile, from->d_tile, L->tile_bytes, cudaMemcpyDeviceToDevice) != cudaSuccess) return false;
@@ -262,7 +262,7 @@ pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ld
     s.values = L->d_values; s.xoff = L->d_xoff; s.strip_start = L->d_strip_start;
     s.cta_desc = L->d_cta_desc; s.strip_info = L->d_strip_info;
     s.gather_idx = gather; s.gather16 = L->d_gather16; s.scatter_idx = scatter; s.bias_piv = L->d_bias;
-    s.x = x; s.y = y; s.partials = L->d_spartials; s.counters = L->d_scounters;
+    s.x = x; s.y = y; s.partials = L->d_spartials; s.counters = L->d_scounters; s.status = L->d_status;
     s.ldx = ldx; s.ldy = ldy; s.x_limit = x_limit; s.n_pad = pk->Npad; s.x_len = x_len; s.max_rows = L->stream_max_rows; s.batch = batch;
     s.act = (int)act; s.out_mode = out_mode;
     return pp::launch_stream(pk->wdtype, pk->B, s, pk->cta_desc.data(), L->stream_grid, stream) == cudaSuccess

@@ -20,6 +20,7 @@ struct StreamArgs {
     void* y;                     // [batch][ldy]
     float* partials;             // [stream_slots][rows_per_strip * kStreamMaxBatch]
     int* counters;               // [S], zero between launches
+    int* status;                 // raised to 1 when the bounded wait for the copy of x gave up; may be NULL
     int ldx, ldy;
     int x_limit;                 // with gather_idx == NULL: columns >= x_limit read 0
     int n_pad;                   // pivoted columns staged into shared memory
