@@ -435,19 +435,16 @@ def main():
     us_step = ms * 1e3 / args.steps                      # one step = one layer on every rank
     value = job_value(us_step, world)
 
-    # end to end from host buffers through the public Python call
+    # end to end from host buffers through the library's host-buffer call (pinned host -> device copy, forward,
+    # device -> host copy, stream synchronize, all inside pp_forward_host)
     n_e2e = min(args.steps, 300)
     xh = torch.from_numpy(wl.x).pin_memory()
     yh = torch.empty((1, lay.M), dtype=torch.float32).pin_memory()
-    xd = torch.empty_like(x)
     for i in range(5 + n_e2e):
         if i == 5:
             torch.cuda.synchronize()
             t0 = time.perf_counter()
-        xd.copy_(xh, non_blocking=True)
-        pb.pp_forward(reps[i % len(reps)], xd, lay.act, out=y)
-        yh.copy_(y, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+        pb.pp_forward_host(reps[i % len(reps)], xh, lay.act, out=yh)
     e2e_us = (time.perf_counter() - t0) / n_e2e * 1e6
     e2e_us = max_over_ranks(e2e_us, world)
 

@@ -205,6 +205,17 @@ pp_status_t pp_layer_clone(pp_layer_t** out, const pp_layer_t* src);
 pp_status_t pp_forward(pp_layer_t* layer, const void* x, void* y, int batch,
                        pp_act_t act, void* cuda_stream);
 
+/* The same product (Eq. 2) from HOST buffers: copies x to the device, runs pp_forward and copies y
+ * back, all on the given stream, and returns after the stream has drained, so y_host is valid on
+ * return.  Unlike the calls above this one synchronises, and its first call on a layer (or a call
+ * with a larger batch than any before) allocates the layer's two staging buffers.
+ * x_host  host, [batch][N] row-major, element type = the layer's wdtype (pinned memory makes the
+ *         copies asynchronous to the host, pageable memory works)
+ * y_host  host, float [batch][M]
+ * Errors: as pp_forward, plus PP_ERR_ALLOC. */
+pp_status_t pp_forward_host(pp_layer_t* layer, const void* x_host, float* y_host, int batch,
+                            pp_act_t act, void* cuda_stream);
+
 /* Output permutation elimination (Section 4.2.2): the same product, but the result stays in
  * the layer's pivoted row order -- the last index array of Listing 1 is dropped and the host
  * relabels the coordinates when it interprets the result (an argmax, a softmax).

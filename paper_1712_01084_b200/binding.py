@@ -63,6 +63,7 @@ def lib() -> ctypes.CDLL:
         "pp_layer_clone": (ci, [ctypes.POINTER(vp), vp]),
         "pp_layer_status": (ci, [vp, ctypes.POINTER(ci)]),
         "pp_forward": (ci, [vp, vp, vp, ci, ci, vp]),
+        "pp_forward_host": (ci, [vp, vp, vp, ci, ci, vp]),
         "pp_chain_create": (ci, [ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(ci), ci, ci]),
         "pp_chain_destroy": (ci, [vp]),
         "pp_chain_forward": (ci, [vp, vp, vp, ci, vp]),
@@ -365,6 +366,24 @@ def pp_forward(layer: Layer, x, act: int = PP_ACT_IDENTITY, out=None, stream=Non
         raise ValueError("out must be float32 [batch][M]")
     _check(lib().pp_forward(layer._h, ctypes.c_void_p(x2.data_ptr()), ctypes.c_void_p(y.data_ptr()),
                             batch, int(act), _stream_ptr(stream)), "pp_forward")
+    return y
+
+
+def pp_forward_host(layer: Layer, x_host, act: int = PP_ACT_IDENTITY, out=None, stream=None):
+    """y = act(W x + b) from host tensors (pp_forward_host): x_host and the returned y are CPU tensors
+    (pinned memory keeps the copies asynchronous); the call returns once y is valid."""
+    import torch
+    if x_host.is_cuda or not x_host.is_contiguous():
+        raise ValueError("x_host must be a contiguous CPU tensor")
+    want = torch.float16 if layer.wdtype == np.float16 else torch.float32
+    if x_host.dtype != want or x_host.shape[-1] != layer.N:
+        raise ValueError("x_host must have the layer's element type and N columns")
+    batch = x_host.numel() // layer.N
+    y = torch.empty((batch, layer.M), dtype=torch.float32) if out is None else out
+    if y.is_cuda or y.dtype != torch.float32 or y.numel() != batch * layer.M or not y.is_contiguous():
+        raise ValueError("out must be a contiguous float32 CPU tensor [batch][M]")
+    _check(lib().pp_forward_host(layer._h, x_host.data_ptr(), y.data_ptr(), batch, int(act), _stream_ptr(stream)),
+           "pp_forward_host")
     return y
 
 

@@ -56,6 +56,10 @@ struct pp_layer {
     void* d_x_piv = nullptr;
     int* d_status = nullptr;
     bool tile_ok = false;
+    // staging buffers of pp_forward_host (grown on demand, never shrunk)
+    unsigned char* d_host_x = nullptr;
+    float* d_host_y = nullptr;
+    int host_batch = 0;
 };
 
 struct pp_lstm {
@@ -132,6 +136,8 @@ void free_layer(pp_layer* L) {
     cudaFree(L->d_scratch);
     cudaFree(L->d_tile);
     cudaFree(L->d_tile_scratch);
+    cudaFree(L->d_host_x);
+    cudaFree(L->d_host_y);
     pp_pack_destroy(L->pk);
     delete L;
 }
@@ -490,6 +496,33 @@ pp_status_t pp_forward(pp_layer_t* L, const void* x, void* y, int batch, pp_act_
     if (act != PP_ACT_IDENTITY && act != PP_ACT_RELU) return PP_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(y)) return PP_ERR_INVALID_ARG;
     return forward_impl(L, x, y, batch, act, static_cast<cudaStream_t>(cuda_stream), false);
+}
+
+pp_status_t pp_forward_host(pp_layer_t* L, const void* x_host, float* y_host, int batch, pp_act_t act, void* cuda_stream) {
+    if (!L || !x_host || !y_host || batch < 1) return PP_ERR_INVALID_ARG;
+    if (act != PP_ACT_IDENTITY && act != PP_ACT_RELU) return PP_ERR_INVALID_ARG;
+    const pp_packed* pk = L->pk;
+    const size_t esz = pk->wdtype == PP_F16 ? 2 : 4;
+    if (batch > L->host_batch) {          // first call, or a larger batch than any before: (re)allocate the staging buffers
+        cudaFree(L->d_host_x); cudaFree(L->d_host_y);
+        L->d_host_x = nullptr; L->d_host_y = nullptr; L->host_batch = 0;
+        if (cudaMalloc(reinterpret_cast<void**>(&L->d_host_x), (size_t)batch * pk->N * esz) != cudaSuccess ||
+            cudaMalloc(reinterpret_cast<void**>(&L->d_host_y), (size_t)batch * pk->M * 4) != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(L->d_host_x); L->d_host_x = nullptr;
+            return PP_ERR_ALLOC;
+        }
+        L->host_batch = batch;
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemcpyAsync(L->d_host_x, x_host, (size_t)batch * pk->N * esz, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return PP_ERR_CUDA;
+    const pp_status_t st = forward_impl(L, L->d_host_x, L->d_host_y, batch, act, stream, false);
+    if (st != PP_OK) return st;
+    if (cudaMemcpyAsync(y_host, L->d_host_y, (size_t)batch * pk->M * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess)
+        return PP_ERR_CUDA;
+    return PP_OK;
 }
 
 pp_status_t pp_layer_output_map(const pp_layer_t* L, int32_t* map) {

@@ -503,3 +503,20 @@ def test_chain_identity_link_with_padding_rows(pb):
     chain.close()
     for l in L:
         l.close()
+
+
+def test_forward_host_matches_device_call(pb):
+    """pp_forward_host (host buffers in, host buffers out) gives the bits of pp_forward, also when a second
+    call brings a larger batch (the staging buffers grow) and for pageable as well as pinned memory."""
+    lay = _rand_layer(4242, 300, 500, 32, np.float16, density=0.4)
+    L = pb.Layer.from_synth(lay)
+    for batch, pin in ((1, True), (5, False), (3, True)):
+        x = np.random.default_rng(batch).uniform(-1, 1, (batch, lay.N)).astype(np.float16)
+        xh = torch.from_numpy(x)
+        xh = xh.pin_memory() if pin else xh
+        yh = pb.pp_forward_host(L, xh, 1)
+        yd = pb.pp_forward(L, _dev(x), 1).cpu()
+        assert torch.equal(yh, yd)
+        y_ref, _, a = po.layer_forward(lay, x.astype(np.float64), act=1, threads=4)
+        _check(yh.numpy(), y_ref, a, np.float16, f"host call batch {batch}")
+    L.close()
