@@ -292,6 +292,36 @@ pp_status_t pp_lstm_forward(pp_lstm_t* lstm, const void* x_seq, void* h, float* 
 pp_status_t pp_lstm_status(pp_lstm_t* lstm, pp_status_t* status);
 
 /* ------------------------------------------------------------------------- *
+ * Feed-back search for the index arrays (Section 3.2: after training without
+ * pruning, pick the permutations that keep the largest sum of absolute weights
+ * in the upper-left and lower-right sub-blocks, by greedy optimisation from
+ * given starting permutations; delete the off-diagonal half; repeat on every
+ * remaining block, the number of blocks doubling each time).  Host only.
+ *
+ * The greedy step is read as an alternating balanced split: with the columns
+ * fixed, the ceil(m/2) rows whose entries lean most to the first column half
+ * take the first row half (the best balanced choice for those columns), then
+ * the same for the columns with the rows fixed, until a sweep changes nothing
+ * or max_sweeps is reached; ties go to the line that comes first; lines keep
+ * their relative order inside a half.
+ *
+ * abs_w         host, float[M][N]: absolute values of the trained layer matrix
+ * levels        bisections; the result has 2^levels diagonal blocks (fill-in
+ *               2^-levels); needs 2^levels <= min(M, N)
+ * row_init, col_init   host, int32[M] / int32[N]: starting permutations
+ *               (pivoted -> original), NULL = identity
+ * row_perm_out, col_perm_out   host, int32[M] / int32[N], pivoted -> original
+ * blocks_out    host, int32[2^levels][4] = (first pivoted row, first pivoted
+ *               column, height, width): the blocks pp_layer_create_blocks takes
+ * kept_sum_out  host, sum of abs_w over the kept blocks; may be NULL
+ * Errors: PP_ERR_INVALID_ARG, PP_ERR_BAD_PERM, PP_ERR_ALLOC.
+ * ------------------------------------------------------------------------- */
+pp_status_t pp_pivot_find(int M, int N, const float* abs_w, int levels, int max_sweeps,
+                          const int32_t* row_init, const int32_t* col_init,
+                          int32_t* row_perm_out, int32_t* col_perm_out, int32_t* blocks_out,
+                          double* kept_sum_out);
+
+/* ------------------------------------------------------------------------- *
  * The paper's own kernel model (Section 4.1.1 and Listing 1), for the layout
  * study of Section 4.1.1 and as the baseline the other kernels are measured
  * against: one thread group per block, one thread per output coordinate running

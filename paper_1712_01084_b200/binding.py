@@ -77,6 +77,7 @@ def lib() -> ctypes.CDLL:
         "pp_lstm_destroy": (ci, [vp]),
         "pp_lstm_forward": (ci, [vp, vp, vp, vp, ci, vp]),
         "pp_lstm_status": (ci, [vp, ctypes.POINTER(ci)]),
+        "pp_pivot_find": (ci, [ci, ci, fp, ci, ci, i32p, i32p, i32p, i32p, i32p, ctypes.POINTER(ctypes.c_double)]),
         "pp_listing1_pack": (ci, [ci, ci, ci, fp, fp]),
         "pp_listing1_create": (ci, [ctypes.POINTER(vp), ci, ci, ci, i32p, i32p, fp]),
         "pp_listing1_destroy": (ci, [vp]),
@@ -578,3 +579,21 @@ class Listing1:
             self.close()
         except Exception:
             pass
+
+
+# ------------------------------------------------- feed-back search for index arrays (Section 3.2)
+def pp_pivot_find(abs_w, levels: int, max_sweeps: int = 32, row_init=None, col_init=None):
+    """(row_perm, col_perm, blocks [2^levels, 4], kept sum) for the absolute weights abs_w [M, N] (pp_pivot_find)."""
+    A = np.ascontiguousarray(abs_w, dtype=np.float32)
+    M, N = A.shape
+    i32p = ctypes.POINTER(ctypes.c_int32)
+    ri = None if row_init is None else np.ascontiguousarray(row_init, dtype=np.int32)
+    ci_ = None if col_init is None else np.ascontiguousarray(col_init, dtype=np.int32)
+    rp, cp = np.empty(M, dtype=np.int32), np.empty(N, dtype=np.int32)
+    bl = np.empty((max(1, 2 ** min(int(levels), 20)), 4), dtype=np.int32)
+    kept = ctypes.c_double(0.0)
+    _check(lib().pp_pivot_find(M, N, A.ctypes.data_as(ctypes.POINTER(ctypes.c_float)), int(levels), int(max_sweeps),
+                               None if ri is None else ri.ctypes.data_as(i32p), None if ci_ is None else ci_.ctypes.data_as(i32p),
+                               rp.ctypes.data_as(i32p), cp.ctypes.data_as(i32p), bl.ctypes.data_as(i32p), ctypes.byref(kept)),
+           "pp_pivot_find")
+    return rp, cp, bl, kept.value

@@ -123,3 +123,28 @@ def test_listing1_rejects_what_it_cannot_run(pb):
     with pytest.raises(pb.PPError) as e:
         pb.Listing1(64, 4, 0, rp[:64][::-1] * 0, rp[:64], np.zeros(4 * 16 * 16, dtype=np.float32))
     assert e.value.status == 2
+
+
+def test_feed_back_search_to_layer(pb):
+    """Section 3.2 end to end: search the index arrays on |W| of a dense matrix with a hidden block structure,
+    keep the diagonal blocks, run the pruned layer, compare with the dense product of the pruned matrix."""
+    rng = np.random.default_rng(321)
+    M = N = 256
+    levels = 3
+    W = (rng.standard_normal((M, N)) * 0.01).astype(np.float32)
+    pr, pc = rng.permutation(M), rng.permutation(N)
+    e = M >> levels
+    for k in range(1 << levels):                       # heavy entries on hidden diagonal blocks
+        W[np.ix_(pr[k * e:(k + 1) * e], pc[k * e:(k + 1) * e])] += rng.standard_normal((e, e)).astype(np.float32)
+    rp, cp, bl, kept = pb.pp_pivot_find(np.abs(W), levels, 32, rng.permutation(M), rng.permutation(N))
+    assert kept > 0.9 * np.abs(W).sum()
+    vals = np.concatenate([W[np.ix_(rp[r0:r0 + h], cp[c0:c0 + w])].ravel() for r0, c0, h, w in bl]).astype(np.float32)
+    L = pb.Layer.from_blocks(M, N, 32, rp, cp, bl, vals)
+    x = rng.uniform(-1, 1, (2, N)).astype(np.float32)
+    y = pb.pp_forward(L, torch.from_numpy(x).cuda(), 0).cpu().numpy()
+    L.close()
+    Wp = po.reconstruct_blocks(M, N, rp, cp, bl, vals)
+    y_ref, _, a = po.dense_forward(Wp, None, x.astype(np.float64), 0)
+    assert np.all(np.abs(y - y_ref) <= 1e-5 * a + 1e-6)
+    mask = Wp != 0                                      # the pruned matrix is W on the kept entries, zero elsewhere
+    assert np.array_equal(Wp[mask], W.astype(np.float64)[mask])

@@ -65,3 +65,39 @@ def test_oracle_blocks_feed_the_block_layer_form():
     W = po.reconstruct_blocks(64, 64, rp, cp, bl, vals)
     assert W.sum() == kept
     assert np.array_equal(W != 0, (W == A) & (A != 0) & (W != 0))
+
+
+# ---------------------------------------------------------------- the library's routine against the oracle
+@pytest.mark.parametrize("M,N,levels,noise", [(64, 64, 2, 0.0), (96, 80, 3, 1.0), (50, 70, 2, 1.0), (128, 128, 4, 1.0)])
+def test_library_matches_oracle_bit_for_bit(M, N, levels, noise):
+    from paper_1712_01084_b200 import binding as pb
+    A, _ = _planted(100 + M, M, N, levels, noise=noise)          # small integers: every sum is exact
+    rng = np.random.default_rng(M)
+    r0, c0 = rng.permutation(M).astype(np.int32), rng.permutation(N).astype(np.int32)
+    rp, cp, bl, kept = pb.pp_pivot_find(A.astype(np.float32), levels, 32, r0, c0)
+    rp_o, cp_o, bl_o, kept_o = pv.pivot_find(A, levels, 32, r0, c0)
+    assert np.array_equal(rp, rp_o) and np.array_equal(cp, cp_o) and np.array_equal(bl, bl_o)
+    assert kept == kept_o
+
+
+def test_library_real_valued_input_is_valid_and_no_worse_than_start():
+    from paper_1712_01084_b200 import binding as pb
+    rng = np.random.default_rng(11)
+    A = np.abs(rng.standard_normal((120, 90))).astype(np.float32)
+    rp, cp, bl, kept = pb.pp_pivot_find(A, 2, 32, None, None)
+    assert sorted(rp) == list(range(120)) and sorted(cp) == list(range(90))
+    assert abs(kept - pv.kept_mass(A, rp, cp, bl)) <= 1e-9 * A.sum()
+    ident = pv.kept_mass(A, np.arange(120), np.arange(90), bl)
+    assert kept >= ident
+    assert kept > 0.25 * A.sum() * 1.15          # two bisections keep a quarter of the entries, but the heavier quarter
+
+
+def test_library_error_codes():
+    from paper_1712_01084_b200 import binding as pb
+    A = np.ones((8, 8), dtype=np.float32)
+    with pytest.raises(pb.PPError) as e:
+        pb.pp_pivot_find(A, 5, 4, None, None)            # more levels than the matrix can be halved
+    assert e.value.status == 1
+    with pytest.raises(pb.PPError) as e:
+        pb.pp_pivot_find(A, 1, 4, np.zeros(8, dtype=np.int32), None)
+    assert e.value.status == 2
