@@ -397,8 +397,9 @@ pp_status_t pp_forward_noalloc(const pp_packed_t* p, const void* device_image,
  * key 5: 0 = never use the persistent kernel, 1 = use it when batch <= 8 and x fits shared memory (default 1)
  * key 6: asynchronous 512-byte weight copies each warp of the persistent kernel keeps in flight: 4, 6 or 8;
  *        0 (default) = 4 when two CTAs fit an SM, else the deepest ring that fits
- * key 7: batch 1 in the persistent kernel: 1 (default) reads x through the index array inside the multiply
- *        loop, 0 permutes x into pivoted order in shared memory first (what batch 2..8 always do)
+ * key 7: how the persistent kernel applies the column permutation: 2 (default) reads x through the index
+ *        array inside the multiply loop for one input vector and, in fp16 layers, for 2..8 vectors; 1 does so
+ *        for one vector only; 0 always permutes x into pivoted order in shared memory first
  * key 8: 1 (default) launches the persistent kernel with programmatic stream serialization, 0 plainly
  * key 10: 1 (default) permutes multi-column inputs in a pre-pass kernel when the layer kernel cannot hold x
  *         twice in shared memory; 0 leaves the gather to the layer kernel; 2 always uses the pre-pass

@@ -257,7 +257,10 @@ pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ld
     int stage_mode = -1;
     const bool rows_aligned = aligned16(x) && (batch == 1 || ((size_t)ldx * x_elt) % 16 == 0);
     const bool has16 = gather && gather == L->d_gather && L->d_gather16;
-    const int fast = gather ? (batch == 1 && pp::g_stage_direct ? (has16 ? 4 : 3) : 1) : 2;
+    // reading x through the index array inside the multiply loop: always for one input vector, for several
+    // (fp16 layers) when tuning key 7 is 2
+    const bool direct = pp::g_stage_direct && (batch == 1 || (pp::g_stage_direct == 2 && pk->wdtype == PP_F16));
+    const int fast = gather ? (direct ? (has16 ? 4 : 3) : 1) : 2;
     if (rows_aligned && pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, fast) <= pp::kStreamSmemLimit)
         stage_mode = fast;
     else if (pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, 0) <= pp::kStreamSmemLimit)
@@ -298,7 +301,11 @@ pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx
         const int nb = batch < pp::kStreamMaxBatch ? batch : pp::kStreamMaxBatch;
         const bool fits = stream_path && aligned16(x) && ((size_t)ldx * x_elt) % 16 == 0 &&
                           pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, nb, 1) <= 113 * 1024;
-        if (!fits || pp::g_prepass == 2) {
+        const bool direct_ok = stream_path && pp::g_stage_direct == 2 && pk->wdtype == PP_F16 && aligned16(x) &&
+                               ((size_t)ldx * x_elt) % 16 == 0 && pp::g_prepass != 2 &&
+                               pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, nb,
+                                                     gather == L->d_gather && L->d_gather16 ? 4 : 3) <= pp::kStreamSmemLimit;
+        if ((!fits && !direct_ok) || pp::g_prepass == 2) {
             const int group = stream_path ? pp::kStreamMaxBatch : chunk_group;
             for (int b0 = 0; b0 < batch; b0 += group) {
                 const int gb = batch - b0 < group ? batch - b0 : group;

@@ -55,7 +55,6 @@ static_assert(sizeof(TileStep) == 32, "read as two 16-byte words");
 extern int g_tile_cluster;   // batched fp16 B = 64 layers: 0 one block-row per CTA, 2 the clustered kernel, 1 whichever fits the layer
 constexpr int kStreamWarps = 16;          // warps per CTA
 constexpr int kStreamMaxStrips = 48;      // strips one CTA may list
-constexpr int kStreamSegSlots = kStreamMaxStrips + kStreamWarps;   // (strip, warp) partial slots in shared memory
 constexpr int kStreamMaxBatch = 8;
 extern int g_use_stream;
 extern int g_tile_min_batch;  // fp16 B = 64 layers take the tensor-core tile path from this batch on (0: never)

@@ -16,7 +16,8 @@ int g_prepass = 1;
 int g_lstm_persist = 1;
 int g_tile_cluster = 1;
 int g_link_identity = 1;
-int g_stage_direct = 1;    // 0: batch 1 also materialises the pivoted x in shared memory
+int g_stage_direct = 2;    // 0: always materialise the pivoted x in shared memory; 1: one input vector is read through the
+                           // index array in the multiply loop; 2: so are 2..8 vectors of fp16 layers
 extern int g_stream_depth; // weight-ring slots per warp of the persistent kernel (pp_stream.cu)
 extern int g_stream_pdl;   // programmatic dependent launch of the persistent kernel (pp_stream.cu)
 }
@@ -309,7 +310,7 @@ pp_status_t pp_set_tuning(int key, int value) {
     if (key == 4 && value >= -1 && value <= 100) { g_stream_snap_pct = value; return PP_OK; }
     if (key == 5 && (value == 0 || value == 1)) { pp::g_use_stream = value; return PP_OK; }
     if (key == 6 && (value == 0 || value == 4 || value == 6 || value == 8)) { pp::g_stream_depth = value; return PP_OK; }
-    if (key == 7 && (value == 0 || value == 1)) { pp::g_stage_direct = value; return PP_OK; }
+    if (key == 7 && value >= 0 && value <= 2) { pp::g_stage_direct = value; return PP_OK; }
     if (key == 8 && (value == 0 || value == 1)) { pp::g_stream_pdl = value; return PP_OK; }
     if (key == 9 && value >= 0) { pp::g_tile_min_batch = value; return PP_OK; }
     if (key == 10 && value >= 0 && value <= 2) { pp::g_prepass = value; return PP_OK; }

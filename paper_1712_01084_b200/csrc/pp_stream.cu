@@ -79,7 +79,7 @@ struct SmemLayout {
     int4* sinfo;     // [kStreamMaxStrips] strip table entries of this CTA's strips
     int* rowdst;     // [max_rows] scatter_idx of this CTA's pivoted rows
     float* rowbias;  // [max_rows] bias_piv of this CTA's pivoted rows
-    float* segp;     // [kStreamSegSlots][RG][batch] parked partial sums
+    float* segp;     // [strips a CTA may list + kStreamWarps][RG][batch] parked partial sums (slot = local strip + warp)
     uint4* ring;     // [kStreamWarps][U][32] weight fragments in flight
     void* xs;        // staged pivoted x   [batch][xs_stride] (absent in staging mode 3)
     int* idxs;       // staging modes 1, 3: gather_idx [n_pad]
@@ -91,6 +91,12 @@ static_assert(kStreamMaxStrips <= 48, "header words 56..103 hold wlohi, 104..105
 
 __host__ __device__ __forceinline__ size_t xs_bytes(int batch, int xs_stride, int esz) {
     return ((size_t)batch * xs_stride * esz + 15) / 16 * 16;
+}
+
+// Bytes of the park slots: a CTA lists at most max_rows / rg strips and a warp parks in slot (local strip + warp);
+// rounded to 128 bytes so that the weight ring behind it keeps its alignment.
+__host__ __device__ __forceinline__ size_t segp_bytes(int max_rows, int rg, int batch) {
+    return ((size_t)(max_rows / rg + kStreamWarps) * rg * batch * 4 + 127) / 128 * 128;
 }
 
 __device__ __forceinline__ SmemLayout carve(unsigned char* base, int rg, int U, const StreamArgs& a, int esz) {
@@ -105,7 +111,7 @@ __device__ __forceinline__ SmemLayout carve(unsigned char* base, int rg, int U, 
     L.rowdst = reinterpret_cast<int*>(base + kHeaderBytes);
     L.rowbias = reinterpret_cast<float*>(L.rowdst + a.max_rows);
     L.segp = L.rowbias + a.max_rows;
-    L.ring = reinterpret_cast<uint4*>(L.segp + kStreamSegSlots * rg * a.batch);
+    L.ring = reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(L.segp) + segp_bytes(a.max_rows, rg, a.batch));
     unsigned char* p = reinterpret_cast<unsigned char*>(L.ring + kStreamWarps * U * 32);
     L.xs = p;
     if (a.stage_mode < 3) p += xs_bytes(a.batch, a.xs_stride, esz);
@@ -208,7 +214,7 @@ __device__ __forceinline__ void finish_stage(const StreamArgs& a, const SmemLayo
         const int dst_stride = via_raw ? a.raw_stride : a.xs_stride;
         const int n_src = via_raw ? a.x_len : a.x_limit;
         const int n_dst = via_raw ? a.x_len : a.n_pad;
-        if (a.stage_mode >= 3 && tid == 0) dst[-1] = T(0.0f);
+        if (a.stage_mode >= 3 && tid < a.batch) dst[tid * dst_stride - 1] = T(0.0f);   // what index -1 reads, in front of every row
         const int done = n_src / EPC * EPC;
         for (int b = 0; b < a.batch; ++b)
             for (int j = done + tid; j < n_dst; j += kThreads)
@@ -504,19 +510,41 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
             mb0 = (uint32_t)rawu[i0.x] | ((uint32_t)rawu[i0.y] << 16);
             mb1 = (uint32_t)rawu[i1.x] | ((uint32_t)rawu[i1.y] << 16);
         };
+        // Several input vectors read through the index array: lane (g, t) fetches its own four entries of
+        // input row g for every fragment (no pivoted copy of x in shared memory, no permutation pass).
+        const bool direct1 = direct && a.batch == 1;
+        const unsigned short* rawg = rawu + g * a.raw_stride;
+        auto gather_row = [&](int xo, uint32_t& b0, uint32_t& b1) {
+            if (!has_x) return;
+            int2 i0, i1;
+            if (idx16) {
+                const uint16_t* t16 = reinterpret_cast<const uint16_t*>(L.idxs) + xo + 2 * t;
+                const uint32_t p0 = *reinterpret_cast<const uint32_t*>(t16);
+                const uint32_t p1 = *reinterpret_cast<const uint32_t*>(t16 + 8);
+                i0 = make_int2((int)(p0 & 0xffffu) - 1, (int)(p0 >> 16) - 1);
+                i1 = make_int2((int)(p1 & 0xffffu) - 1, (int)(p1 >> 16) - 1);
+            } else {
+                i0 = *reinterpret_cast<const int2*>(L.idxs + xo + 2 * t);
+                i1 = *reinterpret_cast<const int2*>(L.idxs + xo + 2 * t + 8);
+            }
+            b0 = (uint32_t)rawg[i0.x] | ((uint32_t)rawg[i0.y] << 16);
+            b1 = (uint32_t)rawg[i1.x] | ((uint32_t)rawg[i1.y] << 16);
+        };
         // Fragments are taken in groups of GRP; fragment wbeg + i sits in ring slot i % U.  A group of 8
         // that lies inside one strip, with all its refills inside the warp's range, runs without any
         // per-fragment test (the common case: a strip is hundreds of fragments long).
         constexpr int GRP = (8 % U == 0) ? 8 : U;
         for (int base = wbeg; base < wend; base += GRP) {
             if (GRP == 8 && base + 8 + U <= wend && base + 8 <= seg_end) {
-                if (direct) gather8(base);
+                if (direct1) gather8(base);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     uint32_t b0 = 0u, b1 = 0u;
-                    if (direct) {
+                    if (direct1) {
                         b0 = __shfl_sync(0xffffffffu, mb0, j * 4 + t);
                         b1 = __shfl_sync(0xffffffffu, mb1, j * 4 + t);
+                    } else if (direct) {
+                        gather_row(xw.get(base + j, wend, lane), b0, b1);
                     } else {
                         const int xoff = xw.get(base + j, wend, lane);
                         if (has_x) {
@@ -541,11 +569,13 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
                         seg_end = min(wend, L.sstart[ls + 1]);
                     }
                     uint32_t b0 = 0u, b1 = 0u;
-                    if (direct) {
+                    if (direct1) {
                         const int in_group = (p - wbeg) & 7;
                         if (in_group == 0) gather8(p);
                         b0 = __shfl_sync(0xffffffffu, mb0, in_group * 4 + t);
                         b1 = __shfl_sync(0xffffffffu, mb1, in_group * 4 + t);
+                    } else if (direct) {
+                        gather_row(xw.get(p, wend, lane), b0, b1);
                     } else {
                         const int xoff = xw.get(p, wend, lane);        // warp-wide shuffle: outside the lane test
                         if (has_x) {
@@ -692,6 +722,10 @@ cudaError_t launch_f32(const StreamLaunch& P, int grid, size_t smem, cudaStream_
     return launch_one<stream_f32_kernel<RG, 8, U>>(P, grid, smem, stream);
 }
 
+// Row stride (elements) of the shared-memory copy of x as given.  With several rows, 8 elements more than the
+// 16-element multiple: the rows then start 4 (fp16) or 8 (fp32) banks apart instead of in the same bank, which
+// matters when lanes of different rows read the same column.
+int raw_stride_for(int x_len, int batch) { return (x_len + 15) / 16 * 16 + (batch > 1 ? 8 : 0); }
 int xs_stride_for(pp_dtype_t dt, int n_pad) { return dt == PP_F16 ? n_pad + 8 : n_pad + 4; }
 
 }  // namespace
@@ -725,11 +759,12 @@ namespace {
 size_t smem_bytes_at(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int depth) {
     const int rg = frag_geom(dt, B).rg_rows;
     const int esz = dt == PP_F16 ? 2 : 4;
-    size_t bytes = (size_t)kHeaderBytes + (size_t)max_rows * 8 + (size_t)kStreamSegSlots * rg * batch * 4 +
+    max_rows = (max_rows + 31) / 32 * 32;          // as the launcher rounds it
+    size_t bytes = (size_t)kHeaderBytes + (size_t)max_rows * 8 + segp_bytes(max_rows, rg, batch) +
                    (size_t)kStreamWarps * depth * 512;
     if (stage_mode < 3) bytes += xs_bytes(batch, xs_stride_for(dt, n_pad), esz);
     if (stage_mode == 1 || stage_mode >= 3)
-        bytes += (size_t)n_pad * (stage_mode == 4 ? 2 : 4) + 16 + (size_t)batch * ((x_len + 15) / 16 * 16) * esz;
+        bytes += (size_t)n_pad * (stage_mode == 4 ? 2 : 4) + 16 + (size_t)batch * raw_stride_for(x_len, batch) * esz;
     return bytes;
 }
 }  // namespace
@@ -740,12 +775,12 @@ cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a_in, const Ct
     StreamLaunch P;
     P.a = a_in;
     StreamArgs& a = P.a;
-    if (a.batch < 1 || a.batch > kStreamMaxBatch || (a.stage_mode >= 3 && a.batch != 1) ||
+    if (a.batch < 1 || a.batch > kStreamMaxBatch || (a.stage_mode >= 3 && a.batch != 1 && dt != PP_F16) ||
         (a.stage_mode == 4 && !a.gather16))
         return cudaErrorInvalidValue;
     a.xs_stride = xs_stride_for(dt, a.n_pad);
-    a.raw_stride = (a.x_len + 15) / 16 * 16;
-    a.max_rows = (a.max_rows + 3) / 4 * 4;
+    a.raw_stride = raw_stride_for(a.x_len, a.batch);
+    a.max_rows = (a.max_rows + 31) / 32 * 32;      // whole strips of either height; keeps the regions behind 128-byte aligned
     if (grid <= kParamCtas)
         for (int c = 0; c < grid; ++c) P.table[c] = host_table[c];
     const int depth = stream_pick_depth(dt, B, a.n_pad, a.x_len, a.max_rows, a.batch, a.stage_mode, grid);

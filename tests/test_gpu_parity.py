@@ -98,7 +98,7 @@ def test_persistent_kernel_batch1_variants(pb, dtype, B, direct, depth):
         for act in (0, 1):
             _run_and_check(pb, lay, x, act, f"direct={direct} depth={depth} B={B}")
     finally:
-        pb.pp_set_tuning(7, 1); pb.pp_set_tuning(6, 0)
+        pb.pp_set_tuning(7, 2); pb.pp_set_tuning(6, 0)
 
 
 @pytest.mark.parametrize("dtype", [np.float32, np.float16])
@@ -520,3 +520,26 @@ def test_forward_host_matches_device_call(pb):
         y_ref, _, a = po.layer_forward(lay, x.astype(np.float64), act=1, threads=4)
         _check(yh.numpy(), y_ref, a, np.float16, f"host call batch {batch}")
     L.close()
+
+
+@pytest.mark.parametrize("B", [16, 32, 64])
+@pytest.mark.parametrize("batch", [2, 3, 5, 8])
+@pytest.mark.parametrize("key7", [2, 1])
+def test_several_vectors_through_the_index_array(pb, B, batch, key7):
+    """fp16, 2..8 input vectors: read through the column index array inside the multiply loop (tuning key 7 = 2,
+    the default: no pivoted copy of x, no pre-pass) or permuted in shared memory first (key 7 = 1); ragged N,
+    padding columns, a block-row without tiles; real values within tolerance and small integers bit for bit."""
+    pb.pp_set_tuning(7, key7)
+    try:
+        for integer in (False, True):
+            lay = _rand_layer(900 + B + batch, 6 * B - 5, 10 * B - 3, B, np.float16, density=0.5, empty_rows=(1,),
+                              integer=integer)
+            rng = np.random.default_rng(batch)
+            x = (rng.integers(-2, 3, (batch, lay.N)) if integer else rng.uniform(-1, 1, (batch, lay.N))).astype(np.float16)
+            for act in (0, 1):
+                y = _run_and_check(pb, lay, x, act, f"direct multi B={B} batch={batch}")
+                if integer:
+                    y_ref, _, _ = po.layer_forward(lay, x.astype(np.float64), act=act)
+                    assert np.array_equal(y.astype(np.float64), y_ref)
+    finally:
+        pb.pp_set_tuning(7, 2)
