@@ -274,9 +274,10 @@ def test_config5_batch1_full(pb, k):
     _run_and_check(pb, wl.layers[0], wl.x, 0, f"config 5 k={k}")
 
 
-@pytest.mark.parametrize("batch", [16])
+@pytest.mark.parametrize("batch", [2, 4, 8, 16])
 def test_config5_small_batch_sampled_rows(pb, batch):
-    """Full size; the oracle evaluates a sample of output rows."""
+    """Full size; the oracle evaluates a sample of output rows.  Batch 2..8 runs the persistent kernel with x read
+    through the index array (one CTA per SM from batch 3 on: two waves of the 296-CTA plan), 16 the tile path."""
     wl = synth.config5(k=32, batch=batch)
     lay = wl.layers[0]
     L = pb.Layer.from_synth(lay)
@@ -284,7 +285,7 @@ def test_config5_small_batch_sampled_rows(pb, batch):
     W = po.reconstruct(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values)
     rows = np.random.default_rng(0).choice(lay.M, 256, replace=False).astype(np.int32)
     y_ref, a = po.dense_forward_rows(W, None, wl.x.astype(np.float64), 0, rows)
-    _check(y[:, rows], y_ref, a, np.float16, "config 5 batch 16 sampled")
+    _check(y[:, rows], y_ref, a, np.float16, f"config 5 batch {batch} sampled")
     L.close()
 
 
