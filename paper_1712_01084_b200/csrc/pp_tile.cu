@@ -554,32 +554,35 @@ __global__ void gather_x_kernel(const __half* __restrict__ x, int ldx, int n, co
     extern __shared__ __half row[];
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the tile kernel may set up meanwhile
     const int b = blockIdx.x;
-    if (b < batch) {
+    if (b >= batch) return;
+    // A thread produces whole 16-byte chunks of the destination (8 consecutive pivoted columns).  The index
+    // entries of its first chunk are requested before the row itself, so that the two round trips overlap.
+    const int n_chunks = n_pad / 8;
+    const int4* idx4 = reinterpret_cast<const int4*>(gather_idx);
+    int i = threadIdx.x;
+    int4 ia = make_int4(-1, -1, -1, -1), ib = ia;
+    if (i < n_chunks) { ia = __ldg(idx4 + 2 * i); ib = __ldg(idx4 + 2 * i + 1); }
+    {
         // 16-byte copies where the row allows it (base and pitch 16-byte aligned), element copies otherwise
         const __half* src = x + (size_t)b * ldx;
         const bool vec = ((reinterpret_cast<uintptr_t>(src) & 15u) == 0);
         const int n8 = vec ? n / 8 : 0;
-        for (int i = threadIdx.x; i < n8; i += blockDim.x)
-            reinterpret_cast<uint4*>(row)[i] = __ldg(reinterpret_cast<const uint4*>(src) + i);
+        for (int c = threadIdx.x; c < n8; c += blockDim.x)
+            reinterpret_cast<uint4*>(row)[c] = __ldg(reinterpret_cast<const uint4*>(src) + c);
         for (int j = n8 * 8 + threadIdx.x; j < n; j += blockDim.x) row[j] = src[j];
     }
     __syncthreads();
-    // 8 independent index loads per thread before the first use, so their latencies overlap
-    for (int j0 = threadIdx.x; j0 < n_pad; j0 += 8 * blockDim.x) {
-        int idx[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int j = j0 + q * blockDim.x;
-            idx[q] = (b < batch && j < n_pad) ? __ldg(gather_idx + j) : -1;
-        }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int j = j0 + q * blockDim.x;
-            if (j < n_pad) {
-                const __half v = idx[q] >= 0 ? row[idx[q]] : __float2half(0.0f);
-                *reinterpret_cast<__half*>(x_sw + (size_t)(j >> 6) * kXBytes + sw128_offset(b, j & 63)) = v;
-            }
-        }
+    const unsigned short* rowu = reinterpret_cast<const unsigned short*>(row);
+    auto pick = [&](int idx) { return idx >= 0 ? (uint32_t)rowu[idx] : 0u; };
+    for (bool first = true; i < n_chunks; i += blockDim.x, first = false) {
+        if (!first) { ia = __ldg(idx4 + 2 * i); ib = __ldg(idx4 + 2 * i + 1); }
+        uint4 v;
+        v.x = pick(ia.x) | (pick(ia.y) << 16);
+        v.y = pick(ia.z) | (pick(ia.w) << 16);
+        v.z = pick(ib.x) | (pick(ib.y) << 16);
+        v.w = pick(ib.z) | (pick(ib.w) << 16);
+        const int j = 8 * i;
+        *reinterpret_cast<uint4*>(x_sw + (size_t)(j >> 6) * kXBytes + sw128_offset(b, j & 63)) = v;
     }
 }
 
