@@ -9,7 +9,7 @@
 //     already has the 128-byte-swizzled shared-memory image the tensor core wants; the packer stores
 //     every weight tile as such an image (8 KiB) too;
 //   * warps 0..3 (one lane each) stream (X block, W tile) pairs into a ring of shared-memory stages
-//     with two bulk asynchronous copies per tile (cp.async.bulk, one request each, no multicast),
+//     with two bulk asynchronous copies per tile (cp.async.bulk, one request each, every CTA fetching for itself),
 //     signalling mbarriers (2-D tensor-map loads of 128-byte rows were request-rate bound: 60 us vs
 //     the same data as two contiguous copies);
 //   * warp 4 issues tcgen05.mma (kind::f16, accumulator in tensor memory) from shared-memory matrix
