@@ -136,14 +136,24 @@ def run_reference(args, rank):
     cores = os.cpu_count() or 1
     W = po.reconstruct(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values)
     x64 = wl.x.astype(np.float64)
+    po.dense_forward(W, None, x64, lay.act, threads=cores)
     t0 = time.perf_counter()
     po.dense_forward(W, None, x64, lay.act, threads=cores)
     t_full = time.perf_counter() - t0
-    # each step is a sample of output rows sized so that the whole run stays near two minutes
+    # each step is the whole layer on all cores when that fits the budget of one step, else a sample of output
+    # rows (one thread) sized from a timed probe, so that the whole run stays near two minutes
     budget = 120.0 / max(1, args.steps + args.warmup)
-    frac = min(1.0, budget / max(t_full, 1e-9))
-    n_rows = max(8, int(lay.M * frac))
-    rows = np.random.default_rng(0).choice(lay.M, n_rows, replace=False).astype(np.int32)
+    rows_all = np.random.default_rng(0).permutation(lay.M).astype(np.int32)
+    if t_full <= budget:
+        n_rows = lay.M
+    else:
+        probe = rows_all[:64]
+        po.dense_forward_rows(W, None, x64, lay.act, probe)
+        t0 = time.perf_counter()
+        po.dense_forward_rows(W, None, x64, lay.act, probe)
+        t_row = (time.perf_counter() - t0) / probe.size
+        n_rows = int(min(lay.M, max(1, budget / max(t_row, 1e-9))))
+    rows = rows_all[:n_rows].copy()
     run = (lambda: po.dense_forward(W, None, x64, lay.act, threads=cores)) if n_rows >= lay.M else \
           (lambda: po.dense_forward_rows(W, None, x64, lay.act, rows))
     used = cores if n_rows >= lay.M else 1
