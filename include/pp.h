@@ -379,12 +379,22 @@ pp_status_t pp_listing1_forward(pp_listing1_t* h, const float* x, float* y, void
  * The first call on a device looks up the array's device address; make that call
  * before any stream capture.  All calls on a device share the array: it is re-
  * initialised by two memsets enqueued ahead of the kernel, and two calls that
- * overlap on the GPU (different streams) race on it. */
+ * overlap on the GPU (different streams) race on it.
+ * pp_noalloc_status reports (and clears) the time-out flag of the current device's
+ * pp_forward_noalloc kernels: *status is PP_ERR_TIMEOUT when a kernel's bounded wait
+ * for the copy of x gave up since the last query (that call's y is invalid), else
+ * PP_OK.  It synchronises with the device and allocates nothing either. */
 pp_status_t pp_pack_device_image_bytes(const pp_packed_t* p, int64_t* bytes);
 pp_status_t pp_pack_device_image(const pp_packed_t* p, void* host_dst, int64_t bytes);
 pp_status_t pp_forward_noalloc(const pp_packed_t* p, const void* device_image,
                                const void* x, void* y, int batch, pp_act_t act,
                                void* cuda_stream);
+pp_status_t pp_noalloc_status(pp_status_t* status);
+
+/* Self-check of host-side bookkeeping that needs no GPU (the table that remembers, per device, which kernels
+ * already have their shared-memory opt-in): PP_OK, or PP_ERR_INVALID_ARG when a check fails.  One process may
+ * drive several GPUs; every kernel attribute is set once per device. */
+pp_status_t pp_selftest_host(void);
 
 /* Tuning knobs read at pack / create time (process-wide; for experiments).
  * key 0: target kilobytes of tile values per work item (default 32)

@@ -5,7 +5,7 @@ Section 3.2 describes the search only in words: take the absolute values of a tr
 pick the row and column permutations that maximise the sum of the entries landing in the upper-left and
 the lower-right sub-block, by a greedy optimisation started from randomly chosen permutations; the
 entries of the two off-diagonal sub-blocks are deleted (half of the block); repeat on every remaining
-block ("the number of blocks doubles after each bisection").  The reading implemented here, step by step:
+block, so that every level has twice as many blocks as the one before (Section 3.2).  The reading implemented here, step by step:
 
   one bisection of a block (rows R, columns C of the current pivoted order, |R| = m, |C| = n):
     side 0 holds the first ceil(m/2) rows / ceil(n/2) columns, side 1 the rest (the starting

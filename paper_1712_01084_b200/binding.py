@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
         "pp_pack_device_image_bytes": (ci, [vp, i64p]),
         "pp_pack_device_image": (ci, [vp, vp, c64]),
         "pp_forward_noalloc": (ci, [vp, vp, vp, vp, ci, ci, vp]),
+        "pp_noalloc_status": (ci, [ctypes.POINTER(ci)]),
+        "pp_selftest_host": (ci, []),
     }
     for name, (res, args) in sig.items():
         fn = getattr(L, name)
@@ -420,6 +422,13 @@ def pp_forward_noalloc(packed: Packed, device_image, x, act: int = PP_ACT_IDENTI
                                     ctypes.c_void_p(x2.data_ptr()), ctypes.c_void_p(out.data_ptr()),
                                     batch, int(act), _stream_ptr(stream)), "pp_forward_noalloc")
     return out
+
+
+def pp_noalloc_status() -> int:
+    """Time-out flag of the current device's pp_forward_noalloc kernels (PP_OK or PP_ERR_TIMEOUT); cleared by the read."""
+    st = ctypes.c_int(0)
+    _check(lib().pp_noalloc_status(ctypes.byref(st)), "pp_noalloc_status")
+    return st.value
 
 
 class Chain:

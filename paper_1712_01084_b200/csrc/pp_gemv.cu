@@ -287,12 +287,17 @@ __global__ void __launch_bounds__(kThreads) gemv_f32_kernel(const GemvArgs a) {
 
 template <auto Kernel>
 cudaError_t launch_one(const GemvArgs& a, int n_items, size_t smem, cudaStream_t stream) {
-    static bool configured = false;   // one flag per kernel instantiation (Kernel is a template argument)
+    static PerDeviceOnce configured;   // one table per kernel instantiation (Kernel is a template argument)
     if (smem > 200 * 1024) return cudaErrorInvalidValue;
-    if (!configured && smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (smem > 48 * 1024) {
+        int dev = -1;
+        cudaError_t e = cudaGetDevice(&dev);
         if (e != cudaSuccess) return e;
-        configured = true;
+        if (!configured.is_done(dev)) {
+            e = cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e != cudaSuccess) return e;
+            configured.mark(dev);
+        }
     }
     Kernel<<<n_items, kThreads, smem, stream>>>(a);
     return cudaGetLastError();

@@ -63,6 +63,16 @@ extern int g_link_identity;  // 1: chain links whose folded map is the identity 
 extern int g_lstm_persist;  // 1: recurrent cells run all steps in one cooperative kernel when the gate weights fit shared memory
 extern int g_stage_direct;   // batch 1: read x through the index array instead of permuting it first
 
+// "Done once" bookkeeping for settings that belong to a device, not to the process (the opt-in to more than
+// 48 KiB of dynamic shared memory, cudaFuncSetAttribute, is one): one flag per device ordinal.  Ordinals beyond
+// the table are never marked, so the setting is simply applied again on every launch there.
+struct PerDeviceOnce {
+    static constexpr int kMaxDevices = 64;
+    bool done[kMaxDevices] = {};
+    bool is_done(int dev) const { return dev >= 0 && dev < kMaxDevices && done[dev]; }
+    void mark(int dev) { if (dev >= 0 && dev < kMaxDevices) done[dev] = true; }
+};
+
 // Geometry of the fragment layout for a (dtype, B) pair.
 struct FragGeom {
     int rg_rows;   // rows covered by one fragment (row-group height)

@@ -1,7 +1,7 @@
 // Recurrent use of one pivoted gate layer as an LSTM cell: z_t = [x_t ; h_{t-1}], g = W z_t,
 // original rows [0,H) input gate, [H,2H) forget gate, [2H,3H) candidate, [3H,4H) output gate;
-// c_t = sig(f) c_{t-1} + sig(i) tanh(g), h_t = sig(o) tanh(c_t); no bias.  (The paper only names
-// recurrent networks as users of FC layers; the cell is the workload's definition.)
+// c_t = sig(f) c_{t-1} + sig(i) tanh(g), h_t = sig(o) tanh(c_t); a bias given to the layer is part of g.
+// (The paper only names recurrent networks as users of FC layers; the cell is the workload's definition.)
 //
 // Cross-layer permutation fusion (Section 4.2.1) applied to the recurrence: the layer input lives
 // in the layer's pivoted column order for all steps, so the matrix-vector kernel copies it without
@@ -285,11 +285,14 @@ size_t lstm_persist_smem(int max_frags, int n_pad, int m_pad) {
 }
 
 cudaError_t launch_lstm_persist(const LstmPersistArgs& a_in, int grid, size_t smem, cudaStream_t stream) {
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(lstm_persist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+    static PerDeviceOnce configured;
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (!configured.is_done(dev)) {
+        e = cudaFuncSetAttribute(lstm_persist_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured.mark(dev);
     }
     LstmPersistArgs a = a_in;
     void* args[] = {&a};

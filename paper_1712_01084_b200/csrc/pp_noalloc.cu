@@ -19,23 +19,32 @@ namespace {
 constexpr size_t kStaticScratchBytes = 1u << 20;   // 1 MiB per GPU, shared by every call
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
+// Raised by the kernel when its bounded wait for the copy of x gives up (the output of that call is invalid).
+static __device__ __align__(16) int g_static_status;
+
 constexpr int kMaxDevices = 64;
 unsigned char* g_scratch_addr[kMaxDevices] = {};   // device address of g_static_scratch, per device
+int* g_status_addr[kMaxDevices] = {};              // device address of g_static_status, per device
 
 // The array's name is only a host-side handle; its device address must be asked for, once per
 // device, with that device current.
-cudaError_t scratch_address(unsigned char** out) {
+cudaError_t scratch_address(unsigned char** out, int** status_out) {
     int dev = -1;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    if (!g_scratch_addr[dev]) {
+    if (!g_scratch_addr[dev] || !g_status_addr[dev]) {
         void* p = nullptr;
         e = cudaGetSymbolAddress(&p, g_static_scratch);
         if (e != cudaSuccess) return e;
+        void* q = nullptr;
+        e = cudaGetSymbolAddress(&q, g_static_status);
+        if (e != cudaSuccess) return e;
         g_scratch_addr[dev] = static_cast<unsigned char*>(p);
+        g_status_addr[dev] = static_cast<int*>(q);
     }
     *out = g_scratch_addr[dev];
+    *status_out = g_status_addr[dev];
     return cudaSuccess;
 }
 
@@ -114,7 +123,8 @@ pp_status_t pp_forward_noalloc(const pp_packed_t* p, const void* device_image, c
     if (stage_mode < 0) return PP_ERR_UNSUPPORTED;
 
     unsigned char* scratch = nullptr;
-    if (scratch_address(&scratch) != cudaSuccess) { cudaGetLastError(); return PP_ERR_CUDA; }
+    int* status_word = nullptr;
+    if (scratch_address(&scratch, &status_word) != cudaSuccess) { cudaGetLastError(); return PP_ERR_CUDA; }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     // the array keeps whatever the last call left: exchange slots must rest at all ones, counters at zero
     if (slot_bytes && cudaMemsetAsync(scratch, 0xff, slot_bytes, stream) != cudaSuccess) return PP_ERR_CUDA;
@@ -135,10 +145,28 @@ pp_status_t pp_forward_noalloc(const pp_packed_t* p, const void* device_image, c
     s.x = x; s.y = y;
     s.partials = reinterpret_cast<float*>(scratch);
     s.counters = reinterpret_cast<int*>(scratch + slot_bytes);
+    s.status = status_word;
     s.ldx = p->N; s.ldy = p->M; s.x_limit = p->N; s.n_pad = p->Npad; s.x_len = p->N; s.max_rows = max_rows;
     s.batch = batch; s.act = (int)act; s.out_mode = pp::OUT_SCATTER_F32;
     return pp::launch_stream(p->wdtype, p->B, s, p->cta_desc.data(), (int)p->cta_desc.size(), stream) == cudaSuccess
                ? PP_OK : PP_ERR_CUDA;
+}
+
+// PP_ERR_TIMEOUT when a pp_forward_noalloc kernel on the current device gave up its bounded wait since the
+// last query; the word is cleared by the read.  Synchronises with the device; allocates nothing.
+pp_status_t pp_noalloc_status(pp_status_t* status) {
+    if (!status) return PP_ERR_INVALID_ARG;
+    *status = PP_OK;
+    unsigned char* scratch = nullptr;
+    int* status_word = nullptr;
+    if (scratch_address(&scratch, &status_word) != cudaSuccess) { cudaGetLastError(); return PP_ERR_CUDA; }
+    int flag = 0;
+    if (cudaMemcpy(&flag, status_word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return PP_ERR_CUDA;
+    if (flag) {
+        *status = PP_ERR_TIMEOUT;
+        if (cudaMemset(status_word, 0, sizeof(int)) != cudaSuccess) return PP_ERR_CUDA;
+    }
+    return PP_OK;
 }
 
 }  // extern "C"

@@ -302,6 +302,22 @@ static void build_tile_steps(pp_packed* p) {
     }
 }
 
+// Host-side self-check (no GPU): the per-device "done once" table keeps devices apart, ignores ordinals it has
+// no slot for (the setting is then re-applied on every launch there) and starts empty.
+pp_status_t pp_selftest_host(void) {
+    pp::PerDeviceOnce t;
+    for (int d = -1; d <= pp::PerDeviceOnce::kMaxDevices; ++d)
+        if (t.is_done(d)) return PP_ERR_INVALID_ARG;
+    t.mark(0);
+    if (!t.is_done(0) || t.is_done(1)) return PP_ERR_INVALID_ARG;
+    t.mark(3);
+    t.mark(-1);
+    t.mark(pp::PerDeviceOnce::kMaxDevices);
+    for (int d = -1; d <= pp::PerDeviceOnce::kMaxDevices; ++d)
+        if (t.is_done(d) != (d == 0 || d == 3)) return PP_ERR_INVALID_ARG;
+    return PP_OK;
+}
+
 pp_status_t pp_set_tuning(int key, int value) {
     if (key == 0 && value >= 1) { g_target_kib = value; return PP_OK; }
     if (key == 1 && value >= 0) { g_min_items = value; return PP_OK; }

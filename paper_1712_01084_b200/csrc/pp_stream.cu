@@ -16,7 +16,7 @@
 //     shared-memory permutation of x behind the outstanding weight loads);
 //   * where a warp's range crosses a strip boundary it parks the finished 16(32)-row partial sum
 //     in shared memory; after the final barrier the CTA adds the parks of every strip in warp
-//     order.  A strip shared by several CTAs (Section 4.1.5's "additional reduction step") goes
+//     order.  A strip shared by several CTAs (the extra sum Section 4.1.5 asks for where blocks share rows) goes
 //     through one global partial sum per CTA, added in CTA order by the last CTA to arrive.
 //   * everything the epilogue needs (row index array, pivoted bias, strip table) is fetched
 //     asynchronously at kernel start, so the tail is shared-memory work plus the stores;
@@ -693,13 +693,17 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const __grid_co
 
 template <auto Kernel>
 cudaError_t launch_one(const StreamLaunch& P, int grid, size_t smem, cudaStream_t stream) {
-    static bool configured = false;   // one flag per kernel instantiation
+    static PerDeviceOnce configured;   // one table per kernel instantiation; the attribute belongs to the device
     if (smem > kStreamSmemLimit) return cudaErrorInvalidValue;
-    if (!configured && smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)kStreamSmemLimit);
+    if (smem > 48 * 1024) {
+        int dev = -1;
+        cudaError_t e = cudaGetDevice(&dev);
         if (e != cudaSuccess) return e;
-        configured = true;
+        if (!configured.is_done(dev)) {
+            e = cudaFuncSetAttribute(Kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStreamSmemLimit);
+            if (e != cudaSuccess) return e;
+            configured.mark(dev);
+        }
     }
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid);

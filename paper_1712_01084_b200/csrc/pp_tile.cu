@@ -615,12 +615,15 @@ static cudaError_t launch_after_gather(void (*kernel)(const TileArgs), int grid,
 
 template <int STAGES, int XB>
 cudaError_t launch_one_row(const TileArgs& a, int Mb, cudaStream_t stream) {
-    static bool configured = false;
+    static PerDeviceOnce configured;
     const size_t smem = (size_t)STAGES * (XB + kWBytes) + (kXBytes - XB) + sizeof(TileSmem<STAGES>) + 1024;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(tile_f16_kernel<STAGES, XB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (!configured.is_done(dev)) {
+        e = cudaFuncSetAttribute(tile_f16_kernel<STAGES, XB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        configured = true;
+        configured.mark(dev);
     }
     return launch_after_gather(tile_f16_kernel<STAGES, XB>, Mb, kThreads, smem, a, stream);
 }
@@ -636,12 +639,15 @@ cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const 
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (use_cluster && a.steps && a.parts) {
-        static bool configured_c = false;
+        static PerDeviceOnce configured_c;
         const size_t smem_c = (size_t)kCStages * kCStageBytes + sizeof(ClusterSmem) + 1024;
-        if (!configured_c) {
+        int dev = -1;
+        e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (!configured_c.is_done(dev)) {
             e = cudaFuncSetAttribute(tile_cluster_f16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_c);
             if (e != cudaSuccess) return e;
-            configured_c = true;
+            configured_c.mark(dev);
         }
         const int groups = (Mb + kTileRows - 1) / kTileRows;
         return launch_after_gather(tile_cluster_f16_kernel, groups * kTileRows, kCThreads, smem_c, a, stream);

@@ -86,7 +86,11 @@ def test_lstm_free_running_256_steps(pb, cell_mode):
     dh = np.max(np.abs(h.cpu().numpy().astype(np.float64) - h_ref))
     dc = np.max(np.abs(c.cpu().numpy().astype(np.float64) - c_ref))
     print(f"free-running drift after 256 steps: max |dh| = {dh:.3e}, max |dc| = {dc:.3e}")
-    assert dh < 2e-3 and dc < 2e-3
+    # No bound follows from the paper (the cell is the workload's).  Both sides round h_t to binary16 after every
+    # step, so the outputs differ by what the fp32 gate arithmetic and the hardware exponential leave (measured
+    # 6.1e-5 on h, 1.4e-6 on c) unless a value lands on the other side of a rounding boundary: one binary16
+    # step below 1 is 4.9e-4.  Limits: that one step for h (8 x the measured drift), 14 x the measured drift for c.
+    assert dh < 5e-4 and dc < 2e-5
     # run it again from zero: identical bits (deterministic kernels, scratch left clean)
     h2 = torch.zeros_like(h); c2 = torch.zeros_like(c)
     pb.pp_lstm_forward(cell, torch.from_numpy(wl.x).cuda(), h2, c2)
@@ -111,8 +115,10 @@ def test_lstm_ragged_strip_counts_and_bias(pb, H, I, B, density, cell_mode):
     pb.pp_lstm_forward(cell, torch.from_numpy(x_seq).cuda(), h, c)
     hr, cr, _ = po.lstm_forward(_dense(lay), x_seq.astype(np.float64), H, h_round="f16", threads=4,
                                 h0=h0, c0=c0, bias=lay.bias.astype(np.float64))
-    assert np.max(np.abs(h.cpu().numpy().astype(np.float64) - hr)) < 4e-3
-    assert np.max(np.abs(c.cpu().numpy().astype(np.float64) - cr)) < 4e-3
+    eh = np.max(np.abs(h.cpu().numpy().astype(np.float64) - hr))
+    ec = np.max(np.abs(c.cpu().numpy().astype(np.float64) - cr))
+    print(f"ragged cell H={H}: max |dh| = {eh:.3e}, max |dc| = {ec:.3e}")
+    assert eh < 4e-3 and ec < 4e-3
     assert cell.status() == 0
     cell.close(); L.close()
 

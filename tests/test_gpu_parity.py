@@ -268,10 +268,26 @@ def test_chain_matches_layer_by_layer_bits(pb):
     chain.close()
 
 
-@pytest.mark.parametrize("k", [128, 16, 8])
+@pytest.mark.parametrize("k", [128, 64, 32, 16, 8])
 def test_config5_batch1_full(pb, k):
     wl = synth.config5(k=k, batch=1)
     _run_and_check(pb, wl.layers[0], wl.x, 0, f"config 5 k={k}")
+
+
+@pytest.mark.parametrize("k,batch", [(128, 16), (128, 128), (64, 128), (32, 16), (8, 128), (8, 16)])
+def test_config5_batched_full(pb, k, batch):
+    """Full size, every output row of every input vector against the fp64 product, with the kernel choice left
+    on automatic: the launch configurations the benchmark times (density 1 takes the clustered tensor-core
+    kernel, sparse layers the one-block-row kernel)."""
+    import os
+    wl = synth.config5(k=k, batch=batch)
+    lay = wl.layers[0]
+    L = pb.Layer.from_synth(lay)
+    y = pb.pp_forward(L, _dev(wl.x), 0).cpu().numpy()
+    assert L.status() == 0
+    y_ref, _, a = po.layer_forward(lay, wl.x.astype(np.float64), act=0, threads=os.cpu_count() or 1)
+    _check(y, y_ref, a, np.float16, f"config 5 k={k} batch {batch}, all rows")
+    L.close()
 
 
 @pytest.mark.parametrize("batch", [2, 4, 8, 16])

@@ -36,6 +36,11 @@ def test_library_exports_every_declared_symbol():
         assert hasattr(L, n), f"{n} declared in include/ but not exported"
 
 
+def test_per_device_bookkeeping_selfcheck():
+    """Kernel attributes are set once per device; the table that remembers them keeps devices apart."""
+    assert pb.lib().pp_selftest_host() == 0
+
+
 def _random_layer(seed, M, N, B, dtype, density=0.4, bias=True):
     rng = np.random.default_rng(seed)
     Mb, Nb = -(-M // B), -(-N // B)

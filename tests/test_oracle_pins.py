@@ -120,6 +120,52 @@ def test_brute_force_tiny(seed):
         np.testing.assert_allclose(ys, ref, rtol=0, atol=1e-12)
 
 
+# ------------------------------------------- row-sampled product (used at full size)
+def test_rows_variant_hand_4x4(hand4):
+    """The row-sampled product on the hand-worked example: rows in a shuffled order, one of them twice."""
+    L = _layer_from_golden(hand4)
+    W = po.reconstruct(**L)
+    x = np.array(hand4["x"])
+    rows = [3, 0, 3, 2, 1]
+    y, a = po.dense_forward_rows(W, np.array(hand4["bias"]), x, 1, rows)
+    assert list(y[0]) == [hand4["y_relu"][r] for r in rows]
+    assert list(a[0]) == [hand4["absW_absx"][r] for r in rows]
+    y0, _ = po.dense_forward_rows(W, None, x, 0, rows)
+    assert list(y0[0]) == [hand4["Wx"][r] for r in rows]
+
+
+@pytest.mark.parametrize("act", [0, 1])
+def test_rows_variant_against_library_matmul(act):
+    """Ragged layer with a bias, three input vectors: the sampled rows (shuffled, one repeated, the last
+    row of W included) must equal the same columns of a numpy matrix product and of the full oracle
+    product, for the values and for the magnitudes |W||x|."""
+    rng = np.random.default_rng(77)
+    M, N, B = 37, 53, 8
+    Mb, Nb = -(-M // B), -(-N // B)
+    T = 17
+    flat = rng.choice(Mb * Nb, size=T, replace=False)
+    tl = np.stack([flat // Nb, flat % Nb], axis=1).astype(np.int32)
+    tv = rng.standard_normal((T, B, B))
+    rp = rng.permutation(Mb * B).astype(np.int32); cp = rng.permutation(Nb * B).astype(np.int32)
+    bias = rng.standard_normal(M)
+    x = rng.standard_normal((3, N))
+    Wb = _brute_W(M, N, B, rp, cp, tl, tv)
+    W = po.reconstruct(M, N, B, rp, cp, tl, tv)
+    rows = np.concatenate([rng.permutation(M)[:20], [M - 1, 0, M - 1]]).astype(np.int32)
+    y, a = po.dense_forward_rows(W, bias, x, act, rows)
+    assert y.shape == (3, rows.size) and a.shape == (3, rows.size)
+    ref = x @ Wb.T + bias
+    if act:
+        ref = np.maximum(ref, 0.0)
+    np.testing.assert_allclose(y, ref[:, rows], rtol=0, atol=1e-12)
+    np.testing.assert_allclose(a, (np.abs(x) @ np.abs(Wb).T)[:, rows], rtol=0, atol=1e-12)
+    yf, _, af = po.dense_forward(W, bias, x, act)
+    assert np.array_equal(y, yf[:, rows]) and np.array_equal(a, af[:, rows])
+    # no rows at all is a valid request
+    y_e, a_e = po.dense_forward_rows(W, bias, x, act, np.zeros(0, dtype=np.int32))
+    assert y_e.shape == (3, 0) and a_e.shape == (3, 0)
+
+
 # -------------------------------------------------------------------- invariants
 def test_identity_perms_density_one_is_plain_gemv():
     rng = np.random.default_rng(7)

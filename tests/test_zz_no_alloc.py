@@ -1,8 +1,8 @@
 """pp_forward_noalloc: the forward call for hosts that may not allocate device memory on the
 inference path (fixed arenas, foreign memory pools, no-synchronisation contexts).  The caller
 uploads the packed layer image itself; the kernel's reduction scratch is a fixed array inside the
-library.  Checked against pp_forward on the same inputs, twice in a row, because every call
-shares (and must re-initialise) that array.  Collected last on purpose."""
+library.  Checked against pp_forward on the same inputs and against the fp64 oracle, twice in a
+row, because every call shares (and must re-initialise) that array.  Collected last on purpose."""
 import numpy as np
 import pytest
 
@@ -43,14 +43,18 @@ def test_noalloc_matches_pp_forward_twice(case):
     image = torch.from_numpy(packed.device_image()).cuda()        # the caller's own device memory
     x = torch.from_numpy(wl.x).cuda()
     ref = pb.pp_forward(layer, x, lay.act)
-    _, _, a = po.layer_forward(lay, wl.x.astype(np.float64), threads=8)
+    y_ref, _, a = po.layer_forward(lay, wl.x.astype(np.float64), threads=8)
     out = torch.empty_like(ref)
     for call in range(2):
         out.fill_(float("nan"))
         pb.pp_forward_noalloc(packed, image, x, lay.act, out=out)
         torch.cuda.synchronize()
-        err = np.abs(out.cpu().numpy().astype(np.float64) - ref.cpu().numpy().astype(np.float64))
-        assert np.all(err <= rtol * a + atol), f"call {call}: max err {err.max()}"
+        assert pb.pp_noalloc_status() == 0, f"call {call}: the kernel's bounded wait gave up"
+        got = out.cpu().numpy().astype(np.float64)
+        err = np.abs(got - ref.cpu().numpy().astype(np.float64))       # against the allocating entry point
+        assert np.all(err <= rtol * a + atol), f"call {call}: max err vs pp_forward {err.max()}"
+        err = np.abs(got - y_ref)                                      # and against the CPU oracle
+        assert np.all(err <= rtol * a + atol), f"call {call}: max err vs oracle {err.max()}"
     # a different layer through the same fixed scratch array, then the first one again
     wl2 = synth.config5(k=16, batch=2, scale=0.25)
     other = wl2.layers[0]
