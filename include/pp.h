@@ -189,6 +189,14 @@ pp_status_t pp_layer_create_blocks(pp_layer_t** out, int M, int N, int B,
  * Synchronises with the device; *status is PP_OK or PP_ERR_TIMEOUT.  The flag is cleared by the read. */
 pp_status_t pp_layer_status(pp_layer_t* layer, pp_status_t* status);
 
+/* Which kernel a pp_forward call with this batch launches, and its launch shape (for reports; host only):
+ * out[0] kernel: 0 chunked matrix-vector, 1 persistent matrix-vector, 2 tensor-core tile kernel with one block-row
+ * per CTA, 3 clustered tensor-core tile kernel; out[1] CTAs; for the persistent kernel also out[2] asynchronous
+ * weight copies each warp keeps in flight, out[3] bytes of dynamic shared memory per CTA, out[4] how x is staged
+ * (StreamArgs::stage_mode), out[5] 1 when launched with programmatic stream serialization.  Assumes 16-byte
+ * aligned x rows. */
+pp_status_t pp_layer_launch_info(const pp_layer_t* layer, int batch, int32_t out[6]);
+
 /* Independent device copy of a layer (own weights, index arrays and scratch), e.g. to
  * serve several streams at once or to rotate copies so that repeated timing runs do not
  * find the weights in L2.  Errors: PP_ERR_INVALID_ARG, PP_ERR_ALLOC, PP_ERR_CUDA. */

@@ -62,6 +62,7 @@ def lib() -> ctypes.CDLL:
         "pp_layer_destroy": (ci, [vp]),
         "pp_layer_clone": (ci, [ctypes.POINTER(vp), vp]),
         "pp_layer_status": (ci, [vp, ctypes.POINTER(ci)]),
+        "pp_layer_launch_info": (ci, [vp, ci, i32p]),
         "pp_forward": (ci, [vp, vp, vp, ci, ci, vp]),
         "pp_forward_host": (ci, [vp, vp, vp, ci, ci, vp]),
         "pp_chain_create": (ci, [ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(ci), ci, ci]),
@@ -318,6 +319,15 @@ class Layer:
         m = np.empty(-(-self.M // self.B) * self.B, dtype=np.int32)
         _check(lib().pp_layer_output_map(self._h, m.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))), "pp_layer_output_map")
         return m
+
+    def launch_info(self, batch: int = 1) -> dict:
+        """Kernel and launch shape a forward call with this batch uses (pp_layer_launch_info)."""
+        o = np.zeros(6, dtype=np.int32)
+        _check(lib().pp_layer_launch_info(self._h, int(batch), o.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))),
+               "pp_layer_launch_info")
+        names = {0: "gemv", 1: "stream", 2: "tile", 3: "tile_cluster"}
+        return {"kernel": names[int(o[0])], "ctas": int(o[1]), "ring_depth": int(o[2]), "smem_bytes": int(o[3]),
+                "stage_mode": int(o[4]), "pdl": int(o[5])}
 
     def status(self) -> int:
         """PP_OK, or PP_ERR_TIMEOUT when a kernel's bounded wait gave up (synchronises; clears the flag)."""

@@ -249,22 +249,28 @@ bool tile_setup(pp_layer* L, const pp_layer* from) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// How the persistent kernel stages x for this call (StreamArgs::stage_mode), or -1 when x does not fit shared memory.
+int pick_stage_mode(const pp_layer* L, bool has_gather, bool own_gather, bool rows_aligned, int x_len, int batch) {
+    const pp_packed* pk = L->pk;
+    const bool has16 = has_gather && own_gather && L->d_gather16;
+    // reading x through the index array inside the multiply loop: always for one input vector, for several
+    // (fp16 layers) when tuning key 7 is 2
+    const bool direct = pp::g_stage_direct && (batch == 1 || (pp::g_stage_direct == 2 && pk->wdtype == PP_F16));
+    const int fast = has_gather ? (direct ? (has16 ? 4 : 3) : 1) : 2;
+    if (rows_aligned && pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, fast) <= pp::kStreamSmemLimit)
+        return fast;
+    if (pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, 0) <= pp::kStreamSmemLimit)
+        return 0;
+    return -1;
+}
+
 // Enqueue one layer in groups of batch columns.
 // Persistent kernel for up to kStreamMaxBatch columns; PP_ERR_UNSUPPORTED when x does not fit shared memory.
 pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_len, int x_elt, void* y, int ldy,
                        int out_mode, int batch, pp_act_t act, cudaStream_t stream, int x_limit, const int32_t* scatter) {
     const pp_packed* pk = L->pk;
-    int stage_mode = -1;
     const bool rows_aligned = aligned16(x) && (batch == 1 || ((size_t)ldx * x_elt) % 16 == 0);
-    const bool has16 = gather && gather == L->d_gather && L->d_gather16;
-    // reading x through the index array inside the multiply loop: always for one input vector, for several
-    // (fp16 layers) when tuning key 7 is 2
-    const bool direct = pp::g_stage_direct && (batch == 1 || (pp::g_stage_direct == 2 && pk->wdtype == PP_F16));
-    const int fast = gather ? (direct ? (has16 ? 4 : 3) : 1) : 2;
-    if (rows_aligned && pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, fast) <= pp::kStreamSmemLimit)
-        stage_mode = fast;
-    else if (pp::stream_smem_bytes(pk->wdtype, pk->B, pk->Npad, x_len, L->stream_max_rows, batch, 0) <= pp::kStreamSmemLimit)
-        stage_mode = 0;
+    const int stage_mode = pick_stage_mode(L, gather != nullptr, gather == L->d_gather, rows_aligned, x_len, batch);
     if (stage_mode < 0) return PP_ERR_UNSUPPORTED;
     pp::StreamArgs s{};
     s.stage_mode = stage_mode;
@@ -461,6 +467,29 @@ pp_status_t pp_layer_status(pp_layer_t* L, pp_status_t* status) {
         *status = PP_ERR_TIMEOUT;
         if (cudaMemset(L->d_status, 0, sizeof(int)) != cudaSuccess) return PP_ERR_CUDA;
     }
+    return PP_OK;
+}
+
+pp_status_t pp_layer_launch_info(const pp_layer_t* L, int batch, int32_t out[6]) {
+    if (!L || !out || batch < 1) return PP_ERR_INVALID_ARG;
+    const pp_packed* pk = L->pk;
+    for (int i = 0; i < 6; ++i) out[i] = 0;
+    if (L->tile_ok && pp::g_tile_min_batch > 0 && batch >= pp::g_tile_min_batch && (size_t)pk->N * 2 <= 48 * 1024) {
+        const bool use_cluster = pp::g_tile_cluster == 2 ||
+                                 (pp::g_tile_cluster == 1 && L->n_tile_steps > 0 && 2 * pk->T >= 7 * (int64_t)L->n_tile_steps);
+        out[0] = use_cluster ? 3 : 2;
+        out[1] = use_cluster ? (pk->Mb + pp::kTileRows - 1) / pp::kTileRows * pp::kTileRows : pk->Mb;
+        return PP_OK;
+    }
+    const int nb = batch < pp::kStreamMaxBatch ? batch : pp::kStreamMaxBatch;
+    const int stage = pp::g_use_stream ? pick_stage_mode(L, true, true, true, pk->N, nb) : -1;
+    const int chunk_group = pp::gemv_group_batch(pk->wdtype);
+    const bool stream_path = stage >= 0 && (batch + pp::kStreamMaxBatch - 1) / pp::kStreamMaxBatch <= (batch + chunk_group - 1) / chunk_group;
+    if (!stream_path) { out[0] = 0; out[1] = L->n_items; return PP_OK; }
+    out[0] = 1; out[1] = L->stream_grid; out[4] = stage;
+    out[2] = pp::stream_pick_depth(pk->wdtype, pk->B, pk->Npad, pk->N, L->stream_max_rows, nb, stage, L->stream_grid);
+    out[3] = (int32_t)pp::stream_launch_smem(pk->wdtype, pk->B, pk->Npad, pk->N, L->stream_max_rows, nb, stage, out[2]);
+    out[5] = pp::g_stream_pdl;
     return PP_OK;
 }
 

@@ -64,6 +64,24 @@ __device__ __forceinline__ void cp_async_4(void* smem_dst, const void* gsrc) {
                  :: "r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc));
 }
 
+#ifdef PP_TRACE
+// Diagnostic builds only: thread 0 of every CTA stamps the global nanosecond timer at the kernel's phases.
+__device__ __forceinline__ void trace_stamp(const StreamArgs& a, int slot) {
+    if (a.trace && threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        a.trace[(size_t)blockIdx.x * 8 + slot] = t;
+        if (slot == 0) {
+            unsigned smid;
+            asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+            a.trace[(size_t)blockIdx.x * 8 + 7] = smid;
+        }
+    }
+}
+#else
+__device__ __forceinline__ void trace_stamp(const StreamArgs&, int) {}
+#endif
+
 __device__ __forceinline__ int x_index(const StreamArgs& a, int pj) {
     if (a.gather_idx) return __ldg(a.gather_idx + pj);
     return pj < a.x_limit ? pj : -1;
@@ -453,6 +471,7 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
 
     // 1. the next kernel in the stream may start its own prologue; this one prefetches what does
     //    not depend on its predecessor: tables, first U weight fragments, column offsets
+    trace_stamp(a, 0);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     init_xbar(L);
     issue_static<RG>(a, d, L);
@@ -465,11 +484,14 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
     // 2. everything before this kernel in the stream is complete from here on: fetch x
     //    (the barrier publishes the mbarrier's initialisation to the threads that will wait on it)
     __syncthreads();
+    trace_stamp(a, 1);
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    trace_stamp(a, 2);
     issue_x<__half>(a, L);
 
     // 3. pivoted x in shared memory
     finish_stage<__half, U>(a, L);
+    trace_stamp(a, 3);
     plan_parks(d, L);
 
     // 4. stream this warp's share
@@ -593,7 +615,9 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
+    trace_stamp(a, 4);
     finalize<RG>(a, d, L);
+    trace_stamp(a, 5);
 }
 
 // ------------------------------------------------------------------ fp32 tiles
@@ -609,6 +633,7 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const __grid_co
     const int wbeg = warp_begin(d, warp), wend = warp_begin(d, warp + 1);
     if (tid <= kStreamWarps) L.wb[tid] = warp_begin(d, tid);
 
+    trace_stamp(a, 0);
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     init_xbar(L);
     issue_static<RG>(a, d, L);
@@ -618,9 +643,12 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const __grid_co
     xw.init(a.xoff, wbeg, wend, lane);
     warm_translations(a);
     __syncthreads();
+    trace_stamp(a, 1);
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    trace_stamp(a, 2);
     issue_x<float>(a, L);
     finish_stage<float, U>(a, L);
+    trace_stamp(a, 3);
     plan_parks(d, L);
 
     float acc[NB][2];
@@ -688,7 +716,9 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const __grid_co
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
+    trace_stamp(a, 4);
     finalize<RG>(a, d, L);
+    trace_stamp(a, 5);
 }
 
 template <auto Kernel>
@@ -734,6 +764,11 @@ int xs_stride_for(pp_dtype_t dt, int n_pad) { return dt == PP_F16 ? n_pad + 8 : 
 
 }  // namespace
 
+#ifdef PP_TRACE
+unsigned long long* g_stream_trace = nullptr;   // diagnostic builds: [calls][kTraceCtas][8] stamps, filled call after call
+int g_stream_trace_calls = 0, g_stream_trace_next = 0;
+constexpr int kTraceCtas = 320;
+#endif
 int g_stream_depth = 0;   // ring slots per warp: 4, 6 or 8; 0 = chosen per launch
 int g_stream_pdl = 1;     // launch with programmatic stream serialization (prologue overlaps the previous kernel)
 
@@ -773,6 +808,10 @@ size_t smem_bytes_at(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, i
 }
 }  // namespace
 
+size_t stream_launch_smem(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int depth) {
+    return smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, depth);
+}
+
 cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a_in, const CtaDesc* host_table, int grid,
                           cudaStream_t stream) {
     if (grid <= 0) return cudaSuccess;
@@ -784,6 +823,11 @@ cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a_in, const Ct
         return cudaErrorInvalidValue;
     a.xs_stride = xs_stride_for(dt, a.n_pad);
     a.raw_stride = raw_stride_for(a.x_len, a.batch);
+#ifdef PP_TRACE
+    a.trace = nullptr;
+    if (g_stream_trace && g_stream_trace_next < g_stream_trace_calls && grid <= kTraceCtas)
+        a.trace = g_stream_trace + (size_t)(g_stream_trace_next++) * kTraceCtas * 8;
+#endif
     a.max_rows = (a.max_rows + 31) / 32 * 32;      // whole strips of either height; keeps the regions behind 128-byte aligned
     if (grid <= kParamCtas)
         for (int c = 0; c < grid; ++c) P.table[c] = host_table[c];
@@ -805,3 +849,13 @@ cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a_in, const Ct
 }
 
 }  // namespace pp
+
+#ifdef PP_TRACE
+// Diagnostic builds only: the next `calls` launches of the persistent kernel write their phase stamps to
+// `device_buffer` (calls x 320 x 8 unsigned 64-bit words).
+extern "C" void pp_trace_set_buffer(void* device_buffer, int calls) {
+    pp::g_stream_trace = static_cast<unsigned long long*>(device_buffer);
+    pp::g_stream_trace_calls = calls;
+    pp::g_stream_trace_next = 0;
+}
+#endif

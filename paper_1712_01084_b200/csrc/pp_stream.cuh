@@ -21,6 +21,7 @@ struct StreamArgs {
     float* partials;             // [stream_slots][rows_per_strip * kStreamMaxBatch]
     int* counters;               // [S], zero between launches
     int* status;                 // raised to 1 when the bounded wait for the copy of x gave up; may be NULL
+    unsigned long long* trace;   // diagnostic builds (PP_TRACE): [grid][8] time stamps of the kernel's phases; else unused
     int ldx, ldy;
     int x_limit;                 // with gather_idx == NULL: columns >= x_limit read 0
     int n_pad;                   // pivoted columns staged into shared memory
@@ -42,6 +43,9 @@ struct StreamArgs {
 // Shared memory the kernel needs for this (dtype, n_pad, batch); the caller falls back to the
 // chunked kernel when it exceeds kStreamSmemLimit.
 size_t stream_smem_bytes(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode);
+// Ring depth a launch picks, and the dynamic shared memory of a launch with that depth (max_rows as in the plan).
+int stream_pick_depth(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int grid);
+size_t stream_launch_smem(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int depth);
 extern int g_stream_depth;   // weight-ring slots per warp: 4, 6 or 8; 0 = chosen per launch
 extern int g_stream_pdl;     // 1: launch with programmatic stream serialization
 constexpr size_t kStreamSmemLimit = 224 * 1024;

@@ -51,6 +51,21 @@ def test_algorithmic_bytes_config5():
     assert got == want
 
 
+def test_tile_column_count_matches_the_packer():
+    """bench.n_tile_col (per-block-row lists padded to 4 entries) is what the packer reports."""
+    from paper_1712_01084_b200 import binding as pb
+    wl = synth.config3(batch=1, scale=1 / 8)
+    for lay in wl.layers:
+        pk = pb.Packed(lay.M, lay.N, lay.B, lay.row_perm, lay.col_perm, lay.tile_list, lay.tile_values, lay.bias)
+        assert bench.n_tile_col(lay) == pk.n_tile_col
+
+
+def test_region_plan_covers_exactly_the_steps():
+    for steps in (1, 20, 999, 1000, 1001, 2500, 20000):
+        main, replays, rem = bench.region_plan(steps)
+        assert main * replays + rem == steps and 0 < main <= bench.GRAPH_CALLS and 0 <= rem < main
+
+
 def test_reference_arm_rank_handling():
     """Under a multi-rank launch only rank 0 runs the CPU oracle; the others exit 0 without output."""
     env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
