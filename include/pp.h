@@ -257,7 +257,21 @@ pp_status_t pp_layer_output_map(const pp_layer_t* layer, int32_t* map);
  * Output permutation elimination (Section 4.2.2): after pp_chain_set_output_pivoted(chain, 1)
  * pp_chain_forward leaves y in the last layer's pivoted row order, float
  * [batch][M_pad_last], padding positions 0; pp_chain_output_map gives the relabelling
- * (as pp_layer_output_map of the last layer).  Errors: PP_ERR_INVALID_ARG. */
+ * (as pp_layer_output_map of the last layer).  Errors: PP_ERR_INVALID_ARG.
+ *
+ * By default a chain is one kernel launch per layer, each launched with programmatic stream serialization so
+ * that its prologue overlaps the previous layer's tail.
+ *
+ * One kernel for the whole chain (tuning key 14 = 1, set before pp_chain_create): when every layer has fp16
+ * weights, batch <= 8 and the largest layer plan is resident on the device at once, pp_chain_forward is ONE
+ * cooperative kernel launch.  Every CTA runs its share of layer 0, then of layer 1, ...; between two layers the
+ * grid meets at a counter in device memory, and each CTA requests the tables and first weights of the next
+ * layer one layer ahead, into the other of two shared-memory regions.  It measured slower than the launch per
+ * layer on the 9216-4096-4096-1000 stack (a layer boundary inside the kernel is four dependent round trips
+ * to the L2: publish, observe, fetch x, exchange partial sums), so it is not the default.  The waits are
+ * bounded: when one gives up, the kernel raises a status word and ends, y is invalid and pp_chain_status
+ * reports PP_ERR_TIMEOUT.  pp_chain_status synchronises with the device, also collects the status words of
+ * the chain's layers (layer-by-layer execution), writes PP_OK or PP_ERR_TIMEOUT to *status and clears them. */
 pp_status_t pp_chain_create(pp_chain_t** out, pp_layer_t* const* layers,
                             const pp_act_t* acts, int n_layers, int max_batch);
 pp_status_t pp_chain_destroy(pp_chain_t* chain);
@@ -266,6 +280,7 @@ pp_status_t pp_chain_output_map(const pp_chain_t* chain, int32_t* map);
 pp_status_t pp_chain_link_info(const pp_chain_t* chain, int32_t* identity);
 pp_status_t pp_chain_forward(pp_chain_t* chain, const void* x, void* y, int batch,
                              void* cuda_stream);
+pp_status_t pp_chain_status(pp_chain_t* chain, pp_status_t* status);
 
 /* ------------------------------------------------------------------------- *
  * Recurrent use: one pivoted layer as the gate matrix of an LSTM cell.  The
@@ -427,7 +442,12 @@ pp_status_t pp_selftest_host(void);
  *         groups' tile-columns carry at least 3.5 of 4 possible tiles on average, else one block-row per CTA
  * key 13: 1 (default) chain links whose folded map is the identity store pivoted rows without an index array,
  *         0 sends them through the map like any other link
- * key 11: 1 (default) lets pp_lstm_forward run all steps in one cooperative kernel when the layer qualifies, 0 never */
+ * key 11: 1 (default) lets pp_lstm_forward run all steps in one cooperative kernel when the layer qualifies, 0 never
+ * key 14: 1 chains of fp16 layers run as one cooperative kernel when they qualify (read at pp_chain_create
+ *         and at every pp_chain_forward), 0 (default) one launch per layer
+ * key 15: polls after which the bounded device-side waits of the persistent kernel (copy of x) and of the chain
+ *         kernel (layer boundaries) give up; 0 (default) = the kernels' own limits (seconds).  Small values exist
+ *         so that tests can see a wait give up: the kernel then raises its status word and still ends by itself */
 pp_status_t pp_set_tuning(int key, int value);
 
 #ifdef __cplusplus

@@ -68,6 +68,7 @@ def lib() -> ctypes.CDLL:
         "pp_chain_create": (ci, [ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.POINTER(ci), ci, ci]),
         "pp_chain_destroy": (ci, [vp]),
         "pp_chain_forward": (ci, [vp, vp, vp, ci, vp]),
+        "pp_chain_status": (ci, [vp, ctypes.POINTER(ci)]),
         "pp_chain_set_output_pivoted": (ci, [vp, ci]),
         "pp_chain_output_map": (ci, [vp, i32p]),
         "pp_chain_link_info": (ci, [vp, i32p]),
@@ -467,6 +468,12 @@ class Chain:
         m = np.empty(-(-last.M // last.B) * last.B, dtype=np.int32)
         _check(lib().pp_chain_output_map(self._h, m.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))), "pp_chain_output_map")
         return m
+
+    def status(self) -> int:
+        """PP_OK, or PP_ERR_TIMEOUT when a bounded device-side wait gave up (synchronises; clears the flags)."""
+        st = ctypes.c_int(0)
+        _check(lib().pp_chain_status(self._h, ctypes.byref(st)), "pp_chain_status")
+        return st.value
 
     def link_info(self) -> np.ndarray:
         """identity[l] = 1 when the link into layer l needs no index array (pp_chain_link_info)."""

@@ -85,6 +85,13 @@ struct pp_chain {
     std::vector<char> identity;    // entry l (l >= 1): the folded map of the link l-1 -> l is the identity (Section 4.2.3)
     bool out_pivoted = false;      // the last layer leaves its output in pivoted row order (Section 4.2.2)
     int max_batch = 0;
+    // one-kernel execution (fp16 layers, batch <= 8): per batch size the layers' kernel arguments in device memory
+    pp::StreamArgs* d_fused_args = nullptr;   // [kStreamMaxBatch][n_layers]
+    int* d_fused_grids = nullptr;             // [n_layers]
+    unsigned* d_fused_sync = nullptr;         // [0] arrival counter, [1] status word
+    int fused_grid = 0;                       // CTAs of the launch (0: the chain runs layer by layer)
+    size_t fused_region[pp::kStreamMaxBatch + 1] = {}; // bytes of one shared-memory region per batch size (0: that batch runs layer by layer)
+    int fused_depth[pp::kStreamMaxBatch + 1] = {};     // weight copies per warp in flight for that batch size (4 or 8)
 };
 
 namespace {
@@ -264,14 +271,10 @@ int pick_stage_mode(const pp_layer* L, bool has_gather, bool own_gather, bool ro
     return -1;
 }
 
-// Enqueue one layer in groups of batch columns.
-// Persistent kernel for up to kStreamMaxBatch columns; PP_ERR_UNSUPPORTED when x does not fit shared memory.
-pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_len, int x_elt, void* y, int ldy,
-                       int out_mode, int batch, pp_act_t act, cudaStream_t stream, int x_limit, const int32_t* scatter) {
+// Arguments of one persistent-kernel launch over this layer.
+pp::StreamArgs make_stream_args(const pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_len, void* y, int ldy,
+                                int out_mode, int batch, pp_act_t act, int x_limit, const int32_t* scatter, int stage_mode) {
     const pp_packed* pk = L->pk;
-    const bool rows_aligned = aligned16(x) && (batch == 1 || ((size_t)ldx * x_elt) % 16 == 0);
-    const int stage_mode = pick_stage_mode(L, gather != nullptr, gather == L->d_gather, rows_aligned, x_len, batch);
-    if (stage_mode < 0) return PP_ERR_UNSUPPORTED;
     pp::StreamArgs s{};
     s.stage_mode = stage_mode;
     s.values = L->d_values; s.xoff = L->d_xoff; s.strip_start = L->d_strip_start;
@@ -280,6 +283,18 @@ pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ld
     s.x = x; s.y = y; s.partials = L->d_spartials; s.counters = L->d_scounters; s.status = L->d_status;
     s.ldx = ldx; s.ldy = ldy; s.x_limit = x_limit; s.n_pad = pk->Npad; s.x_len = x_len; s.max_rows = L->stream_max_rows; s.batch = batch;
     s.act = (int)act; s.out_mode = out_mode;
+    return s;
+}
+
+// Enqueue one layer in groups of batch columns.
+// Persistent kernel for up to kStreamMaxBatch columns; PP_ERR_UNSUPPORTED when x does not fit shared memory.
+pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_len, int x_elt, void* y, int ldy,
+                       int out_mode, int batch, pp_act_t act, cudaStream_t stream, int x_limit, const int32_t* scatter) {
+    const pp_packed* pk = L->pk;
+    const bool rows_aligned = aligned16(x) && (batch == 1 || ((size_t)ldx * x_elt) % 16 == 0);
+    const int stage_mode = pick_stage_mode(L, gather != nullptr, gather == L->d_gather, rows_aligned, x_len, batch);
+    if (stage_mode < 0) return PP_ERR_UNSUPPORTED;
+    const pp::StreamArgs s = make_stream_args(L, gather, x, ldx, x_len, y, ldy, out_mode, batch, act, x_limit, scatter, stage_mode);
     return pp::launch_stream(pk->wdtype, pk->B, s, pk->cta_desc.data(), L->stream_grid, stream) == cudaSuccess
                ? PP_OK : PP_ERR_CUDA;
 }
@@ -359,6 +374,7 @@ pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx
 namespace {
 // Uploads a packed layer to the current device; takes ownership of pk (freed on failure).
 pp_status_t layer_from_pack(pp_layer_t** out, pp_packed* pk);
+void chain_plan_fused(pp_chain* C);
 }
 
 extern "C" {
@@ -620,11 +636,19 @@ pp_status_t pp_chain_create(pp_chain_t** out, pp_layer_t* const* layers, const p
              cudaMemset(C->d_inter[(size_t)l - 1], 0, ibytes) == cudaSuccess;
         if (!ok) st = PP_ERR_ALLOC;
     }
+    if (ok) {
+        ok = cudaMalloc(reinterpret_cast<void**>(&C->d_fused_args), sizeof(pp::StreamArgs) * pp::kStreamMaxBatch * (size_t)n_layers) == cudaSuccess &&
+             cudaMalloc(reinterpret_cast<void**>(&C->d_fused_grids), 4 * (size_t)n_layers) == cudaSuccess &&
+             cudaMalloc(reinterpret_cast<void**>(&C->d_fused_sync), 256) == cudaSuccess &&
+             cudaMemset(C->d_fused_sync, 0, 256) == cudaSuccess;
+        if (!ok) st = PP_ERR_ALLOC;
+    }
     if (!ok) {
         cudaGetLastError();
         pp_chain_destroy(C);
         return st;
     }
+    chain_plan_fused(C);
     *out = C;
     return PP_OK;
 }
@@ -633,47 +657,153 @@ pp_status_t pp_chain_destroy(pp_chain_t* C) {
     if (!C) return PP_OK;
     for (int32_t* q : C->d_q) cudaFree(q);
     for (void* b : C->d_inter) cudaFree(b);
+    cudaFree(C->d_fused_args); cudaFree(C->d_fused_grids); cudaFree(C->d_fused_sync);
     delete C;
     return PP_OK;
 }
+
+}  // extern "C"
+
+namespace {
+
+// What layer l of a chain reads and writes: layer 0 gathers the call's x through its own column index array; every
+// later layer finds its input already in its pivoted column order (written there by its producer's epilogue).
+struct ChainLink {
+    const int32_t* gather; const void* x; int ldx, x_len, x_limit;
+    void* y; int ldy, out_mode; const int32_t* scatter;
+};
+ChainLink chain_link(const pp_chain* C, int l, const void* x, void* y) {
+    const int n = (int)C->layers.size();
+    const pp_layer* L = C->layers[(size_t)l];
+    const pp_packed* pk = L->pk;
+    ChainLink k{};
+    k.gather = l == 0 ? L->d_gather : nullptr;
+    k.x = l == 0 ? x : C->d_inter[(size_t)l - 1];
+    k.ldx = k.x_len = k.x_limit = l == 0 ? pk->N : pk->Npad;
+    k.scatter = L->d_scatter;
+    if (l == n - 1) {
+        k.y = y;
+        k.ldy = C->out_pivoted ? pk->Mpad : pk->M;
+        k.out_mode = C->out_pivoted ? pp::OUT_PIVOTED_F32 : pp::OUT_SCATTER_F32;
+    } else {
+        const pp_packed* nx = C->layers[(size_t)l + 1]->pk;
+        const bool f16 = nx->wdtype == PP_F16;
+        k.y = C->d_inter[(size_t)l];
+        k.ldy = nx->Npad;
+        if (C->identity[(size_t)l + 1] && pp::g_link_identity) {
+            k.out_mode = f16 ? pp::OUT_PIVOTED_F16 : pp::OUT_PIVOTED_F32;
+        } else {
+            k.out_mode = f16 ? pp::OUT_SCATTER_F16 : pp::OUT_SCATTER_F32;
+            k.scatter = C->d_q[(size_t)l + 1];
+        }
+    }
+    return k;
+}
+
+// One-kernel execution of the chain: possible when every layer is fp16, its input fits the persistent kernel's
+// bulk-copy staging for the batch, and the largest plan is resident at once.  (Re)builds the per-batch argument
+// arrays; leaves fused_grid = 0 when the chain does not qualify.
+void chain_plan_fused(pp_chain* C) {
+    const int n = (int)C->layers.size();
+    C->fused_grid = 0;
+    for (size_t b = 0; b <= (size_t)pp::kStreamMaxBatch; ++b) { C->fused_region[b] = 0; C->fused_depth[b] = 0; }
+    if (n < 2 || n > pp::kChainMaxLayers || !pp::g_chain_fused || !pp::g_use_stream) return;
+    int grid = 0;
+    std::vector<int> grids((size_t)n);
+    for (int l = 0; l < n; ++l) {
+        const pp_layer* L = C->layers[(size_t)l];
+        if (L->pk->wdtype != PP_F16 || L->stream_grid < 1) return;
+        grids[(size_t)l] = L->stream_grid;
+        grid = std::max(grid, L->stream_grid);
+    }
+    std::vector<pp::StreamArgs> args((size_t)pp::kStreamMaxBatch * n);
+    const int top = std::min(C->max_batch, pp::kStreamMaxBatch);
+    bool any = false;
+    for (int batch = 1; batch <= top; ++batch) {
+        size_t region[2] = {0, 0};                            // at 4 and at 8 weight copies per warp
+        bool ok = true;
+        for (int l = 0; l < n && ok; ++l) {
+            const pp_layer* L = C->layers[(size_t)l];
+            const pp_packed* pk = L->pk;
+            const ChainLink k = chain_link(C, l, nullptr, nullptr);
+            const bool rows_aligned = batch == 1 || ((size_t)k.ldx * 2) % 16 == 0;
+            const int stage = pick_stage_mode(L, k.gather != nullptr, true, rows_aligned, k.x_len, batch);
+            if (stage < 1) { ok = false; break; }            // x must arrive by bulk copy
+            pp::StreamArgs a = make_stream_args(L, k.gather, k.x, k.ldx, k.x_len, k.y, k.ldy, k.out_mode, batch,
+                                                C->acts[(size_t)l], k.x_limit, k.scatter, stage);
+            pp::stream_finish_args(PP_F16, a);
+            a.status = reinterpret_cast<int*>(C->d_fused_sync + 1);
+            args[(size_t)(batch - 1) * n + l] = a;
+            for (int q = 0; q < 2; ++q)
+                region[q] = std::max(region[q], pp::stream_launch_smem(PP_F16, pk->B, pk->Npad, k.x_len, L->stream_max_rows,
+                                                                       batch, stage, q ? 8 : 4));
+        }
+        if (!ok) continue;
+        // the deeper ring when two regions of it fit and the plans stay resident, else the shallow one
+        for (int q = 1; q >= 0; --q) {
+            const size_t r = (region[q] + 1023) / 1024 * 1024;
+            if (2 * r <= pp::kStreamSmemLimit && pp::chain_resident_ctas(2 * r, q ? 8 : 4) >= grid) {
+                C->fused_region[(size_t)batch] = r;
+                C->fused_depth[(size_t)batch] = q ? 8 : 4;
+                any = true;
+                break;
+            }
+        }
+    }
+    if (!any) return;
+    if (cudaMemcpy(C->d_fused_args, args.data(), args.size() * sizeof(pp::StreamArgs), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(C->d_fused_grids, grids.data(), (size_t)n * 4, cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaGetLastError();
+        return;
+    }
+    C->fused_grid = grid;
+}
+
+}  // namespace
+
+extern "C" {
 
 pp_status_t pp_chain_forward(pp_chain_t* C, const void* x, void* y, int batch, void* cuda_stream) {
     if (!C || !x || !y || batch < 1 || batch > C->max_batch || x == y) return PP_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(y)) return PP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int n = (int)C->layers.size();
-    const void* cur = x;
+    if (C->fused_grid > 0 && batch <= pp::kStreamMaxBatch && C->fused_region[(size_t)batch] > 0 && pp::g_chain_fused) {
+        // all layers in one cooperative kernel, the grid meeting at a counter between layers
+        pp::ChainLaunch P{};
+        P.layers = C->d_fused_args + (size_t)(batch - 1) * n;
+        P.grids = C->d_fused_grids;
+        P.x = x; P.y = y;
+        P.counter = C->d_fused_sync; P.status = reinterpret_cast<int*>(C->d_fused_sync + 1);
+        P.n_layers = n; P.polls = 0; P.region_bytes = (int)C->fused_region[(size_t)batch];
+        return pp::launch_chain_f16(P, C->fused_grid, 2 * C->fused_region[(size_t)batch], C->fused_depth[(size_t)batch], stream) == cudaSuccess
+                   ? PP_OK : PP_ERR_CUDA;
+    }
     for (int l = 0; l < n; ++l) {
         pp_layer* L = C->layers[(size_t)l];
-        const pp_packed* pk = L->pk;
-        const int x_elt = pk->wdtype == PP_F16 ? 2 : 4;
-        // layer 0 gathers through its own column index array; every later layer finds its input
-        // already in its pivoted column order (written there by its producer's epilogue)
-        const int32_t* gather = l == 0 ? L->d_gather : nullptr;
-        const int ldx = l == 0 ? pk->N : pk->Npad;
-        const int x_len = ldx;
-        const int x_limit = l == 0 ? pk->N : pk->Npad;
-        pp_status_t st;
-        if (l == n - 1) {
-            if (C->out_pivoted)
-                st = run_layer(L, gather, cur, ldx, x_len, x_elt, y, pk->Mpad, pp::OUT_PIVOTED_F32, batch, C->acts[(size_t)l],
-                               stream, x_limit);
-            else
-                st = run_layer(L, gather, cur, ldx, x_len, x_elt, y, pk->M, pp::OUT_SCATTER_F32, batch, C->acts[(size_t)l],
-                               stream, x_limit);
-        } else {
-            const pp_packed* nx = C->layers[(size_t)l + 1]->pk;
-            const bool f16 = nx->wdtype == PP_F16;
-            if (C->identity[(size_t)l + 1] && pp::g_link_identity)
-                st = run_layer(L, gather, cur, ldx, x_len, x_elt, C->d_inter[(size_t)l], nx->Npad,
-                               f16 ? pp::OUT_PIVOTED_F16 : pp::OUT_PIVOTED_F32, batch, C->acts[(size_t)l], stream, x_limit);
-            else
-                st = run_layer(L, gather, cur, ldx, x_len, x_elt, C->d_inter[(size_t)l], nx->Npad,
-                               f16 ? pp::OUT_SCATTER_F16 : pp::OUT_SCATTER_F32, batch, C->acts[(size_t)l], stream, x_limit,
-                               C->d_q[(size_t)l + 1]);
-            cur = C->d_inter[(size_t)l];
-        }
+        const ChainLink k = chain_link(C, l, x, y);
+        const pp_status_t st = run_layer(L, k.gather, k.x, k.ldx, k.x_len, L->pk->wdtype == PP_F16 ? 2 : 4, k.y, k.ldy, k.out_mode,
+                                         batch, C->acts[(size_t)l], stream, k.x_limit, k.scatter);
         if (st != PP_OK) return st;
+    }
+    return PP_OK;
+}
+
+pp_status_t pp_chain_status(pp_chain_t* C, pp_status_t* status) {
+    if (!C || !status) return PP_ERR_INVALID_ARG;
+    *status = PP_OK;
+    unsigned words[2] = {0u, 0u};
+    if (cudaDeviceSynchronize() != cudaSuccess ||
+        cudaMemcpy(words, C->d_fused_sync, sizeof(words), cudaMemcpyDeviceToHost) != cudaSuccess) return PP_ERR_CUDA;
+    if (words[1]) {
+        *status = PP_ERR_TIMEOUT;        // the launch that gave up left its arrival counter behind: clear both
+        if (cudaMemset(C->d_fused_sync, 0, sizeof(words)) != cudaSuccess) return PP_ERR_CUDA;
+    }
+    for (pp_layer* L : C->layers) {      // layer-by-layer execution raises the layers' own words
+        pp_status_t st = PP_OK;
+        const pp_status_t rc = pp_layer_status(L, &st);
+        if (rc != PP_OK) return rc;
+        if (st != PP_OK) *status = st;
     }
     return PP_OK;
 }
@@ -681,6 +811,7 @@ pp_status_t pp_chain_forward(pp_chain_t* C, const void* x, void* y, int batch, v
 pp_status_t pp_chain_set_output_pivoted(pp_chain_t* C, int enable) {
     if (!C || (enable != 0 && enable != 1)) return PP_ERR_INVALID_ARG;
     C->out_pivoted = enable != 0;
+    chain_plan_fused(C);                 // the last layer's store mode is part of the one-kernel arguments
     return PP_OK;
 }
 
@@ -702,6 +833,10 @@ pp_status_t pp_lstm_status(pp_lstm_t* R, pp_status_t* status) {
     if (cudaMemcpy(&flag, R->d_sync + 1, sizeof(flag), cudaMemcpyDeviceToHost) != cudaSuccess) return PP_ERR_CUDA;
     *status = flag ? PP_ERR_TIMEOUT : PP_OK;
     if (flag && cudaMemset(R->d_sync + 1, 0, sizeof(flag)) != cudaSuccess) return PP_ERR_CUDA;
+    pp_status_t layer_st = PP_OK;                 // the per-step path raises the gate layer's own word
+    const pp_status_t rc = pp_layer_status(R->gates, &layer_st);
+    if (rc != PP_OK) return rc;
+    if (layer_st != PP_OK) *status = layer_st;
     return PP_OK;
 }
 

@@ -10,6 +10,7 @@
 #include <cuda_fp16.h>
 
 #include "pp_lstm.cuh"
+#include "pp_stream.cuh"
 
 namespace pp {
 namespace {
@@ -229,6 +230,7 @@ __global__ void __launch_bounds__(kPersistThreads, 1) lstm_persist_kernel(const 
         }
         // every CTA collects all packets (two per 16-byte load), bounded retries on the ones not there yet
         bool gave_up = false;
+        const unsigned spin_limit = a.spin_limit ? a.spin_limit : kSpinLimit;
         const int n_pairs = a.m_pad / 2;
         for (int base = 0; base < n_pairs; base += 8 * kPersistThreads) {
             uint4 v[8];
@@ -244,7 +246,7 @@ __global__ void __launch_bounds__(kPersistThreads, 1) lstm_persist_kernel(const 
                 if (i >= n_pairs) continue;
                 unsigned spins = 0;
                 while (v[k].y != tag || v[k].w != tag) {
-                    if (++spins > kSpinLimit || ((spins & 1023u) == 0 && *reinterpret_cast<volatile int*>(a.status))) {
+                    if (++spins > spin_limit || ((spins & 1023u) == 0 && *reinterpret_cast<volatile int*>(a.status))) {
                         gave_up = true;
                         break;
                     }
@@ -295,6 +297,7 @@ cudaError_t launch_lstm_persist(const LstmPersistArgs& a_in, int grid, size_t sm
         configured.mark(dev);
     }
     LstmPersistArgs a = a_in;
+    a.spin_limit = (unsigned)g_stream_wait_polls;
     void* args[] = {&a};
     return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(lstm_persist_kernel), dim3((unsigned)grid),
                                        dim3(kPersistThreads), args, smem, stream);

@@ -41,6 +41,7 @@ struct LstmPersistArgs {
     int I, H, n_pad, m_pad, steps;
     int n_strips;                // S
     int strips_per_cta;          // power of two <= 16
+    unsigned spin_limit;         // re-reads of one packet before a wait gives up (0: the kernel's own limit; set by the launcher)
 };
 
 // Shared memory the persistent kernel needs, or 0 when the layer does not qualify (weights of one

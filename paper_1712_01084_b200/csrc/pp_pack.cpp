@@ -16,6 +16,8 @@ int g_prepass = 1;
 int g_lstm_persist = 1;
 int g_tile_cluster = 1;
 int g_link_identity = 1;
+int g_chain_fused = 0;      // measured: one launch per layer (programmatic dependent launch) is the faster way through a chain
+extern int g_stream_wait_polls;   // poll limit of the bounded device-side waits (pp_stream.cu)
 int g_stage_direct = 2;    // 0: always materialise the pivoted x in shared memory; 1: one input vector is read through the
                            // index array in the multiply loop; 2: so are 2..8 vectors of fp16 layers
 extern int g_stream_depth; // weight-ring slots per warp of the persistent kernel (pp_stream.cu)
@@ -333,6 +335,8 @@ pp_status_t pp_set_tuning(int key, int value) {
     if (key == 11 && (value == 0 || value == 1)) { pp::g_lstm_persist = value; return PP_OK; }
     if (key == 12 && value >= 0 && value <= 2) { pp::g_tile_cluster = value; return PP_OK; }
     if (key == 13 && (value == 0 || value == 1)) { pp::g_link_identity = value; return PP_OK; }
+    if (key == 14 && (value == 0 || value == 1)) { pp::g_chain_fused = value; return PP_OK; }
+    if (key == 15 && value >= 0) { pp::g_stream_wait_polls = value; return PP_OK; }
     return PP_ERR_INVALID_ARG;
 }
 

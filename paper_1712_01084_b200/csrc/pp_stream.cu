@@ -216,11 +216,12 @@ __device__ __forceinline__ void init_xbar(const SmemLayout& L) {
     }
 }
 
-constexpr int kXWaitPolls = 1 << 22;   // polls of the x barrier before the kernel gives up (seconds; a copy that lands never gets near it)
+constexpr int kXWaitPolls = 1 << 22;   // default polls of the x barrier before the kernel gives up (seconds; a copy that lands never gets near it)
 
-// Phase 3: wait for the copies of phases 1 and 2, finish the staged pivoted x.
+// Phase 3: wait for the copies of phases 1 and 2, finish the staged pivoted x.  x_parity: phase of the x barrier
+// this use completes (0 for the first use in a kernel, alternating after that).
 template <typename T, int U>
-__device__ __forceinline__ void finish_stage(const StreamArgs& a, const SmemLayout& L) {
+__device__ __forceinline__ void finish_stage(const StreamArgs& a, const SmemLayout& L, uint32_t x_parity = 0u) {
     constexpr int EPC = 16 / (int)sizeof(T);
     const int tid = threadIdx.x;
     const T* x = static_cast<const T*>(a.x);
@@ -242,10 +243,25 @@ __device__ __forceinline__ void finish_stage(const StreamArgs& a, const SmemLayo
     if (a.stage_mode != 0 && (a.stage_mode != 2 ? a.x_len : a.x_limit) >= EPC) {   // and so must x
         const uint32_t bar = (uint32_t)__cvta_generic_to_shared(L.xbar);
         uint32_t ok = 0u;
-        for (int i = 0; i < kXWaitPolls && !ok; ++i)
-            asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\nselp.u32 %0, 1, 0, p;\n}"
-                         : "=r"(ok) : "r"(bar) : "memory");
-        if (!ok && a.status) *a.status = 1;      // bounded wait gave up: the output of this call is invalid
+        // Normally up to kXWaitPolls polls that may each suspend the thread for a while (seconds in all).  A
+        // caller-set limit counts polls that return at once, so that a test can make the wait run out on purpose.
+        if (a.wait_polls > 0) {
+            for (int i = 0; i < a.wait_polls && !ok; ++i)
+                asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                             : "=r"(ok) : "r"(bar), "r"(x_parity) : "memory");
+        } else {
+            for (int i = 0; i < kXWaitPolls && !ok; ++i)
+                asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                             : "=r"(ok) : "r"(bar), "r"(x_parity) : "memory");
+        }
+        if (!ok) {
+            // bounded wait gave up: the output of this call is invalid.  The copy is still in flight; it must have
+            // landed before this CTA's shared memory is given back, so wait once more with the kernel's own limit.
+            if (a.status) *a.status = 1;
+            for (int i = 0; i < kXWaitPolls && !ok; ++i)
+                asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                             : "=r"(ok) : "r"(bar), "r"(x_parity) : "memory");
+        }
     }
     if (a.stage_mode == 1) {
         __syncthreads();
@@ -455,42 +471,75 @@ struct XoffWindow {
 };
 
 // ------------------------------------------------------------------ fp16 tiles
+// How a layer body meets the producer of its input.  release(): the consumer of this layer's output may start
+// its own prologue.  wait(): called by all threads after a CTA barrier; on return everything the producer wrote
+// is visible; false when a bounded wait gave up (the CTA then leaves the kernel).
+struct LaunchDependency {      // the producer is the previous kernel in the stream (programmatic dependent launch)
+    __device__ __forceinline__ void release() const { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+    __device__ __forceinline__ bool wait() const {
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        return true;
+    }
+};
+
+// What a layer requests before it meets its producer: its tables and the first U weight fragments of every warp
+// (nothing here depends on the producer).  The cp.async groups it commits are the caller's to wait for.
 template <int U>
-__global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_constant__ StreamLaunch P) {
+__device__ __forceinline__ void stream_f16_prologue(const StreamArgs& a, const CtaDesc d, unsigned char* smem_raw) {
+    const SmemLayout L = carve(smem_raw, 16, U, a, 2);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int wbeg = warp_begin(d, warp), wend = warp_begin(d, warp + 1);
+    if (tid <= kStreamWarps) L.wb[tid] = warp_begin(d, tid);
+    issue_static<16>(a, d, L);
+    const WeightRing<U> ring{L.ring + (warp * U) * 32 + lane, reinterpret_cast<const uint4*>(a.values) + lane};
+    ring.prologue(wbeg, wend);
+}
+
+struct NothingEarly {
+    __device__ __forceinline__ void operator()() const {}
+};
+
+// One fp16 layer on this CTA's range `d`: prologue (tables, first weights; skipped when the caller has already
+// requested them into this layer's shared memory), dependency wait, x, multiply, epilogue.  `early` runs between
+// the prologue and the dependency wait (a chain requests the next layer's prologue there).
+// The x barrier must have been initialised (init_xbar) and published by a CTA barrier or be past an earlier use.
+// Returns false when the dependency wait gave up; nothing of x or y has been touched then.
+template <int U, class Dep, class Early = NothingEarly>
+__device__ __forceinline__ bool stream_f16_layer(const StreamArgs& a, const CtaDesc d, unsigned char* smem_raw,
+                                                 uint32_t x_parity, const Dep& dep, bool prologue_done = false,
+                                                 const Early& early = Early{}) {
     constexpr int RG = 16;
-    const StreamArgs& a = P.a;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
     const SmemLayout L = carve(smem_raw, RG, U, a, 2);
     __half* xs = static_cast<__half*>(L.xs);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
-    const CtaDesc d = cta_range(P);
     const int wbeg = warp_begin(d, warp), wend = warp_begin(d, warp + 1);
-    if (tid <= kStreamWarps) L.wb[tid] = warp_begin(d, tid);
 
-    // 1. the next kernel in the stream may start its own prologue; this one prefetches what does
-    //    not depend on its predecessor: tables, first U weight fragments, column offsets
+    // 1. the consumer of this layer may start its own prologue; this one prefetches what does
+    //    not depend on its producer: tables, first U weight fragments, column offsets
     trace_stamp(a, 0);
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    init_xbar(L);
-    issue_static<RG>(a, d, L);
+    dep.release();
+    if (!prologue_done) stream_f16_prologue<U>(a, d, smem_raw);
     const WeightRing<U> ring{L.ring + (warp * U) * 32 + lane, reinterpret_cast<const uint4*>(a.values) + lane};
-    ring.prologue(wbeg, wend);
+    early();
     XoffWindow xw;
     xw.init(a.xoff, wbeg, wend, lane);
     warm_translations(a);
 
-    // 2. everything before this kernel in the stream is complete from here on: fetch x
+    // 2. everything the producer wrote is complete from here on: fetch x
     //    (the barrier publishes the mbarrier's initialisation to the threads that will wait on it)
     __syncthreads();
     trace_stamp(a, 1);
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!dep.wait()) {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");     // the prologue's copies land before shared memory is given back
+        return false;
+    }
     trace_stamp(a, 2);
     issue_x<__half>(a, L);
 
     // 3. pivoted x in shared memory
-    finish_stage<__half, U>(a, L);
+    finish_stage<__half, U>(a, L, x_parity);
     trace_stamp(a, 3);
     plan_parks(d, L);
 
@@ -618,6 +667,125 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_co
     trace_stamp(a, 4);
     finalize<RG>(a, d, L);
     trace_stamp(a, 5);
+    return true;
+}
+
+template <int U>
+__global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_constant__ StreamLaunch P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    init_xbar(carve(smem_raw, 16, U, P.a, 2));
+    stream_f16_layer<U>(P.a, cta_range(P), smem_raw, 0u, LaunchDependency{});
+}
+
+// ------------------------------------------------------------------ a whole chain of fp16 layers in one kernel
+// Cooperative launch (every CTA resident).  CTA c runs its range of layer 0, then of layer 1, ...; between two
+// layers the grid meets at a counter in global memory: a CTA that has stored its part of layer l adds one, and
+// before it reads layer l's output it waits until all CTAs have done so.  The tables and the first weights of
+// layer l + 1 are requested BEFORE that wait, so they arrive while the slowest CTA of layer l finishes; for layers
+// of a few MiB that is the whole layer.  The wait is bounded: when it gives up the CTA raises the status word and
+// leaves; every other CTA sees the word inside its own wait and leaves too.
+struct GridCounterDependency {
+    unsigned* counter;
+    unsigned target;         // arrivals that complete the producer layer (0: nothing to wait for)
+    int* status;
+    int polls;
+    __device__ __forceinline__ void release() const {}
+    __device__ __forceinline__ bool wait() const {
+        __shared__ int ok_flag;
+        if (threadIdx.x == 0) {
+            int ok = target == 0u;
+            for (int i = 0; i < polls && !ok; ++i) {
+                unsigned seen;
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+                ok = seen >= target;
+                if (!ok && (i & 63) == 63 && *reinterpret_cast<volatile int*>(status)) break;
+            }
+            if (!ok) *status = 1;
+            // the producer's stores came through the generic proxy; x is fetched by bulk copies (asynchronous proxy)
+            asm volatile("fence.proxy.async.global;" ::: "memory");
+            ok_flag = ok;
+        }
+        __syncthreads();
+        return ok_flag != 0;
+    }
+};
+
+constexpr int kChainPolls = 1 << 22;
+
+template <int U>
+__global__ void __launch_bounds__(kThreads, 1) chain_f16_kernel(const ChainLaunch P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ StreamArgs args[kChainMaxLayers];
+    __shared__ CtaDesc desc[kChainMaxLayers];
+    const unsigned n_ctas = gridDim.x;
+    // Two shared-memory regions alternate between the layers: while layer l works in one, the tables and first
+    // weights of layer l + 1 arrive in the other.
+    auto region = [&](int l) { return smem_raw + (size_t)(l & 1) * P.region_bytes; };
+    // programmatic dependent launch: the next kernel in the stream may be scheduled as CTAs of this one retire
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (threadIdx.x < 2) {          // the x barrier sits at the same place in every layer's carving of a region
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"((uint32_t)__cvta_generic_to_shared(region(threadIdx.x) + 104 * 4)));
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // all layers' arguments and this CTA's range of every layer, in two rounds of loads
+    {
+        const int n_words = P.n_layers * (int)(sizeof(StreamArgs) / 4);
+        for (int i = threadIdx.x; i < n_words; i += kThreads)
+            reinterpret_cast<uint32_t*>(args)[i] = __ldg(reinterpret_cast<const uint32_t*>(P.layers) + i);
+        __syncthreads();
+        if (threadIdx.x < P.n_layers) {
+            const int l = threadIdx.x;
+            CtaDesc dd{0, 0, 0, -1};                         // s_count < 0: this CTA is not part of the layer's plan
+            if ((int)blockIdx.x < __ldg(P.grids + l)) {
+                const int4 v = __ldg(reinterpret_cast<const int4*>(args[l].cta_desc) + blockIdx.x);
+                dd = CtaDesc{v.x, v.y, v.z, v.w};
+            }
+            desc[l] = dd;
+            if (l == 0) args[l].x = P.x;                      // the call's input and output; everything between is the chain's
+            if (l == P.n_layers - 1) args[l].y = P.y;
+            args[l].wait_polls = P.polls;
+#ifdef PP_TRACE
+            args[l].trace = P.trace ? P.trace + (size_t)l * 320 * 8 : nullptr;
+#endif
+        }
+        __syncthreads();
+    }
+    if (desc[0].s_count >= 0) stream_f16_prologue<U>(args[0], desc[0], region(0));
+    // everything before this kernel in the stream (the previous call on these buffers) is complete from here on
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    uint32_t x_uses[2] = {0u, 0u};
+    bool alive = true;
+    for (int l = 0; l < P.n_layers && alive; ++l) {
+        const StreamArgs& a = args[l];
+        const GridCounterDependency dep{P.counter, l == 0 ? 0u : n_ctas * (unsigned)l, P.status,
+                                        P.polls > 0 ? P.polls : kChainPolls};
+        auto next_prologue = [&]() {
+            if (l + 1 < P.n_layers && desc[l + 1].s_count >= 0)
+                stream_f16_prologue<U>(args[l + 1], desc[l + 1], region(l + 1));
+        };
+        if (desc[l].s_count >= 0) {
+            const bool has_x = a.stage_mode != 0 && (a.stage_mode != 2 ? a.x_len : a.x_limit) >= 8;
+            alive = stream_f16_layer<U>(a, desc[l], region(l), x_uses[l & 1] & 1u, dep, true, next_prologue);
+            if (alive && has_x) ++x_uses[l & 1];
+        } else {
+            next_prologue();
+            __syncthreads();
+            alive = dep.wait();
+        }
+        if (alive && l + 1 < P.n_layers) {
+            // this CTA's part of layer l is stored: make it visible, then count this CTA in
+            __threadfence();
+            __syncthreads();
+            if (threadIdx.x == 0) atomicAdd(P.counter, 1u);
+        }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    // Last use of the counter by this CTA.  Whoever is last of all puts it back to zero for the next launch; a
+    // launch that gave up leaves it for the host to clear (pp_chain_status).
+    if (alive && threadIdx.x == 0) {
+        const unsigned total = n_ctas * (unsigned)P.n_layers;
+        if (atomicAdd(P.counter, 1u) == total - 1u) *P.counter = 0u;
+    }
 }
 
 // ------------------------------------------------------------------ fp32 tiles
@@ -769,6 +937,7 @@ unsigned long long* g_stream_trace = nullptr;   // diagnostic builds: [calls][kT
 int g_stream_trace_calls = 0, g_stream_trace_next = 0;
 constexpr int kTraceCtas = 320;
 #endif
+int g_stream_wait_polls = 0;   // polls before a bounded device-side wait gives up; 0 = the kernels' defaults
 int g_stream_depth = 0;   // ring slots per warp: 4, 6 or 8; 0 = chosen per launch
 int g_stream_pdl = 1;     // launch with programmatic stream serialization (prologue overlaps the previous kernel)
 
@@ -808,6 +977,74 @@ size_t smem_bytes_at(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, i
 }
 }  // namespace
 
+void stream_finish_args(pp_dtype_t dt, StreamArgs& a) {
+    a.xs_stride = xs_stride_for(dt, a.n_pad);
+    a.raw_stride = raw_stride_for(a.x_len, a.batch);
+    a.max_rows = (a.max_rows + 31) / 32 * 32;      // whole strips of either height; keeps the regions behind 128-byte aligned
+    a.wait_polls = g_stream_wait_polls;
+    a.trace = nullptr;
+}
+
+namespace {
+template <int U>
+int chain_resident_ctas_u(size_t smem) {
+    int dev = 0, sms = 0, per_sm = 0, coop = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop ||
+        cudaFuncSetAttribute(chain_f16_kernel<U>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStreamSmemLimit) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, chain_f16_kernel<U>, kThreads, smem) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    return per_sm * sms;
+}
+
+template <int U>
+cudaError_t launch_chain_u(const ChainLaunch& P, int grid, size_t smem, cudaStream_t stream) {
+    static PerDeviceOnce configured;
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (!configured.is_done(dev)) {
+        e = cudaFuncSetAttribute(chain_f16_kernel<U>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kStreamSmemLimit);
+        if (e != cudaSuccess) return e;
+        configured.mark(dev);
+    }
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_stream_pdl ? 2 : 1;
+    return cudaLaunchKernelEx(&cfg, chain_f16_kernel<U>, P);
+}
+}  // namespace
+
+int chain_resident_ctas(size_t smem, int depth) {
+    return depth == 8 ? chain_resident_ctas_u<8>(smem) : chain_resident_ctas_u<4>(smem);
+}
+
+cudaError_t launch_chain_f16(const ChainLaunch& P_in, int grid, size_t smem, int depth, cudaStream_t stream) {
+    if (smem > kStreamSmemLimit || grid < 1 || (depth != 4 && depth != 8)) return cudaErrorInvalidValue;
+    ChainLaunch P = P_in;
+    if (P.polls <= 0) P.polls = g_stream_wait_polls;
+    if (P.n_layers < 1 || P.n_layers > kChainMaxLayers || smem < 2 * (size_t)P.region_bytes) return cudaErrorInvalidValue;
+    P.trace = nullptr;
+#ifdef PP_TRACE
+    if (g_stream_trace && g_stream_trace_next + P.n_layers <= g_stream_trace_calls && grid <= kTraceCtas) {
+        P.trace = g_stream_trace + (size_t)g_stream_trace_next * kTraceCtas * 8;
+        g_stream_trace_next += P.n_layers;
+    }
+#endif
+    return depth == 8 ? launch_chain_u<8>(P, grid, smem, stream) : launch_chain_u<4>(P, grid, smem, stream);
+}
+
 size_t stream_launch_smem(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int depth) {
     return smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, depth);
 }
@@ -821,14 +1058,11 @@ cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a_in, const Ct
     if (a.batch < 1 || a.batch > kStreamMaxBatch || (a.stage_mode >= 3 && a.batch != 1 && dt != PP_F16) ||
         (a.stage_mode == 4 && !a.gather16))
         return cudaErrorInvalidValue;
-    a.xs_stride = xs_stride_for(dt, a.n_pad);
-    a.raw_stride = raw_stride_for(a.x_len, a.batch);
+    stream_finish_args(dt, a);
 #ifdef PP_TRACE
-    a.trace = nullptr;
     if (g_stream_trace && g_stream_trace_next < g_stream_trace_calls && grid <= kTraceCtas)
         a.trace = g_stream_trace + (size_t)(g_stream_trace_next++) * kTraceCtas * 8;
 #endif
-    a.max_rows = (a.max_rows + 31) / 32 * 32;      // whole strips of either height; keeps the regions behind 128-byte aligned
     if (grid <= kParamCtas)
         for (int c = 0; c < grid; ++c) P.table[c] = host_table[c];
     const int depth = stream_pick_depth(dt, B, a.n_pad, a.x_len, a.max_rows, a.batch, a.stage_mode, grid);

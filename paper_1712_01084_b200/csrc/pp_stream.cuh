@@ -21,6 +21,7 @@ struct StreamArgs {
     float* partials;             // [stream_slots][rows_per_strip * kStreamMaxBatch]
     int* counters;               // [S], zero between launches
     int* status;                 // raised to 1 when the bounded wait for the copy of x gave up; may be NULL
+    int wait_polls;              // polls before the bounded wait for the copy of x gives up (0: the kernel's default; set by the launcher)
     unsigned long long* trace;   // diagnostic builds (PP_TRACE): [grid][8] time stamps of the kernel's phases; else unused
     int ldx, ldy;
     int x_limit;                 // with gather_idx == NULL: columns >= x_limit read 0
@@ -49,6 +50,28 @@ size_t stream_launch_smem(pp_dtype_t dt, int B, int n_pad, int x_len, int max_ro
 extern int g_stream_depth;   // weight-ring slots per warp: 4, 6 or 8; 0 = chosen per launch
 extern int g_stream_pdl;     // 1: launch with programmatic stream serialization
 constexpr size_t kStreamSmemLimit = 224 * 1024;
+
+// A chain of fp16 layers in one cooperative kernel (batch <= 8).  `layers` holds one complete StreamArgs per layer
+// (as stream_finish_args leaves them; cta_desc must point to the plan in device memory); x of the first and y of
+// the last layer come with the launch.
+constexpr int kChainMaxLayers = 8;
+struct ChainLaunch {
+    const StreamArgs* layers;    // device, [n_layers]
+    const int* grids;            // device, [n_layers]: CTAs of each layer's plan (<= the launch's grid)
+    const void* x;               // input of layer 0
+    void* y;                     // output of the last layer
+    unsigned* counter;           // device, zero between launches: arrivals at the layer boundaries
+    int* status;                 // raised to 1 when a bounded wait gave up
+    int n_layers;
+    int region_bytes;            // bytes of one of the two shared-memory regions the layers alternate between
+    int polls;                   // polls of a boundary wait before it gives up (0: default)
+    unsigned long long* trace;   // diagnostic builds (PP_TRACE): [n_layers][320][8] phase stamps; else unused
+};
+void stream_finish_args(pp_dtype_t dt, StreamArgs& a);       // strides and rounding the launcher applies to a layer's arguments
+int chain_resident_ctas(size_t smem, int depth);            // CTAs of the chain kernel the device holds at once (0: no cooperative launch)
+// smem: 2 * region_bytes; depth: weight copies each warp keeps in flight (4 or 8), the same for every layer
+cudaError_t launch_chain_f16(const ChainLaunch& P, int grid, size_t smem, int depth, cudaStream_t stream);
+extern int g_stream_wait_polls;
 
 // host_table: the plan's CTA ranges in host memory (grid entries); small plans travel to the
 // kernel inside its parameters so that no CTA starts with a dependent global load.

@@ -23,6 +23,7 @@
 #include <cuda_fp16.h>
 
 #include "pp_gemv.cuh"
+#include "pp_stream.cuh"
 #include "pp_tile.cuh"
 
 namespace pp {
@@ -53,8 +54,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* b, uint32_t parity) {
                  : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: false after kPollLimit polls, or at once when another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* b, uint32_t parity) {     // never suspends the thread
+    uint32_t ok;
+    asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok) : "r"(smem_u32(b)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false after the poll limit, or at once when another role already gave up.  polls == 0 is the
+// normal case (kPollLimit polls that may each suspend the thread for a while: seconds in all).  A caller-set
+// limit counts polls that return at once, so that a test can make a wait run out on purpose.
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort_flag, int polls) {
+    if (polls > 0) {
+        for (int i = 0; i < polls; ++i) {
+            if (mbar_test_wait(b, parity)) return true;
+            if (*abort_flag) return false;
+        }
+        *abort_flag = 1;
+        return false;
+    }
     for (int i = 0; i < kPollLimit; ++i) {
         if (mbar_try_wait(b, parity)) return true;
         if ((i & 1023) == 1023 && *abort_flag) return false;
@@ -172,7 +189,7 @@ tile_f16_kernel(const TileArgs a) {
             const int rot = k > 0 ? (int)(((long long)br * k) / gridDim.x) : 0;
             for (int t = warp; t < k; t += kProducers) {
                 const int s = t % kStages;
-                if (t >= kStages && !mbar_wait(&sm->empty[s], ((t / kStages) & 1) ^ 1, abort_flag)) break;
+                if (t >= kStages && !mbar_wait(&sm->empty[s], ((t / kStages) & 1) ^ 1, abort_flag, a.polls)) break;
                 // block-rows start at different tiles of their lists, so that CTAs running side by side
                 // do not all ask the L2 for the same X segment at the same moment
                 const int tt = (t + rot) % k;
@@ -195,21 +212,24 @@ tile_f16_kernel(const TileArgs a) {
     } else if (warp == kProducers) {
         // ---------------- MMA issuer (one lane)
         if (lane == 0) {
-            bool ok = true;
+            bool ok = true, issued = false;
             const uint64_t desc0 = smem_desc_sw128(smem_u32(stages));
             for (int t = 0; t < k && ok; ++t) {
                 const int s = t % kStages;
-                ok = mbar_wait(&sm->full[s], (t / kStages) & 1, abort_flag);
+                ok = mbar_wait(&sm->full[s], (t / kStages) & 1, abort_flag, a.polls);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint64_t xd = desc_advance(desc0, (uint32_t)(s * kStageBytes)), wd = desc_advance(xd, XB);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)
                     umma_f16(tmem, desc_advance(xd, kk * 32), desc_advance(wd, kk * 32), t > 0 || kk > 0);
+                issued = true;
                 umma_commit(&sm->empty[s]);          // frees the stage once these MMAs have read it
             }
-            if (k > 0 && ok) umma_commit(&sm->acc_full);   // accumulator complete
-            else mbar_arrive(&sm->acc_full);               // nothing to wait for (no tile, or giving up)
+            // accumulator complete; when giving up after some tiles, the epilogue (and the release of tensor
+            // memory behind it) still waits for the instructions already issued
+            if (issued) umma_commit(&sm->acc_full);
+            else mbar_arrive(&sm->acc_full);               // nothing was issued: nothing to wait for
         }
     } else {
         // ---------------- epilogue: 4 warps, warp (w % 4) owns tensor-memory lanes 32 (w % 4) ..
@@ -223,7 +243,7 @@ tile_f16_kernel(const TileArgs a) {
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         // the tensor-memory loads below are warp-wide instructions: the whole warp takes one decision
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(&sm->acc_full, 0, abort_flag) && !*abort_flag);
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(&sm->acc_full, 0, abort_flag, 0) && !*abort_flag);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (ok && q * 32 < a.batch) {
 #pragma unroll
@@ -396,7 +416,7 @@ tile_cluster_f16_kernel(const TileArgs a) {
             int last = -1;
             const uint32_t xbytes = (uint32_t)((a.batch + 7) / 8) * 1024u;   // live 8-row groups of the X block only
             for (int t = warp; t < n_steps; t += kCProducers) {
-                if (t >= kCStages && !mbar_wait(&sm->empty[s], ((t / kCStages) & 1) ^ 1, abort_flag)) break;
+                if (t >= kCStages && !mbar_wait(&sm->empty[s], ((t / kCStages) & 1) ^ 1, abort_flag, a.polls)) break;
                 const TileStep st = step_at((t + rot) % n_steps);
                 unsigned char* dst = stages + s * kCStageBytes;
                 mbar_expect_tx(&sm->full[s], xbytes + (uint32_t)(st.ntiles * kWBytes));
@@ -420,7 +440,7 @@ tile_cluster_f16_kernel(const TileArgs a) {
             for (int t = 0; t < n_steps && ok; ++t) {
                 const int s = t % kCStages;
                 const TileStep st = step_at((t + rot) % n_steps);
-                ok = mbar_wait(&sm->full[s], (t / kCStages) & 1, abort_flag);
+                ok = mbar_wait(&sm->full[s], (t / kCStages) & 1, abort_flag, a.polls);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t xa = smem_u32(stages + s * kCStageBytes);
@@ -445,8 +465,8 @@ tile_cluster_f16_kernel(const TileArgs a) {
                 umma_commit(&sm->empty[s]);          // frees the stage once these MMAs have read it
             }
             sm->acc_mask = ok ? mask : 0u;
-            if (mask != 0u && ok) umma_commit(&sm->acc_full);   // accumulators complete
-            else mbar_arrive(&sm->acc_full);                    // nothing in flight to wait for (no tile, or giving up)
+            if (mask != 0u) umma_commit(&sm->acc_full);         // accumulators complete (also when giving up: whatever was issued must finish)
+            else mbar_arrive(&sm->acc_full);                    // nothing was issued: nothing to wait for
             mbar_arrive(&sm->acc_full);                         // releases acc_mask to the epilogue warps
         }
     }
@@ -462,7 +482,7 @@ tile_cluster_f16_kernel(const TileArgs a) {
             sm->bias[b] = live ? __ldg(a.bias_piv + br * 64 + b) : 0.0f;
             sm->dst[b] = live ? (a.pivoted ? br * 64 + b : __ldg(a.scatter_idx + br * 64 + b)) : -1;
         }
-        ok = __all_sync(0xffffffffu, mbar_wait(&sm->acc_full, 0, abort_flag) && !*abort_flag);
+        ok = __all_sync(0xffffffffu, mbar_wait(&sm->acc_full, 0, abort_flag, 0) && !*abort_flag);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -628,8 +648,10 @@ cudaError_t launch_one_row(const TileArgs& a, int Mb, cudaStream_t stream) {
     return launch_after_gather(tile_f16_kernel<STAGES, XB>, Mb, kThreads, smem, a, stream);
 }
 
-cudaError_t launch_tile(const TileArgs& a, const void* x, int ldx, int n, const int32_t* gather_idx, int n_pad, int Mb,
+cudaError_t launch_tile(const TileArgs& a_in, const void* x, int ldx, int n, const int32_t* gather_idx, int n_pad, int Mb,
                         bool use_cluster, cudaStream_t stream) {
+    TileArgs a = a_in;
+    a.polls = g_stream_wait_polls;
     if (a.batch < 1 || a.batch > kTileBatch) return cudaErrorInvalidValue;
     if ((size_t)n * 2 > 48 * 1024) return cudaErrorInvalidValue;
     // rows past the batch keep whatever an earlier call left there: every row of the product is independent

@@ -23,6 +23,7 @@ struct TileArgs {
     int batch;                   // rows of this chunk (1..kTileBatch)
     int act;
     int pivoted;                 // 1: y[b][pivoted row] (Section 4.2.2), 0: y[b][scatter_idx[pivoted row]]
+    int polls;                   // polls after which a bounded wait gives up (0: the kernels' own limit; set by the launcher)
     // clustered kernel only
     const TileStep* steps;       // steps of all groups
     const int32_t* parts;        // [groups][kTileRows + 1] step boundaries of each cluster's CTAs

@@ -225,12 +225,21 @@ def _chain_bound(layers, res, dtype_tol):
     return e
 
 
+@pytest.fixture(params=[1, 0], ids=["one_kernel", "kernel_per_layer"])
+def chain_mode(request, pb):
+    """Chains of fp16 layers run as one cooperative kernel (tuning key 14 = 1) or one launch per layer (default)."""
+    pb.pp_set_tuning(14, request.param)
+    yield request.param
+    pb.pp_set_tuning(14, 0)
+
+
 @pytest.mark.parametrize("batch", [1, 8])
-def test_config3_chain_full(pb, batch):
+def test_config3_chain_full(pb, batch, chain_mode):
     wl = synth.config3(batch=batch)
     layers = [pb.Layer.from_synth(l) for l in wl.layers]
     chain = pb.Chain(layers, [l.act for l in wl.layers], max_batch=8)
     y = pb.pp_chain_forward(chain, _dev(wl.x)).cpu().numpy().astype(np.float64)
+    assert chain.status() == 0
     res = po.chain_forward(wl.layers, wl.x.astype(np.float64), round_intermediate="f16", threads=8)
     bound = _chain_bound(wl.layers, res, TOL[np.dtype(np.float16)])
     worst = np.max(np.abs(y - res[-1][1]) / bound)
@@ -242,6 +251,40 @@ def test_config3_chain_full(pb, batch):
         _check(yl, res[li][1], res[li][2], np.float16, f"config 3 layer {li}")
     chain.close()
     for l in layers:
+        l.close()
+
+
+@pytest.mark.parametrize("B,dims", [(16, [200, 150, 90, 33]), (32, [700, 333, 64, 129, 10]), (64, [256, 1000, 70])])
+@pytest.mark.parametrize("batch", [1, 3, 8])
+def test_chain_one_kernel_equals_kernel_per_layer(pb, B, dims, batch):
+    """fp16 chains: the cooperative one-kernel execution, the launch-per-layer execution and the oracle give the
+    same bits on integer data (ragged sizes, empty block-rows, layers whose plans have different CTA counts,
+    twice in a row: the boundary counter must be left clean)."""
+    lays = []
+    for l in range(len(dims) - 1):
+        lay = _rand_layer(900 + 10 * B + l, dims[l + 1], dims[l], B, np.float16, density=0.5, integer=True,
+                          empty_rows=(1,) if l == 1 else ())
+        lay.tile_values = (np.sign(lay.tile_values) * (np.abs(lay.tile_values) > 3)).astype(np.float16)   # entries in {-1,0,1}
+        lay.bias = np.sign(lay.bias).astype(np.float32)
+        lay.act = 1 if l + 2 < len(dims) else 0
+        lays.append(lay)
+    x = np.random.default_rng(B + batch).integers(-1, 2, (batch, dims[0])).astype(np.float16)
+    L = [pb.Layer.from_synth(l) for l in lays]
+    outs = []
+    try:
+        pb.pp_set_tuning(14, 1)                         # read when the chain is created and at every call
+        chain = pb.Chain(L, [l.act for l in lays], max_batch=8)
+        for mode in (1, 1, 0):
+            pb.pp_set_tuning(14, mode)
+            outs.append(pb.pp_chain_forward(chain, _dev(x)).cpu().numpy())
+            assert chain.status() == 0
+    finally:
+        pb.pp_set_tuning(14, 0)
+    assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])
+    res = po.chain_forward(lays, x.astype(np.float64), round_intermediate="f16")
+    assert np.array_equal(outs[0].astype(np.float64), res[-1][1])
+    chain.close()
+    for l in L:
         l.close()
 
 
