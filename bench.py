@@ -349,8 +349,9 @@ def roof_fields(peaks, abytes, us, flops=None):
 def paper_geometry(pb, torch, synth, sizes=(64, 128, 256, 512, 1024, 2048, 4096), per_sides=(32, 16, 8, 4)):
     """The geometry the paper itself measures (Section 5): size x size, 1/fill-in square blocks on the diagonal
     of the pivoted matrix, batch 1, here fp32.  Per case: this library's kernels (blocks through
-    pp_layer_create_blocks, grid = block edge clamped to 16..64) and the plain one-thread-per-row kernels in the
-    three physical layouts of Section 4.1.1.  "warm" repeats one layer as the paper's 2,500-call average does;
+    pp_layer_create_blocks, grid = block edge clamped to 16..64) and the plain kernels of the layout study: the
+    three physical layouts of Section 4.1.1 ("brc", "bcr", "cbr") with a lane per output row ("rows") and with
+    the lanes of a warp along the columns ("k").  "warm" repeats one layer as the paper's 2,500-call average does;
     "cold" rotates copies that together exceed twice the L2 (given where at most 96 copies do)."""
     geo = {}
     for size in sizes:
@@ -373,12 +374,12 @@ def paper_geometry(pb, torch, synth, sizes=(64, 128, 256, 512, 1024, 2048, 4096)
                 for r in reps[1:]:
                     r.close()
             L0.close()
-            if edge <= 1024:
-                x1, y1 = x.reshape(-1), y.reshape(-1)
-                fl = pb.lib().pp_listing1_forward
+            x1, y1 = x.reshape(-1), y.reshape(-1)
+            fl = pb.lib().pp_layout_forward
+            for mname, mapping in (("rows", pb.PP_MAP_ROWS_PER_LANE), ("k", pb.PP_MAP_LANES_ALONG_K)):
                 for name, layout in (("brc", pb.PP_LAYOUT_BRC), ("bcr", pb.PP_LAYOUT_BCR), ("cbr", pb.PP_LAYOUT_CBR)):
-                    K = pb.Listing1(size, per_side, layout, lay.row_perm, lay.col_perm, lay.block_values)
-                    row[f"row_per_thread_{name}_us_warm"] = round(quick_us(
+                    K = pb.LayoutStudy(size, per_side, layout, mapping, lay.row_perm, lay.col_perm, lay.block_values)
+                    row[f"{mname}_{name}_us_warm"] = round(quick_us(
                         torch, lambda i, sp: _check_status(pb, fl(K._h, x1.data_ptr(), y1.data_ptr(), sp)), 64), 3)
                     K.close()
             geo[f"size{size}_fill{100.0 / per_side:g}"] = row

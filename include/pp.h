@@ -345,34 +345,34 @@ pp_status_t pp_pivot_find(int M, int N, const float* abs_w, int levels, int max_
                           double* kept_sum_out);
 
 /* ------------------------------------------------------------------------- *
- * The paper's own kernel model (Section 4.1.1 and Listing 1), for the layout
- * study of Section 4.1.1 and as the baseline the other kernels are measured
- * against: one thread group per block, one thread per output coordinate running
- * along its row of the block, the block's input slice fetched by the group
- * through the column index array, the result stored through the row index array.
- * Geometry of Section 5: a size x size matrix, n_blocks identical square blocks
- * of edge size / n_blocks, block k on pivoted rows and columns [k*edge, (k+1)*edge).
- * fp32, one input vector, no bias, no activation.
+ * Layout study (Section 4.1.1, Table 2): plain fp32 kernels over the three physical layouts of M_block the
+ * paper compares, crossed with two ways of giving the work to threads.  They exist to repeat the paper's
+ * comparison on this GPU and as the yardstick for the library's own kernels; no other call uses them.
+ * Geometry of Section 5: a size x size matrix, n_blocks identical square blocks of edge size / n_blocks,
+ * block k on pivoted rows and columns [k*edge, (k+1)*edge).  One input vector, no bias, no activation.
  *
  * layout: physical order of M_block (rightmost axis fastest):
  *   PP_LAYOUT_BRC block,row,column  PP_LAYOUT_BCR block,column,row  PP_LAYOUT_CBR column,block,row
+ * mapping: PP_MAP_ROWS_PER_LANE   a lane owns one output row and walks along it (the thread mapping the
+ *                                 paper describes: one thread per output coordinate);
+ *          PP_MAP_LANES_ALONG_K   a warp owns four output rows, its lanes stride over the columns and
+ *                                 the row sums are finished by a shuffle reduction.
  * row_perm, col_perm   host, int32[size], pivoted -> original (no padding)
  * block_values         host, float[n_blocks][edge][edge], row-major per block
  * x, y                 device, float[size]; must not alias
- * pp_listing1_pack writes the values in the chosen layout to host memory out
- * (n_blocks*edge*edge floats); create uses it before the upload.
- * Errors: PP_ERR_INVALID_ARG (sizes, NULL, size not a multiple of n_blocks),
- * PP_ERR_BAD_PERM, PP_ERR_UNSUPPORTED when edge > 1024 (one thread per block row),
- * PP_ERR_ALLOC, PP_ERR_CUDA.  pp_listing1_forward only enqueues.
+ * pp_layout_pack writes the values in the chosen layout to host memory out (n_blocks*edge*edge floats);
+ * create uses it before the upload.
+ * Errors: PP_ERR_INVALID_ARG (sizes, NULL, size not a multiple of n_blocks, unknown layout or mapping),
+ * PP_ERR_BAD_PERM, PP_ERR_ALLOC, PP_ERR_CUDA.  pp_layout_forward only enqueues.
  * ------------------------------------------------------------------------- */
-typedef struct pp_listing1 pp_listing1_t;
+typedef struct pp_layout_study pp_layout_study_t;
 typedef enum { PP_LAYOUT_BRC = 0, PP_LAYOUT_BCR = 1, PP_LAYOUT_CBR = 2 } pp_layout_t;
-pp_status_t pp_listing1_pack(int size, int n_blocks, pp_layout_t layout, const float* block_values, float* out);
-pp_status_t pp_listing1_create(pp_listing1_t** out, int size, int n_blocks, pp_layout_t layout,
-                               const int32_t* row_perm, const int32_t* col_perm,
-                               const float* block_values);
-pp_status_t pp_listing1_destroy(pp_listing1_t* h);
-pp_status_t pp_listing1_forward(pp_listing1_t* h, const float* x, float* y, void* cuda_stream);
+typedef enum { PP_MAP_ROWS_PER_LANE = 0, PP_MAP_LANES_ALONG_K = 1 } pp_mapping_t;
+pp_status_t pp_layout_pack(int size, int n_blocks, pp_layout_t layout, const float* block_values, float* out);
+pp_status_t pp_layout_create(pp_layout_study_t** out, int size, int n_blocks, pp_layout_t layout, pp_mapping_t mapping,
+                             const int32_t* row_perm, const int32_t* col_perm, const float* block_values);
+pp_status_t pp_layout_destroy(pp_layout_study_t* h);
+pp_status_t pp_layout_forward(pp_layout_study_t* h, const float* x, float* y, void* cuda_stream);
 
 /* ------------------------------------------------------------------------- *
  * Forward call that allocates nothing (the paper has no counterpart; this is a

@@ -80,10 +80,10 @@ def lib() -> ctypes.CDLL:
         "pp_lstm_forward": (ci, [vp, vp, vp, vp, ci, vp]),
         "pp_lstm_status": (ci, [vp, ctypes.POINTER(ci)]),
         "pp_pivot_find": (ci, [ci, ci, fp, ci, ci, i32p, i32p, i32p, i32p, i32p, ctypes.POINTER(ctypes.c_double)]),
-        "pp_listing1_pack": (ci, [ci, ci, ci, fp, fp]),
-        "pp_listing1_create": (ci, [ctypes.POINTER(vp), ci, ci, ci, i32p, i32p, fp]),
-        "pp_listing1_destroy": (ci, [vp]),
-        "pp_listing1_forward": (ci, [vp, vp, vp, vp]),
+        "pp_layout_pack": (ci, [ci, ci, ci, fp, fp]),
+        "pp_layout_create": (ci, [ctypes.POINTER(vp), ci, ci, ci, ci, i32p, i32p, fp]),
+        "pp_layout_destroy": (ci, [vp]),
+        "pp_layout_forward": (ci, [vp, vp, vp, vp]),
         "pp_pack_device_image_bytes": (ci, [vp, i64p]),
         "pp_pack_device_image": (ci, [vp, vp, c64]),
         "pp_forward_noalloc": (ci, [vp, vp, vp, vp, ci, ci, vp]),
@@ -558,32 +558,33 @@ def pp_lstm_forward(lstm: Lstm, x_seq, h, c, stream=None):
     return h, c
 
 
-# ------------------------------------------------- the paper's kernel model (Listing 1)
+# ------------------------------------------------- layout study (Section 4.1.1)
 PP_LAYOUT_BRC, PP_LAYOUT_BCR, PP_LAYOUT_CBR = 0, 1, 2
+PP_MAP_ROWS_PER_LANE, PP_MAP_LANES_ALONG_K = 0, 1
 
 
-def pp_listing1_pack(size, n_blocks, layout, block_values) -> np.ndarray:
+def pp_layout_pack(size, n_blocks, layout, block_values) -> np.ndarray:
     bv = np.ascontiguousarray(block_values, dtype=np.float32).reshape(-1)
     out = np.empty_like(bv)
     fp = ctypes.POINTER(ctypes.c_float)
-    _check(lib().pp_listing1_pack(int(size), int(n_blocks), int(layout), bv.ctypes.data_as(fp), out.ctypes.data_as(fp)),
-           "pp_listing1_pack")
+    _check(lib().pp_layout_pack(int(size), int(n_blocks), int(layout), bv.ctypes.data_as(fp), out.ctypes.data_as(fp)),
+           "pp_layout_pack")
     return out
 
 
-class Listing1:
-    """The paper's kernel (one thread group per block, one thread per output row) with a chosen
-    physical layout of the blocks (pp_listing1_create / pp_listing1_forward)."""
+class LayoutStudy:
+    """Plain fp32 kernel over one physical layout of the blocks and one thread mapping
+    (pp_layout_create / pp_layout_forward): the yardstick of the layout study."""
 
-    def __init__(self, size, n_blocks, layout, row_perm, col_perm, block_values):
+    def __init__(self, size, n_blocks, layout, mapping, row_perm, col_perm, block_values):
         rp, rpp = _i32(row_perm)
         cp, cpp = _i32(col_perm)
         bv = np.ascontiguousarray(block_values, dtype=np.float32).reshape(-1)
         if size % n_blocks or bv.size != n_blocks * (size // n_blocks) ** 2 or rp.size != size or cp.size != size:
             raise ValueError("sizes do not describe n_blocks square blocks of edge size/n_blocks")
         self._h = ctypes.c_void_p()
-        _check(lib().pp_listing1_create(ctypes.byref(self._h), int(size), int(n_blocks), int(layout), rpp, cpp,
-                                        bv.ctypes.data_as(ctypes.POINTER(ctypes.c_float))), "pp_listing1_create")
+        _check(lib().pp_layout_create(ctypes.byref(self._h), int(size), int(n_blocks), int(layout), int(mapping), rpp, cpp,
+                                      bv.ctypes.data_as(ctypes.POINTER(ctypes.c_float))), "pp_layout_create")
         self.size = int(size)
 
     def forward(self, x, out=None, stream=None):
@@ -592,12 +593,12 @@ class Listing1:
         if x.dtype != torch.float32 or x.numel() != self.size:
             raise ValueError("x must be float32 with `size` elements")
         y = torch.empty(self.size, dtype=torch.float32, device=x.device) if out is None else out
-        _check(lib().pp_listing1_forward(self._h, x.data_ptr(), y.data_ptr(), _stream_ptr(stream)), "pp_listing1_forward")
+        _check(lib().pp_layout_forward(self._h, x.data_ptr(), y.data_ptr(), _stream_ptr(stream)), "pp_layout_forward")
         return y
 
     def close(self):
         if self._h:
-            lib().pp_listing1_destroy(self._h)
+            lib().pp_layout_destroy(self._h)
             self._h = ctypes.c_void_p()
 
     def __del__(self):

@@ -97,15 +97,17 @@ def test_block_layer_in_a_chain(pb):
     ch.close(); L0.close(); L1.close()
 
 
-# ------------------------------------------------ the paper's kernel model (Section 4.1.1, Listing 1)
-@pytest.mark.parametrize("layout", [0, 1, 2])
-@pytest.mark.parametrize("size,blocks_per_side", [(512, 16), (1024, 4), (96, 8), (2048, 2), (60, 5)])
-def test_listing1_kernel_layouts(pb, layout, size, blocks_per_side):
-    """One thread group per block, one thread per output row, in the three layouts; same numbers as the oracle."""
+# ------------------------------------------------ layout study (Section 4.1.1): three layouts x two thread mappings
+@pytest.mark.parametrize("mapping", [0, 1], ids=["rows_per_lane", "lanes_along_k"])
+@pytest.mark.parametrize("layout", [0, 1, 2], ids=["brc", "bcr", "cbr"])
+@pytest.mark.parametrize("size,blocks_per_side", [(512, 16), (1024, 4), (96, 8), (4096, 2), (60, 5), (2600, 2)])
+def test_layout_study_kernels(pb, layout, mapping, size, blocks_per_side):
+    """Every layout with every mapping gives the oracle's numbers (block edges from 12 to 2048: below a warp,
+    ragged against the 128-row and 32-row CTA shapes, and longer than one staged chunk of 1024 columns)."""
     for integer in (False, True):
         wl = synth.paper_square(size, blocks_per_side, 1, wdtype="f32", integer_values=integer)
         lay = wl.layers[0]
-        K = pb.Listing1(size, blocks_per_side, layout, lay.row_perm, lay.col_perm, lay.block_values)
+        K = pb.LayoutStudy(size, blocks_per_side, layout, mapping, lay.row_perm, lay.col_perm, lay.block_values)
         y = K.forward(torch.from_numpy(wl.x[0]).cuda()).cpu().numpy()
         K.close()
         y_ref, _, a = _reference(lay, wl.x, 0)
@@ -115,14 +117,16 @@ def test_listing1_kernel_layouts(pb, layout, size, blocks_per_side):
             assert np.all(np.abs(y.astype(np.float64) - y_ref[0]) <= 1e-5 * a[0] + 1e-6)
 
 
-def test_listing1_rejects_what_it_cannot_run(pb):
-    rp = np.arange(4096, dtype=np.int32)
+def test_layout_study_rejects_bad_arguments(pb):
+    rp = np.arange(64, dtype=np.int32)
+    v = np.zeros(4 * 16 * 16, dtype=np.float32)
     with pytest.raises(pb.PPError) as e:
-        pb.Listing1(4096, 2, 0, rp, rp, np.zeros(2 * 2048 * 2048, dtype=np.float32))     # 2048 threads per group
-    assert e.value.status == 6
-    with pytest.raises(pb.PPError) as e:
-        pb.Listing1(64, 4, 0, rp[:64][::-1] * 0, rp[:64], np.zeros(4 * 16 * 16, dtype=np.float32))
+        pb.LayoutStudy(64, 4, 0, 0, rp * 0, rp, v)                 # not a permutation
     assert e.value.status == 2
+    for layout, mapping in ((3, 0), (0, 2)):
+        with pytest.raises(pb.PPError) as e:
+            pb.LayoutStudy(64, 4, layout, mapping, rp, rp, v)
+        assert e.value.status == 1
 
 
 def test_feed_back_search_to_layer(pb):

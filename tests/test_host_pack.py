@@ -526,12 +526,12 @@ def test_blocks_error_codes():
     assert status([[-1, 0, 2, 2]], v[:4]) == 3
 
 
-# ------------------------------------------------ physical layouts of the paper's kernel (Section 4.1.1)
+# ------------------------------------------------ physical layouts of the layout study (Section 4.1.1)
 @pytest.mark.parametrize("size,nb", [(64, 4), (96, 8), (40, 5)])
-def test_listing1_layouts(size, nb):
+def test_layout_study_layouts(size, nb):
     """BRC = block,row,column; BCR = block,column,row; CBR = column,block,row (rightmost axis fastest)."""
     E = size // nb
     v = np.arange(nb * E * E, dtype=np.float32).reshape(nb, E, E)
-    assert np.array_equal(pb.pp_listing1_pack(size, nb, pb.PP_LAYOUT_BRC, v), v.reshape(-1))
-    assert np.array_equal(pb.pp_listing1_pack(size, nb, pb.PP_LAYOUT_BCR, v), v.transpose(0, 2, 1).reshape(-1))
-    assert np.array_equal(pb.pp_listing1_pack(size, nb, pb.PP_LAYOUT_CBR, v), v.transpose(2, 0, 1).reshape(-1))
+    assert np.array_equal(pb.pp_layout_pack(size, nb, pb.PP_LAYOUT_BRC, v), v.reshape(-1))
+    assert np.array_equal(pb.pp_layout_pack(size, nb, pb.PP_LAYOUT_BCR, v), v.transpose(0, 2, 1).reshape(-1))
+    assert np.array_equal(pb.pp_layout_pack(size, nb, pb.PP_LAYOUT_CBR, v), v.transpose(2, 0, 1).reshape(-1))
