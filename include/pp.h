@@ -207,8 +207,8 @@ pp_status_t pp_layer_clone(pp_layer_t** out, const pp_layer_t* src);
  * y   device, [batch][M] row-major, float, must not alias x
  * batch >= 1.  batch <= 8 runs the persistent matrix-vector kernel; larger batches run it in
  * groups of 8 columns or the chunked kernel in groups of up to 32; fp16 layers with B = 64 and
- * batch >= 9 run a tensor-core tile kernel in chunks of 128 rows (such layers keep a second,
- * row-major copy of their tiles on the device for it).
+ * batch >= 9 run a tensor-core tile kernel in chunks of 128 rows (such layers keep a second copy of their
+ * tiles on the device for it, unless they were created with tuning key 9 = 0).
  * cuda_stream: a cudaStream_t (NULL = default stream).  Enqueues only. */
 pp_status_t pp_forward(pp_layer_t* layer, const void* x, void* y, int batch,
                        pp_act_t act, void* cuda_stream);
@@ -436,7 +436,11 @@ pp_status_t pp_selftest_host(void);
  * key 8: 1 (default) launches the persistent kernel with programmatic stream serialization, 0 plainly
  * key 10: 1 (default) permutes multi-column inputs in a pre-pass kernel when the layer kernel cannot hold x
  *         twice in shared memory; 0 leaves the gather to the layer kernel; 2 always uses the pre-pass
- * key 9: smallest batch for which fp16 layers with B = 64 take the tensor-core tile path (default 9: measured faster than the matrix-vector kernels from there on; 0 = never)
+ * key 9: smallest batch for which fp16 layers with B = 64 take the tensor-core tile path (default 9: measured
+ *        faster than the matrix-vector kernels from there on; 0 = never).  Such layers hold their tiles twice on
+ *        the device (fragment order for the matrix-vector kernels, 8 KiB shared-memory images for the tile
+ *        kernels: 2 x T x 8 KiB); a layer created while this key is 0 skips the second copy and never takes the
+ *        tile path, whatever the key says later
  * key 12: tensor-core kernel of batched fp16 B = 64 layers: 0 one block-row per CTA; 2 the clustered kernel (4
  *         block-rows per cluster of 4 CTAs share every X block); 1 (default) the clustered kernel when the
  *         groups' tile-columns carry at least 3.5 of 4 possible tiles on average, else one block-row per CTA

@@ -219,6 +219,8 @@ bool alloc_layer(pp_layer* L, const LayerLayout& lo) {
 bool tile_setup(pp_layer* L, const pp_layer* from) {
     const pp_packed* pk = L->pk;
     if (pk->wdtype != PP_F16 || pk->B != 64) return true;
+    if (!from && pp::g_tile_min_batch == 0) return true;      // the tile path is switched off: no second copy of the weights
+    if (from && !from->tile_ok) return true;
     const size_t rp = round256((size_t)(pk->Mb + 1) * 4), tb = (size_t)pk->T * 64 * 64 * 2;
     const int groups = (pk->Mb + pp::kTileRows - 1) / pp::kTileRows;
     const size_t pb = round256((size_t)groups * (pp::kTileRows + 1) * 4);

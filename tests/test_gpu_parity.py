@@ -448,6 +448,26 @@ def test_tile_path_both_kernels_same_bits_and_repeatable(pb):
     L.close()
 
 
+def test_layer_created_without_tile_copy(pb):
+    """A layer created while tuning key 9 is 0 keeps no second copy of its tiles: every batch runs the
+    matrix-vector kernels, also after the key is back at its default, and clones inherit that."""
+    lay = _rand_layer(77, 4 * 64, 6 * 64, 64, np.float16, density=0.6)
+    x = np.random.default_rng(5).uniform(-1, 1, (40, lay.N)).astype(np.float16)
+    pb.pp_set_tuning(9, 0)
+    try:
+        L = pb.Layer.from_synth(lay)
+    finally:
+        pb.pp_set_tuning(9, 9)
+    C = L.clone()
+    assert L.launch_info(40)["kernel"] in ("gemv", "stream") and C.launch_info(40)["kernel"] in ("gemv", "stream")
+    y_ref, _, a = po.layer_forward(lay, x.astype(np.float64), act=1)
+    for layer in (L, C):
+        _check(pb.pp_forward(layer, _dev(x), 1).cpu().numpy(), y_ref, a, np.float16, "no tile copy")
+    full = pb.Layer.from_synth(lay)
+    assert full.launch_info(40)["kernel"] in ("tile", "tile_cluster")
+    L.close(); C.close(); full.close()
+
+
 def test_config5_batch128_tile_path_sampled_rows(pb, tile_kernel):
     """Full size (8192 x 8192, density 25 %), batch 128, in the launch configuration the bench times;
     the oracle evaluates a sample of output rows."""
