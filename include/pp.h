@@ -115,6 +115,15 @@ pp_status_t pp_pack_info(const pp_packed_t* p, int64_t out[13]);
  *        steps [b[r], b[r+1])) 15 position of every sorted tile in the step-ordered images (int32[T]) */
 pp_status_t pp_pack_get(const pp_packed_t* p, int which, void* dst, int64_t bytes);
 
+/* Plan of the persistent tensor-core kernel (fp16, B = 64) for n_ctas CTAs: the steps of pp_pack_get(13) cut into
+ * one contiguous range per CTA, balanced by bytes, and the units (part of one group of 4 block-rows that one CTA
+ * computes) in (group, step) order.  units_out: int32[n_units][8] = first step, end step, group, position among
+ * the group's units, units of the group, index of the group's first unit, 0, 0; cta_unit_out: int32[n_ctas + 1],
+ * CTA c owns units cta_unit[c] .. cta_unit[c + 1].  With units_out == cta_unit_out == NULL only *n_units_out is
+ * written.  Host only.  Errors: PP_ERR_UNSUPPORTED for other layers, PP_ERR_INVALID_ARG. */
+pp_status_t pp_pack_tile_units(const pp_packed_t* p, int n_ctas, int32_t* units_out, int64_t capacity_units,
+                               int64_t* n_units_out, int32_t* cta_unit_out);
+
 /* Inverse of the value re-ordering: writes the sorted tile list (int32[T][2])
  * and the tiles in their original row-major form ([T][B][B], wdtype). */
 pp_status_t pp_pack_unpack(const pp_packed_t* p, int32_t* tile_list_out, void* tile_values_out);
@@ -191,7 +200,7 @@ pp_status_t pp_layer_status(pp_layer_t* layer, pp_status_t* status);
 
 /* Which kernel a pp_forward call with this batch launches, and its launch shape (for reports; host only):
  * out[0] kernel: 0 chunked matrix-vector, 1 persistent matrix-vector, 2 tensor-core tile kernel with one block-row
- * per CTA, 3 clustered tensor-core tile kernel; out[1] CTAs; for the persistent kernel also out[2] asynchronous
+ * per CTA, 3 clustered tensor-core tile kernel, 4 persistent tensor-core tile kernel; out[1] CTAs; for the persistent kernel also out[2] asynchronous
  * weight copies each warp keeps in flight, out[3] bytes of dynamic shared memory per CTA, out[4] how x is staged
  * (StreamArgs::stage_mode), out[5] 1 when launched with programmatic stream serialization.  Assumes 16-byte
  * aligned x rows. */
@@ -442,8 +451,11 @@ pp_status_t pp_selftest_host(void);
  *        kernels: 2 x T x 8 KiB); a layer created while this key is 0 skips the second copy and never takes the
  *        tile path, whatever the key says later
  * key 12: tensor-core kernel of batched fp16 B = 64 layers: 0 one block-row per CTA; 2 the clustered kernel (4
- *         block-rows per cluster of 4 CTAs share every X block); 1 (default) the clustered kernel when the
- *         groups' tile-columns carry at least 3.5 of 4 possible tiles on average, else one block-row per CTA
+ *         block-rows per cluster of 4 CTAs share every X block); 3 the persistent kernel (one CTA per SM over an
+ *         equal share of the layer's steps, two accumulator sets in tensor memory, groups split between CTAs
+ *         summed through partial-sum slots in global memory in a fixed order; measured slower than the other
+ *         two, kept as an option); 1 (default) the clustered kernel when the groups' tile-columns carry at
+ *         least 3.5 of 4 possible tiles on average, else one block-row per CTA
  * key 13: 1 (default) chain links whose folded map is the identity store pivoted rows without an index array,
  *         0 sends them through the map like any other link
  * key 11: 1 (default) lets pp_lstm_forward run all steps in one cooperative kernel when the layer qualifies, 0 never

@@ -57,6 +57,7 @@ def lib() -> ctypes.CDLL:
         "pp_pack_info": (ci, [vp, i64p]),
         "pp_pack_get": (ci, [vp, ci, vp, c64]),
         "pp_pack_unpack": (ci, [vp, i32p, vp]),
+        "pp_pack_tile_units": (ci, [vp, ci, i32p, c64, i64p, i32p]),
         "pp_fold_perm": (ci, [i32p, ci, ci, i32p, ci, ci, i32p]),
         "pp_layer_create": (ci, create_args),
         "pp_layer_destroy": (ci, [vp]),
@@ -225,6 +226,17 @@ class Packed:
             return out.reshape(-1, 5)
         return out.reshape(-1, 4) if which in ("cta_desc", "strip_info") else out
 
+    def tile_units(self, n_ctas: int):
+        """Plan of the persistent tensor-core kernel for n_ctas CTAs (pp_pack_tile_units): (units [n, 8], cta_unit [n_ctas + 1])."""
+        n = ctypes.c_int64(0)
+        _check(lib().pp_pack_tile_units(self._h, int(n_ctas), None, 0, ctypes.byref(n), None), "pp_pack_tile_units")
+        units = np.zeros((n.value, 8), dtype=np.int32)
+        cta_unit = np.zeros(int(n_ctas) + 1, dtype=np.int32)
+        i32p = ctypes.POINTER(ctypes.c_int32)
+        _check(lib().pp_pack_tile_units(self._h, int(n_ctas), units.ctypes.data_as(i32p), n.value, ctypes.byref(n),
+                                        cta_unit.ctypes.data_as(i32p)), "pp_pack_tile_units")
+        return units, cta_unit
+
     def unpack(self):
         tl = np.empty((self.T, 2), dtype=np.int32)
         tv = np.empty((self.T, self.B, self.B), dtype=self.wdtype)
@@ -326,7 +338,7 @@ class Layer:
         o = np.zeros(6, dtype=np.int32)
         _check(lib().pp_layer_launch_info(self._h, int(batch), o.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))),
                "pp_layer_launch_info")
-        names = {0: "gemv", 1: "stream", 2: "tile", 3: "tile_cluster"}
+        names = {0: "gemv", 1: "stream", 2: "tile", 3: "tile_cluster", 4: "tile_persist"}
         return {"kernel": names[int(o[0])], "ctas": int(o[1]), "ring_depth": int(o[2]), "smem_bytes": int(o[3]),
                 "stage_mode": int(o[4]), "pdl": int(o[5])}
 

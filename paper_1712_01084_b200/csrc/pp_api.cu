@@ -53,6 +53,14 @@ struct pp_layer {
     pp::TileStep* d_tile_steps = nullptr;
     int n_tile_steps = 0;
     unsigned char* d_tile_scratch = nullptr;
+    // persistent tile kernel: units, first unit of every CTA, partial-sum slots, group counters (one allocation)
+    unsigned char* d_persist = nullptr;
+    pp::TileUnit* d_units = nullptr;
+    int32_t* d_cta_unit = nullptr;
+    float* d_unit_partials = nullptr;
+    int* d_group_sync = nullptr;
+    size_t group_sync_bytes = 0;
+    int persist_ctas = 0;
     void* d_x_piv = nullptr;
     int* d_status = nullptr;
     bool tile_ok = false;
@@ -143,6 +151,7 @@ void free_layer(pp_layer* L) {
     cudaFree(L->d_scratch);
     cudaFree(L->d_tile);
     cudaFree(L->d_tile_scratch);
+    cudaFree(L->d_persist);
     cudaFree(L->d_host_x);
     cudaFree(L->d_host_y);
     pp_pack_destroy(L->pk);
@@ -213,6 +222,42 @@ bool alloc_layer(pp_layer* L, const LayerLayout& lo) {
     return true;
 }
 
+// Plan of the persistent tile kernel for this device (one CTA per SM; see build_tile_units) and its device
+// blocks.  false: allocation failed.
+bool persist_setup(pp_layer* L) {
+    const pp_packed* pk = L->pk;
+    int dev = 0, sms = 0, coop = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return true;                                  // no plan: the other tile kernels remain
+    }
+    if (!coop || sms < 1) return true;
+    const int G = sms;
+    const int groups = (pk->Mb + pp::kTileRows - 1) / pp::kTileRows;
+    std::vector<pp::TileUnit> units;
+    std::vector<int32_t> cta_unit;
+    try {
+        pp::build_tile_units(pk, G, units, cta_unit);
+    } catch (const std::bad_alloc&) {
+        return false;
+    }
+    const size_t ub = round256(units.size() * sizeof(pp::TileUnit)), cb = round256(((size_t)G + 1) * 4);
+    const size_t gb = round256((size_t)groups * 2 * 4), pb = round256(pp::tile_unit_partial_bytes(units.size()));
+    if (cudaMalloc(reinterpret_cast<void**>(&L->d_persist), ub + cb + gb + pb) != cudaSuccess) return false;
+    L->d_units = reinterpret_cast<pp::TileUnit*>(L->d_persist);
+    L->d_cta_unit = reinterpret_cast<int32_t*>(L->d_persist + ub);
+    L->d_group_sync = reinterpret_cast<int*>(L->d_persist + ub + cb);
+    L->d_unit_partials = reinterpret_cast<float*>(L->d_persist + ub + cb + gb);
+    L->group_sync_bytes = gb;
+    if (cudaMemcpy(L->d_units, units.data(), units.size() * sizeof(pp::TileUnit), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(L->d_cta_unit, cta_unit.data(), cta_unit.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemset(L->d_group_sync, 0, gb) != cudaSuccess)
+        return false;
+    L->persist_ctas = G;
+    return true;
+}
+
 // Device blocks and tensor maps of the tensor-core tile path.  `host` uploads from the packed layer,
 // otherwise the weights block is copied from another layer's.  A layer that is not eligible, or a
 // driver without the tensor-map encoder, simply has no tile path (tile_plan stays NULL).
@@ -252,6 +297,7 @@ bool tile_setup(pp_layer* L, const pp_layer* from) {
             (tb && cudaMemcpy(L->d_tiles_rm, pk->tiles_rm.data(), tb, cudaMemcpyHostToDevice) != cudaSuccess))   // already swizzled by the packer
             return false;
     }
+    if (!persist_setup(L)) return false;
     L->tile_ok = true;
     return true;
 }
@@ -484,8 +530,21 @@ pp_status_t pp_layer_status(pp_layer_t* L, pp_status_t* status) {
     if (flag) {
         *status = PP_ERR_TIMEOUT;
         if (cudaMemset(L->d_status, 0, sizeof(int)) != cudaSuccess) return PP_ERR_CUDA;
+        // a persistent tile kernel that gave up may have left its group counters behind
+        if (L->d_group_sync && cudaMemset(L->d_group_sync, 0, L->group_sync_bytes) != cudaSuccess) return PP_ERR_CUDA;
     }
     return PP_OK;
+}
+
+// Which tile kernel a batched call of this layer takes: 0 one block-row per CTA, 2 clustered, 3 persistent.
+static int pick_tile_kernel(const pp_layer* L) {
+    const pp_packed* pk = L->pk;
+    if (pp::g_tile_cluster == 3) return L->persist_ctas > 0 ? 3 : 0;
+    if (pp::g_tile_cluster == 0 || pp::g_tile_cluster == 2) return pp::g_tile_cluster;
+    if (L->persist_ctas > 0 && pp::g_tile_persist_auto) return 3;
+    // The clustered kernel pays an exchange between its CTAs and walks every tile-column some block-row of
+    // a group uses: it wins (measured) once a step carries 3.5 of its 4 possible tiles on average.
+    return L->n_tile_steps > 0 && 2 * pk->T >= 7 * (int64_t)L->n_tile_steps ? 2 : 0;
 }
 
 pp_status_t pp_layer_launch_info(const pp_layer_t* L, int batch, int32_t out[6]) {
@@ -493,10 +552,9 @@ pp_status_t pp_layer_launch_info(const pp_layer_t* L, int batch, int32_t out[6])
     const pp_packed* pk = L->pk;
     for (int i = 0; i < 6; ++i) out[i] = 0;
     if (L->tile_ok && pp::g_tile_min_batch > 0 && batch >= pp::g_tile_min_batch && (size_t)pk->N * 2 <= 48 * 1024) {
-        const bool use_cluster = pp::g_tile_cluster == 2 ||
-                                 (pp::g_tile_cluster == 1 && L->n_tile_steps > 0 && 2 * pk->T >= 7 * (int64_t)L->n_tile_steps);
-        out[0] = use_cluster ? 3 : 2;
-        out[1] = use_cluster ? (pk->Mb + pp::kTileRows - 1) / pp::kTileRows * pp::kTileRows : pk->Mb;
+        const int kernel = pick_tile_kernel(L);
+        out[0] = kernel == 3 ? 4 : kernel == 2 ? 3 : 2;
+        out[1] = kernel == 3 ? L->persist_ctas : kernel == 2 ? (pk->Mb + pp::kTileRows - 1) / pp::kTileRows * pp::kTileRows : pk->Mb;
         return PP_OK;
     }
     const int nb = batch < pp::kStreamMaxBatch ? batch : pp::kStreamMaxBatch;
@@ -528,15 +586,14 @@ static pp_status_t forward_impl(pp_layer* L, const void* x, void* y, int batch, 
         t.tiles_sw = static_cast<const unsigned char*>(L->d_tiles_rm); t.x_sw = static_cast<const unsigned char*>(L->d_x_piv);
         t.ldy = ldy; t.act = (int)act; t.pivoted = pivoted ? 1 : 0;
         t.steps = L->d_tile_steps; t.parts = L->d_tile_parts; t.Mb = pk->Mb; t.tile_pos = L->d_tile_pos;
-        // The clustered kernel pays an exchange between its CTAs and walks every tile-column some block-row of
-        // a group uses: it wins (measured) once a step carries 3.5 of its 4 possible tiles on average.
-        const bool use_cluster = pp::g_tile_cluster == 2 ||
-                                 (pp::g_tile_cluster == 1 && L->n_tile_steps > 0 && 2 * pk->T >= 7 * (int64_t)L->n_tile_steps);
+        t.units = L->d_units; t.cta_unit = L->d_cta_unit; t.unit_partials = L->d_unit_partials;
+        t.group_sync = L->d_group_sync; t.persist_ctas = L->persist_ctas;
+        const int kernel = pick_tile_kernel(L);
         for (int b0 = 0; b0 < batch; b0 += pp::kTileBatch) {
             t.batch = batch - b0 < pp::kTileBatch ? batch - b0 : pp::kTileBatch;
             t.y = static_cast<float*>(y) + (size_t)b0 * ldy;
             const char* xc = static_cast<const char*>(x) + (size_t)b0 * pk->N * 2;
-            if (pp::launch_tile(t, xc, pk->N, pk->N, L->d_gather, pk->Npad, pk->Mb, use_cluster, stream) != cudaSuccess)
+            if (pp::launch_tile(t, xc, pk->N, pk->N, L->d_gather, pk->Npad, pk->Mb, kernel, stream) != cudaSuccess)
                 return PP_ERR_CUDA;
         }
         return PP_OK;

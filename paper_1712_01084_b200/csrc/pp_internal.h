@@ -52,7 +52,8 @@ struct TileStep {
     int32_t pad;
 };
 static_assert(sizeof(TileStep) == 32, "read as two 16-byte words");
-extern int g_tile_cluster;   // batched fp16 B = 64 layers: 0 one block-row per CTA, 2 the clustered kernel, 1 whichever fits the layer
+extern int g_tile_cluster;   // batched fp16 B = 64 layers: 0 one block-row per CTA, 2 the clustered kernel, 3 the persistent kernel, 1 automatic
+extern int g_tile_persist_auto;   // 1: the automatic choice is the persistent kernel whenever the layer has a plan for it
 constexpr int kStreamWarps = 16;          // warps per CTA
 constexpr int kStreamMaxStrips = 48;      // strips one CTA may list
 constexpr int kStreamMaxBatch = 8;

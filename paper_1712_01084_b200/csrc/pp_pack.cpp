@@ -15,6 +15,7 @@ int g_tile_min_batch = 9;
 int g_prepass = 1;
 int g_lstm_persist = 1;
 int g_tile_cluster = 1;
+int g_tile_persist_auto = 0;
 int g_link_identity = 1;
 int g_chain_fused = 0;      // measured: one launch per layer (programmatic dependent launch) is the faster way through a chain
 extern int g_stream_wait_polls;   // poll limit of the bounded device-side waits (pp_stream.cu)
@@ -224,7 +225,78 @@ void build_stream_plan(pp_packed* p) {
 
 }  // namespace
 
+namespace pp {
+// Plan of the persistent tile kernel for n_ctas CTAs: the step sequence of all groups cut into one contiguous
+// range per CTA (equal shares of the cost: an X block counts as two tiles), and the units those ranges make with
+// the groups, in (group, step) order.  Every group is covered: one without tiles gets an empty unit, so that its
+// rows still receive act(bias).  A CTA's units are consecutive: cta_unit[c] .. cta_unit[c + 1].
+void build_tile_units(const pp_packed* pk, int n_ctas, std::vector<TileUnit>& units, std::vector<int32_t>& cta_unit) {
+    constexpr int R = kTileRows;
+    const int groups = (pk->Mb + R - 1) / R;
+    const std::vector<TileStep>& steps = pk->tile_steps;
+    const int S = (int)steps.size();
+    const int G = std::max(1, n_ctas);
+    std::vector<int64_t> cum((size_t)S + 1, 0);
+    for (int i = 0; i < S; ++i) cum[(size_t)i + 1] = cum[(size_t)i] + 2 + steps[(size_t)i].ntiles;
+    std::vector<int> cta_step((size_t)G + 1, S);
+    cta_step[0] = 0;
+    for (int c = 1; c < G; ++c) {
+        const int64_t want = cum[(size_t)S] * c / G;
+        cta_step[(size_t)c] = (int)(std::lower_bound(cum.begin(), cum.end(), want) - cum.begin());
+        cta_step[(size_t)c] = std::max(cta_step[(size_t)c], cta_step[(size_t)c - 1]);
+    }
+    auto owner_of = [&](int step) {                   // the CTA whose range holds this step position
+        const int c = (int)(std::upper_bound(cta_step.begin(), cta_step.begin() + G, step) - cta_step.begin()) - 1;
+        return std::min(std::max(c, 0), G - 1);
+    };
+    units.clear();
+    std::vector<int> unit_cta;
+    for (int g = 0; g < groups; ++g) {
+        const int gs = pk->tile_parts[(size_t)g * (R + 1)], ge = pk->tile_parts[(size_t)g * (R + 1) + R];
+        const size_t first = units.size();
+        if (gs == ge) {
+            units.push_back(TileUnit{gs, gs, g, 0, 1, (int32_t)first, {0, 0}});
+            unit_cta.push_back(owner_of(std::min(gs, std::max(S - 1, 0))));
+        } else {
+            for (int s0 = gs; s0 < ge;) {
+                const int c = owner_of(s0);
+                const int s1 = std::min(ge, std::max(cta_step[(size_t)c + 1], s0 + 1));
+                units.push_back(TileUnit{s0, s1, g, (int32_t)(units.size() - first), 0, (int32_t)first, {0, 0}});
+                unit_cta.push_back(c);
+                s0 = s1;
+            }
+        }
+        for (size_t u = first; u < units.size(); ++u) units[u].n_parts = (int32_t)(units.size() - first);
+    }
+    cta_unit.assign((size_t)G + 1, (int32_t)units.size());
+    size_t u = 0;
+    for (int c = 0; c < G; ++c) {
+        cta_unit[(size_t)c] = (int32_t)u;
+        while (u < units.size() && unit_cta[u] <= c) ++u;      // owners never decrease along the sequence
+    }
+}
+}  // namespace pp
+
 extern "C" {
+
+pp_status_t pp_pack_tile_units(const pp_packed_t* p, int n_ctas, int32_t* units_out, int64_t capacity_units,
+                               int64_t* n_units_out, int32_t* cta_unit_out) {
+    if (!p || n_ctas < 1 || !n_units_out) return PP_ERR_INVALID_ARG;
+    if (p->wdtype != PP_F16 || p->B != 64) return PP_ERR_UNSUPPORTED;
+    try {
+        std::vector<pp::TileUnit> units;
+        std::vector<int32_t> cta_unit;
+        pp::build_tile_units(p, n_ctas, units, cta_unit);
+        *n_units_out = (int64_t)units.size();
+        if (!units_out && !cta_unit_out) return PP_OK;              // count only
+        if (!units_out || !cta_unit_out || capacity_units < (int64_t)units.size()) return PP_ERR_INVALID_ARG;
+        std::memcpy(units_out, units.data(), units.size() * sizeof(pp::TileUnit));
+        std::memcpy(cta_unit_out, cta_unit.data(), cta_unit.size() * 4);
+    } catch (const std::bad_alloc&) {
+        return PP_ERR_ALLOC;
+    }
+    return PP_OK;
+}
 
 const char* pp_status_string(pp_status_t s) {
     switch (s) {
@@ -333,7 +405,7 @@ pp_status_t pp_set_tuning(int key, int value) {
     if (key == 9 && value >= 0) { pp::g_tile_min_batch = value; return PP_OK; }
     if (key == 10 && value >= 0 && value <= 2) { pp::g_prepass = value; return PP_OK; }
     if (key == 11 && (value == 0 || value == 1)) { pp::g_lstm_persist = value; return PP_OK; }
-    if (key == 12 && value >= 0 && value <= 2) { pp::g_tile_cluster = value; return PP_OK; }
+    if (key == 12 && value >= 0 && value <= 3) { pp::g_tile_cluster = value; return PP_OK; }
     if (key == 13 && (value == 0 || value == 1)) { pp::g_link_identity = value; return PP_OK; }
     if (key == 14 && (value == 0 || value == 1)) { pp::g_chain_fused = value; return PP_OK; }
     if (key == 15 && value >= 0) { pp::g_stream_wait_polls = value; return PP_OK; }

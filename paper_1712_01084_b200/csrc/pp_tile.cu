@@ -561,6 +561,340 @@ tile_cluster_f16_kernel(const TileArgs a) {
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Persistent variant: every SM streams an equal share of the layer.
+// The steps of all groups (a step = one tile-column of a group of kTileRows block-rows: one X block and the
+// up to kTileRows tiles the group has there) form one sequence, which the host cuts into one contiguous range
+// per CTA, balanced by bytes; one CTA per SM.  The part of a group that falls into one CTA's range is a unit:
+//   * the producers and the MMA issuer walk the CTA's steps without a break; consecutive units alternate between
+//     two sets of kTileRows accumulators in tensor memory (512 columns in all), so that the epilogue warps work
+//     on one unit while the next one is being multiplied;
+//   * a unit that covers its whole group stores the group's rows itself (bias, activation, row index array);
+//   * otherwise every unit of the group writes its partial sums to its own slots in global memory ([chunk]
+//     [quad of output rows][batch row][4 floats]: a warp's 16-byte stores and loads are contiguous) and counts
+//     itself in at the group's arrival counter; the group's 8 chunks of 32 output rows are dealt out to the
+//     units, and each unit, once all have arrived (bounded wait), adds the partial sums of its chunks in unit
+//     order and stores those rows.  No atomics on data, the same bits on every run; the last unit to finish
+//     reading puts the group's two counters back to zero.
+constexpr int kPStages = 4;
+constexpr int kPStageBytes = kXBytes + kTileRows * kWBytes;    // 48 KiB: one X block + up to 4 tiles
+constexpr int kPTmemCols = 2 * 64 * kTileRows;                 // two accumulator sets
+constexpr int kPThreads = 32 * (kProducers + 1 + 4);
+constexpr int kPChunks = 2 * kTileRows;                        // chunks of 32 output rows per group
+constexpr int kGroupPolls = 1 << 22;
+
+struct PersistSmem {
+    uint64_t full[kPStages];
+    uint64_t empty[kPStages];
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+    int group_ready;          // written by one epilogue thread after its bounded wait for the group's units
+    uint32_t acc_mask[2];     // per accumulator set: block-rows that received at least one tile
+    float xpose[4][32 * 33];  // one transposition tile per epilogue warp
+    int4 steps[kStepCap][2];  // this CTA's first kStepCap step records
+};
+
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(addr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ TileUnit load_unit(const TileUnit* p) {
+    const int4 lo = __ldg(reinterpret_cast<const int4*>(p)), hi = __ldg(reinterpret_cast<const int4*>(p) + 1);
+    TileUnit u;
+    u.step_begin = lo.x; u.step_end = lo.y; u.group = lo.z; u.part = lo.w; u.n_parts = hi.x; u.first_unit = hi.y;
+    u.pad[0] = u.pad[1] = 0;
+    return u;
+}
+
+#ifdef PP_TRACE
+__device__ __forceinline__ void tile_stamp(const TileArgs& a, int slot) {
+    if (a.trace) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        a.trace[(size_t)blockIdx.x * 8 + slot] = t;
+    }
+}
+#else
+__device__ __forceinline__ void tile_stamp(const TileArgs&, int) {}
+#endif
+
+// Which unit of a group finishes chunk q of the group's rows.
+__device__ __forceinline__ int chunk_owner(int q, int n_parts) { return n_parts <= kPChunks ? q % n_parts : q; }
+
+__global__ void __launch_bounds__(kPThreads, 1)
+tile_persist_f16_kernel(const TileArgs a) {
+    static_assert(kTileRows == 4, "step records carry four tile slots");
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* stages = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    PersistSmem* sm = reinterpret_cast<PersistSmem*>(stages + kPStages * kPStageBytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int u0 = __ldg(a.cta_unit + blockIdx.x), u1 = __ldg(a.cta_unit + blockIdx.x + 1);
+    int cs = 0, ce = 0;                       // this CTA's steps: from its first unit's first step to its last unit's last
+    if (u0 < u1) {
+        cs = __ldg(&a.units[u0].step_begin);
+        ce = __ldg(&a.units[u1 - 1].step_end);
+    }
+    // This CTA's step records go to shared memory once: read from global memory inside the loops they cost the
+    // producers and the MMA issuer one L2 round trip per step.
+    for (int i = threadIdx.x; i < 2 * (ce - cs) && i < 2 * kStepCap; i += kPThreads)
+        sm->steps[i >> 1][i & 1] = __ldg(reinterpret_cast<const int4*>(a.steps + cs) + i);
+    auto step_at = [&](int i) {
+        return i < kStepCap ? unpack_step(sm->steps[i][0], sm->steps[i][1]) : load_step(a.steps + cs + i);
+    };
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kPStages; ++s) { mbar_init(&sm->full[s], 1); mbar_init(&sm->empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&sm->acc_full[s], 2); mbar_init(&sm->acc_empty[s], 4); }
+        sm->abort_flag = 0;
+        sm->acc_mask[0] = sm->acc_mask[1] = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kProducers) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     :: "r"(smem_u32(&sm->tmem_base)), "r"(kPTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = sm->tmem_base;
+    volatile int* abort_flag = &sm->abort_flag;
+    if (threadIdx.x == 0) tile_stamp(a, 0);
+
+    if (warp < kProducers) {
+        // ---------------- producers: warp w (one lane) feeds steps cs + w, cs + w + kProducers, ... into stage w
+        if (lane == 0) {
+            const int s = warp;
+            int last = -1;
+            const uint32_t xbytes = (uint32_t)((a.batch + 7) / 8) * 1024u;   // live 8-row groups of the X block only
+            for (int t = warp; t < ce - cs; t += kProducers) {
+                if (t >= kPStages && !mbar_wait(&sm->empty[s], ((t / kPStages) & 1) ^ 1, abort_flag, a.polls)) break;
+                const TileStep st = step_at(t);
+                unsigned char* dst = stages + s * kPStageBytes;
+                mbar_expect_tx(&sm->full[s], xbytes + (uint32_t)(st.ntiles * kWBytes));
+                bulk_load(dst + kXBytes, a.tiles_sw + (size_t)st.pos * kWBytes, (uint32_t)(st.ntiles * kWBytes), &sm->full[s]);
+                // the permuted input comes from the gather kernel launched just before: everything up to here
+                // (set-up, the first weight copies) may overlap its tail
+                if (t == warp) asm volatile("griddepcontrol.wait;" ::: "memory");
+                bulk_load(dst, a.x_sw + (size_t)st.col * kXBytes, xbytes, &sm->full[s]);
+                last = t;
+            }
+            if (*abort_flag && last >= 0) {
+                // let the copy still in flight land before shared memory goes away
+                for (int i = 0; i < kPollLimit && !mbar_try_wait(&sm->full[s], (last / kPStages) & 1); ++i) {}
+            }
+        }
+    } else if (warp == kProducers) {
+        // ---------------- MMA issuer (one lane): unit after unit, alternating between the two accumulator sets
+        if (lane == 0) {
+            bool ok = true;
+            int t = 0;                                   // steps issued so far, over all units
+            for (int u = u0; u < u1; ++u) {
+                const int set = (u - u0) & 1, use = (u - u0) >> 1;
+                const int n = __ldg(&a.units[u].step_end) - __ldg(&a.units[u].step_begin);
+                uint32_t mask = 0u;
+                // the epilogue must have drained this set's previous unit
+                if (ok && use > 0) ok = mbar_wait(&sm->acc_empty[set], (use - 1) & 1, abort_flag, 0);
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                for (int i = 0; i < n && ok; ++i, ++t) {
+                    const int s = t % kPStages;
+                    const TileStep st = step_at(t);
+                    ok = mbar_wait(&sm->full[s], (t / kPStages) & 1, abort_flag, a.polls);
+                    if (!ok) break;
+                    if (t == 0) tile_stamp(a, 1);
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t xa = smem_u32(stages + s * kPStageBytes);
+                    int slot = 0;
+                    for (int j = 0; j < kTileRows;) {
+                        if (st.tile[j] < 0) { ++j; continue; }
+                        const bool started = ((mask >> j) & 1u) != 0u;
+                        int nn = 1;
+                        while (j + nn < kTileRows && st.tile[j + nn] >= 0 && (((mask >> (j + nn)) & 1u) != 0u) == started) ++nn;
+                        const uint32_t wa = xa + kXBytes + slot * kWBytes;
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            umma_f16_n(tmem + (uint32_t)(set * 64 * kTileRows + j * 64), smem_desc_sw128(xa + kk * 32),
+                                       smem_desc_sw128(wa + kk * 32), nn, started || kk > 0);
+                        mask |= ((1u << nn) - 1u) << j;
+                        slot += nn;
+                        j += nn;
+                    }
+                    umma_commit(&sm->empty[s]);          // frees the stage once these MMAs have read it
+                }
+                sm->acc_mask[set] = ok ? mask : 0u;
+                if (mask != 0u) umma_commit(&sm->acc_full[set]);   // whatever was issued must finish, also when giving up
+                else mbar_arrive(&sm->acc_full[set]);
+                mbar_arrive(&sm->acc_full[set]);                   // releases acc_mask to the epilogue warps
+            }
+            tile_stamp(a, 2);
+        }
+    } else {
+        // ---------------- epilogue warps: warp (w % 4) owns tensor-memory lanes 32 (w % 4) .., thread = batch row
+        const int q = warp & 3, b = q * 32 + lane;
+        const bool live_warp = q * 32 < a.batch;          // a warp whose 32 batch rows all lie past the batch only keeps the barriers
+        float* xpose = sm->xpose[q];
+        bool ok = true;
+        // rows [c0, c0 + 32) of a block-row: bias, activation, store.  The 32 x 32 block is transposed through
+        // shared memory so that the lanes of a store run over output rows (32 scattered words of ONE row of y).
+        auto store_chunk = [&](const uint32_t (&r)[32], float bias, int dst) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) xpose[lane * 33 + j] = __uint_as_float(r[j]);
+            __syncwarp();
+#pragma unroll 8
+            for (int rr = 0; rr < 32; ++rr) {
+                const int bb = q * 32 + rr;
+                float v = xpose[rr * 33 + lane] + bias;
+                if (a.act == PP_ACT_RELU) v = fmaxf(v, 0.0f);
+                if (dst >= 0 && bb < a.batch) a.y[(size_t)bb * a.ldy + dst] = v;
+            }
+            __syncwarp();
+        };
+        // bias and destination row of the chunks of unit `un` that this unit stores (lane = row of the chunk)
+        auto chunk_rows = [&](const TileUnit& un, float (&cbias)[kPChunks], int (&cdst)[kPChunks]) {
+#pragma unroll
+            for (int c = 0; c < kPChunks; ++c) {
+                const int br = un.group * kTileRows + (c >> 1), row = br * 64 + (c & 1) * 32 + lane;
+                const bool mine = (un.n_parts == 1 || chunk_owner(c, un.n_parts) == un.part) && br < a.Mb;
+                cbias[c] = mine ? __ldg(a.bias_piv + row) : 0.0f;
+                cdst[c] = !mine ? -1 : (a.pivoted ? row : __ldg(a.scatter_idx + row));
+            }
+        };
+        // First pass, unit after unit as the accumulators complete: a unit that owns its whole group stores the
+        // rows; any other writes its partial sums to its slots and counts itself in at the group's counter.
+        // Nothing here waits for another CTA, so no CTA's publication can be held up by a neighbour's.
+        for (int u = u0; u < u1; ++u) {
+            const int set = (u - u0) & 1, use = (u - u0) >> 1;
+            const TileUnit un = load_unit(a.units + u);
+            float cbias[kPChunks];
+            int cdst[kPChunks];
+            if (un.n_parts == 1) chunk_rows(un, cbias, cdst);        // requested while the unit is still being multiplied
+            ok = __all_sync(0xffffffffu, ok && mbar_wait(&sm->acc_full[set], use & 1, abort_flag, 0) && !*abort_flag);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t mask = sm->acc_mask[set];
+            const uint32_t tbase = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(set * 64 * kTileRows);
+            if (ok && live_warp) {
+                float* mine = a.unit_partials + (size_t)u * (kPChunks * kTileBatch * 32);
+#pragma unroll
+                for (int c = 0; c < kPChunks; ++c) {
+                    uint32_t r[32];
+                    if ((mask >> (c >> 1)) & 1u) {              // warp-uniform: the tensor-memory load is a warp-wide instruction
+                        tmem_ld32(tbase + (uint32_t)(c * 32), r);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = 0u;
+                    }
+                    if (un.n_parts == 1) {
+                        store_chunk(r, cbias[c], cdst[c]);
+                    } else if (b < a.batch) {
+                        // [chunk][row quad j][batch row][4]: the 32 lanes of a store write one contiguous 512-byte run
+                        uint4* dst = reinterpret_cast<uint4*>(mine) + (size_t)c * (8 * kTileBatch) + b;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) dst[(size_t)j * kTileBatch] = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            if (lane == 0) mbar_arrive(&sm->acc_empty[set]);         // the accumulator set may be reused
+            if (un.n_parts > 1) {
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (ok && warp == kProducers + 1 && lane == 0) atomicAdd(a.group_sync + 2 * un.group, 1);
+            }
+        }
+        if (warp == kProducers + 1 && lane == 0) tile_stamp(a, 3);
+        // Second pass: for every split group this CTA has a unit of, wait (bounded) until all units of the group
+        // have arrived, add the partial sums of this unit's chunks in unit order and store those rows; the last
+        // unit to finish reading puts the group's counters back to zero.
+        for (int u = u0; u < u1; ++u) {
+            const TileUnit un = load_unit(a.units + u);
+            if (un.n_parts == 1) continue;
+            float cbias[kPChunks];
+            int cdst[kPChunks];
+            chunk_rows(un, cbias, cdst);
+            int* gsync = a.group_sync + 2 * un.group;
+            if (warp == kProducers + 1 && lane == 0) {
+                int ready = 0;
+                if (ok) {
+                    const int limit = a.polls > 0 ? a.polls : kGroupPolls;
+                    for (int i = 0; i < limit && !ready; ++i) {
+                        int seen;
+                        asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(gsync) : "memory");
+                        ready = seen >= un.n_parts;
+                        if (!ready && (i & 63) == 63 && *reinterpret_cast<volatile int*>(a.status)) break;
+                    }
+                    if (!ready) { *abort_flag = 1; *a.status = 1; }
+                }
+                sm->group_ready = ready;
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            ok = ok && sm->group_ready != 0;
+            if (ok && live_warp) {
+#pragma unroll
+                for (int c = 0; c < kPChunks; ++c) {
+                    if (chunk_owner(c, un.n_parts) != un.part) continue;
+                    uint32_t r[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = 0u;
+                    if (b < a.batch) {
+                        // the partial sums were written by other SMs: read them past the L1 (ld.global.cg); the loads of
+                        // two units are in flight together, the additions stay in unit order
+                        const uint4* base = reinterpret_cast<const uint4*>(a.unit_partials) +
+                                            ((size_t)un.first_unit * kPChunks + c) * (8 * kTileBatch) + b;
+                        const size_t unit_stride = (size_t)kPChunks * 8 * kTileBatch;
+                        for (int p = 0; p < un.n_parts; p += 2) {
+                            const bool two = p + 1 < un.n_parts;
+                            uint4 v0[8], v1[8];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) v0[j] = __ldcg(base + (size_t)p * unit_stride + (size_t)j * kTileBatch);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j)
+                                v1[j] = two ? __ldcg(base + (size_t)(p + 1) * unit_stride + (size_t)j * kTileBatch) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                r[4 * j] = __float_as_uint(__uint_as_float(r[4 * j]) + __uint_as_float(v0[j].x));
+                                r[4 * j + 1] = __float_as_uint(__uint_as_float(r[4 * j + 1]) + __uint_as_float(v0[j].y));
+                                r[4 * j + 2] = __float_as_uint(__uint_as_float(r[4 * j + 2]) + __uint_as_float(v0[j].z));
+                                r[4 * j + 3] = __float_as_uint(__uint_as_float(r[4 * j + 3]) + __uint_as_float(v0[j].w));
+                            }
+                            if (two) {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) {
+                                    r[4 * j] = __float_as_uint(__uint_as_float(r[4 * j]) + __uint_as_float(v1[j].x));
+                                    r[4 * j + 1] = __float_as_uint(__uint_as_float(r[4 * j + 1]) + __uint_as_float(v1[j].y));
+                                    r[4 * j + 2] = __float_as_uint(__uint_as_float(r[4 * j + 2]) + __uint_as_float(v1[j].z));
+                                    r[4 * j + 3] = __float_as_uint(__uint_as_float(r[4 * j + 3]) + __uint_as_float(v1[j].w));
+                                }
+                            }
+                        }
+                    }
+                    store_chunk(r, cbias[c], cdst[c]);
+                }
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");           // every warp has read; group_ready may be rewritten
+            if (ok && warp == kProducers + 1 && lane == 0) {
+                if (atomicAdd(gsync + 1, 1) == un.n_parts - 1) { gsync[0] = 0; gsync[1] = 0; }
+            }
+        }
+        if (warp == kProducers + 1 && lane == 0) tile_stamp(a, 4);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0 && sm->abort_flag) *a.status = 1;
+    if (warp == kProducers) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kPTmemCols) : "memory");
+    }
+}
+
 // Byte offset of element (row r, column c) inside a 128-byte-swizzled block of 128-byte rows:
 // the 16-byte chunk index is XOR-ed with the row index modulo 8.
 __host__ __device__ __forceinline__ uint32_t sw128_offset(int r, int c) {
@@ -608,6 +942,10 @@ __global__ void gather_x_kernel(const __half* __restrict__ x, int ldx, int n, co
 
 }  // namespace
 
+#ifdef PP_TRACE
+unsigned long long* g_tile_trace = nullptr;
+#endif
+
 void swizzle_tile_64x64(const void* row_major, void* out) {
     const unsigned char* src = static_cast<const unsigned char*>(row_major);
     unsigned char* dst = static_cast<unsigned char*>(out);
@@ -618,18 +956,21 @@ void swizzle_tile_64x64(const void* row_major, void* out) {
 
 // Launch with programmatic stream serialization: the kernel may start while the gather kernel before it
 // still runs; its producers wait for that kernel (griddepcontrol.wait) before they touch the permuted input.
+// cooperative: the CTAs wait on one another (units of a group), so all of them must be resident at once.
 static cudaError_t launch_after_gather(void (*kernel)(const TileArgs), int grid, int threads, size_t smem, const TileArgs& a,
-                                       cudaStream_t stream) {
+                                       cudaStream_t stream, bool cooperative = false) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)threads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeCooperative;
+    attr[1].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = cooperative ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, kernel, a);
 }
 
@@ -649,9 +990,14 @@ cudaError_t launch_one_row(const TileArgs& a, int Mb, cudaStream_t stream) {
 }
 
 cudaError_t launch_tile(const TileArgs& a_in, const void* x, int ldx, int n, const int32_t* gather_idx, int n_pad, int Mb,
-                        bool use_cluster, cudaStream_t stream) {
+                        int kernel, cudaStream_t stream) {
+    const bool use_cluster = kernel == 2;
     TileArgs a = a_in;
     a.polls = g_stream_wait_polls;
+    a.trace = nullptr;
+#ifdef PP_TRACE
+    a.trace = g_tile_trace;
+#endif
     if (a.batch < 1 || a.batch > kTileBatch) return cudaErrorInvalidValue;
     if ((size_t)n * 2 > 48 * 1024) return cudaErrorInvalidValue;
     // rows past the batch keep whatever an earlier call left there: every row of the product is independent
@@ -660,6 +1006,19 @@ cudaError_t launch_tile(const TileArgs& a_in, const void* x, int ldx, int n, con
                                                               const_cast<unsigned char*>(a.x_sw), a.batch);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
+    if (kernel == 3 && a.units && a.cta_unit && a.persist_ctas > 0 && a.unit_partials && a.group_sync) {
+        static PerDeviceOnce configured_p;
+        const size_t smem_p = (size_t)kPStages * kPStageBytes + sizeof(PersistSmem) + 1024;
+        int dev = -1;
+        e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        if (!configured_p.is_done(dev)) {
+            e = cudaFuncSetAttribute(tile_persist_f16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_p);
+            if (e != cudaSuccess) return e;
+            configured_p.mark(dev);
+        }
+        return launch_after_gather(tile_persist_f16_kernel, a.persist_ctas, kPThreads, smem_p, a, stream, true);
+    }
     if (use_cluster && a.steps && a.parts) {
         static PerDeviceOnce configured_c;
         const size_t smem_c = (size_t)kCStages * kCStageBytes + sizeof(ClusterSmem) + 1024;
@@ -680,3 +1039,9 @@ cudaError_t launch_tile(const TileArgs& a_in, const void* x, int ldx, int n, con
 }
 
 }  // namespace pp
+
+#ifdef PP_TRACE
+// Diagnostic builds only: launches of the persistent tile kernel write their phase stamps to `device_buffer`
+// (148 x 8 unsigned 64-bit words, overwritten by every launch).
+extern "C" void pp_trace_set_tile_buffer(void* device_buffer) { pp::g_tile_trace = static_cast<unsigned long long*>(device_buffer); }
+#endif

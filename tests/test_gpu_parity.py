@@ -378,9 +378,10 @@ def test_input_permutation_prepass(pb, dtype, prepass):
 
 
 # ------------------------------------------------------------------ tensor-core tile path (batch >= 64)
-@pytest.fixture(params=[2, 0, 1], ids=["clustered", "row-per-cta", "auto"])
+@pytest.fixture(params=[2, 0, 3, 1], ids=["clustered", "row-per-cta", "persistent", "auto"])
 def tile_kernel(pb, request):
-    """Both tensor-core kernels: a cluster of 4 CTAs per 4 block-rows, or one CTA per block-row."""
+    """The tensor-core kernels: a cluster of 4 CTAs per 4 block-rows, one CTA per block-row, or one persistent CTA
+    per SM over an equal share of the layer's steps."""
     pb.pp_set_tuning(12, request.param)
     yield request.param
     pb.pp_set_tuning(12, 1)
@@ -428,10 +429,13 @@ def test_tile_path_both_kernels_same_bits_and_repeatable(pb):
         y1b = pb.pp_forward(L, _dev(x), 0).cpu().numpy()
         pb.pp_set_tuning(12, 0)
         y0 = pb.pp_forward(L, _dev(x), 0).cpu().numpy()
+        pb.pp_set_tuning(12, 3)
+        y3 = pb.pp_forward(L, _dev(x), 0).cpu().numpy()
+        y3b = pb.pp_forward(L, _dev(x), 0).cpu().numpy()
     finally:
         pb.pp_set_tuning(12, 1)
     assert L.status() == 0
-    assert np.array_equal(y1, y1b) and np.array_equal(y1, y0)
+    assert np.array_equal(y1, y1b) and np.array_equal(y1, y0) and np.array_equal(y1, y3) and np.array_equal(y3, y3b)
     y_ref, _, _ = po.layer_forward(lay, x.astype(np.float64), act=0, threads=8)
     assert np.array_equal(y1.astype(np.float64), y_ref)
     L.close()
@@ -464,7 +468,7 @@ def test_layer_created_without_tile_copy(pb):
     for layer in (L, C):
         _check(pb.pp_forward(layer, _dev(x), 1).cpu().numpy(), y_ref, a, np.float16, "no tile copy")
     full = pb.Layer.from_synth(lay)
-    assert full.launch_info(40)["kernel"] in ("tile", "tile_cluster")
+    assert full.launch_info(40)["kernel"] in ("tile", "tile_cluster", "tile_persist")
     L.close(); C.close(); full.close()
 
 

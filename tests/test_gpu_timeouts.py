@@ -54,7 +54,7 @@ def test_persistent_kernel_x_wait_runs_out(pb, one_poll):
     L.close()
 
 
-@pytest.mark.parametrize("tile_kernel", [0, 2], ids=["one_block_row", "clustered"])
+@pytest.mark.parametrize("tile_kernel", [0, 2, 3], ids=["one_block_row", "clustered", "persistent"])
 def test_tile_kernels_stage_wait_runs_out(pb, one_poll, tile_kernel):
     wl = synth.config5(k=128, batch=40, scale=0.125)      # 1024 x 1024, every tile kept
     lay = wl.layers[0]
@@ -63,7 +63,7 @@ def test_tile_kernels_stage_wait_runs_out(pb, one_poll, tile_kernel):
     y_ref, _, a = po.layer_forward(lay, wl.x.astype(np.float64))
     pb.pp_set_tuning(12, tile_kernel)
     try:
-        assert L.launch_info(40)["kernel"] in ("tile", "tile_cluster")
+        assert L.launch_info(40)["kernel"] in ("tile", "tile_cluster", "tile_persist")
         one_poll(1)
         pb.pp_forward(L, x, lay.act)
         assert L.status() == PP_ERR_TIMEOUT

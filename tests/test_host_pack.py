@@ -526,6 +526,47 @@ def test_blocks_error_codes():
     assert status([[-1, 0, 2, 2]], v[:4]) == 3
 
 
+@pytest.mark.parametrize("n_ctas", [1, 7, 148, 500])
+@pytest.mark.parametrize("density,empty_rows", [(1.0, ()), (0.4, ()), (0.1, (0, 1, 2, 3, 9)), (0.02, ())])
+def test_persistent_tile_plan_covers_every_step_once(n_ctas, density, empty_rows):
+    """Plan of the persistent tensor-core kernel: every step of every group falls into exactly one unit, a group
+    without tiles still has a (step-less) unit, a group's units are numbered in order and know their count and
+    first index, a CTA's units are consecutive, and the CTAs' shares of the cost differ by at most one step."""
+    rng = np.random.default_rng(17)
+    M, N, B = 13 * 64 - 5, 11 * 64, 64
+    Mb, Nb = -(-M // B), N // B
+    grid = [(br, bc) for br in range(Mb) for bc in range(Nb) if br not in empty_rows]
+    sel = rng.permutation(len(grid))[:max(1, int(density * len(grid)))]
+    tl = np.array([grid[i] for i in sel], dtype=np.int32)
+    tv = rng.standard_normal((tl.shape[0], B, B)).astype(np.float16)
+    pk = pb.Packed(M, N, B, rng.permutation(Mb * B).astype(np.int32), rng.permutation(N).astype(np.int32), tl, tv)
+    steps, parts = pk.get("tile_steps"), pk.get("tile_parts")
+    units, cta_unit = pk.tile_units(n_ctas)
+    groups = -(-Mb // 4)
+    assert cta_unit[0] == 0 and cta_unit[-1] == len(units) and np.all(np.diff(cta_unit) >= 0)
+    covered = np.zeros(len(steps), dtype=np.int32)
+    seen_groups = []
+    for u, (s0, s1, g, part, n_parts, first, _, _) in enumerate(units):
+        assert parts[g, 0] <= s0 <= s1 <= parts[g, 4]
+        covered[s0:s1] += 1
+        assert first <= u < first + n_parts and part == u - first and units[first, 2] == g
+        assert (s0 == s1) == (parts[g, 0] == parts[g, 4])           # step-less units only for groups without tiles
+        seen_groups.append(g)
+    assert np.all(covered == 1)
+    assert sorted(set(seen_groups)) == list(range(groups)) and seen_groups == sorted(seen_groups)
+    # a CTA's steps are contiguous, and the shares are balanced to within one step's cost
+    cost = 2 + steps[:, 5] if len(steps) else np.zeros(0)
+    share = []
+    for c in range(n_ctas):
+        mine = units[cta_unit[c]:cta_unit[c + 1]]
+        if len(mine):
+            assert np.all(mine[1:, 0] == mine[:-1, 1])
+        share.append(sum(int(cost[s0:s1].sum()) for s0, s1 in mine[:, :2]))
+    assert sum(share) == int(cost.sum())
+    if len(steps):
+        assert max(share) - min(share) <= 2 * int(cost.max())
+
+
 # ------------------------------------------------ physical layouts of the layout study (Section 4.1.1)
 @pytest.mark.parametrize("size,nb", [(64, 4), (96, 8), (40, 5)])
 def test_layout_study_layouts(size, nb):
