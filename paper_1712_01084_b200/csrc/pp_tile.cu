@@ -146,6 +146,7 @@ tile_f16_kernel(const TileArgs a) {
     TileSmem<STAGES>* sm = reinterpret_cast<TileSmem<STAGES>*>(stages + kStages * kStageBytes + (kXBytes - XB));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int br = blockIdx.x;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next call's gather kernel may fetch its index entries meanwhile
     const int t0 = __ldg(a.row_ptr + br), k = __ldg(a.row_ptr + br + 1) - t0;
 
     // The block-row's tile list goes to shared memory once, by the whole CTA, while tensor memory is set
@@ -372,6 +373,7 @@ tile_cluster_f16_kernel(const TileArgs a) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint32_t rank;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next call's gather kernel may fetch its index entries meanwhile
     const int grp = blockIdx.x / kTileRows, n_groups = gridDim.x / kTileRows;
     const int p0 = __ldg(a.parts + grp * (kTileRows + 1) + rank);
     const int n_steps = __ldg(a.parts + grp * (kTileRows + 1) + rank + 1) - p0;
@@ -639,6 +641,7 @@ tile_persist_f16_kernel(const TileArgs a) {
     unsigned char* stages = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     PersistSmem* sm = reinterpret_cast<PersistSmem*>(stages + kPStages * kPStageBytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next call's gather kernel may fetch its index entries meanwhile
     const int u0 = __ldg(a.cta_unit + blockIdx.x), u1 = __ldg(a.cta_unit + blockIdx.x + 1);
     int cs = 0, ce = 0;                       // this CTA's steps: from its first unit's first step to its last unit's last
     if (u0 < u1) {
@@ -916,6 +919,10 @@ __global__ void gather_x_kernel(const __half* __restrict__ x, int ldx, int n, co
     int i = threadIdx.x;
     int4 ia = make_int4(-1, -1, -1, -1), ib = ia;
     if (i < n_chunks) { ia = __ldg(idx4 + 2 * i); ib = __ldg(idx4 + 2 * i + 1); }
+    // Launched with programmatic stream serialization behind whatever precedes it in the stream (typically the
+    // previous call's tile kernel, which may still read the permuted-input blocks this kernel is about to
+    // overwrite, or the producer of x): the index entries above are the layer's own, everything below waits.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     {
         // 16-byte copies where the row allows it (base and pitch 16-byte aligned), element copies otherwise
         const __half* src = x + (size_t)b * ldx;
@@ -1002,9 +1009,21 @@ cudaError_t launch_tile(const TileArgs& a_in, const void* x, int ldx, int n, con
     if ((size_t)n * 2 > 48 * 1024) return cudaErrorInvalidValue;
     // rows past the batch keep whatever an earlier call left there: every row of the product is independent
     // and the epilogue drops those rows
-    gather_x_kernel<<<a.batch, 1024, ((size_t)n * 2 + 15) / 16 * 16, stream>>>(static_cast<const __half*>(x), ldx, n, gather_idx, n_pad,
-                                                              const_cast<unsigned char*>(a.x_sw), a.batch);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e;
+    {
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)a.batch);
+        cfg.blockDim = dim3(1024);
+        cfg.dynamicSmemBytes = ((size_t)n * 2 + 15) / 16 * 16;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = g_stream_pdl ? 1 : 0;
+        e = cudaLaunchKernelEx(&cfg, gather_x_kernel, static_cast<const __half*>(x), ldx, n, gather_idx, n_pad,
+                               const_cast<unsigned char*>(a.x_sw), a.batch);
+    }
     if (e != cudaSuccess) return e;
     if (kernel == 3 && a.units && a.cta_unit && a.persist_ctas > 0 && a.unit_partials && a.group_sync) {
         static PerDeviceOnce configured_p;
