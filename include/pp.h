@@ -454,7 +454,8 @@ pp_status_t pp_selftest_host(void);
  *         block-rows per cluster of 4 CTAs share every X block); 3 the persistent kernel (one CTA per SM over an
  *         equal share of the layer's steps, two accumulator sets in tensor memory, groups split between CTAs
  *         summed through partial-sum slots in global memory in a fixed order; measured slower than the other
- *         two, kept as an option); 1 (default) the clustered kernel when the groups' tile-columns carry at
+ *         two, kept as an option: the key must be 3 when the layer is created, because the plan and its
+ *         slots, 128 KiB per unit, are only allocated then; other layers fall back to one block-row per CTA); 1 (default) the clustered kernel when the groups' tile-columns carry at
  *         least 3.5 of 4 possible tiles on average, else one block-row per CTA
  * key 13: 1 (default) chain links whose folded map is the identity store pivoted rows without an index array,
  *         0 sends them through the map like any other link

@@ -226,6 +226,7 @@ bool alloc_layer(pp_layer* L, const LayerLayout& lo) {
 // blocks.  false: allocation failed.
 bool persist_setup(pp_layer* L) {
     const pp_packed* pk = L->pk;
+    if (pp::g_tile_cluster != 3) return true;       // opt-in: the partial-sum slots are 128 KiB per unit (tens of MiB for a large layer)
     int dev = 0, sms = 0, coop = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) {

@@ -394,6 +394,8 @@ def test_tile_path_small_layer(pb, batch, tile_kernel):
     lay = _rand_layer(900 + batch, 5 * 64 - 3, 9 * 64 - 7, 64, np.float16, density=0.45, empty_rows=(2,))
     x = np.random.default_rng(batch).uniform(-1, 1, (batch, lay.N)).astype(np.float16)
     L = pb.Layer.from_synth(lay)
+    want = {0: "tile", 2: "tile_cluster", 3: "tile_persist"}.get(tile_kernel)
+    assert want is None or L.launch_info(batch)["kernel"] == want
     for act in (0, 1):
         y = pb.pp_forward(L, _dev(x), act).cpu().numpy()
         assert L.status() == 0
@@ -422,8 +424,10 @@ def test_tile_path_both_kernels_same_bits_and_repeatable(pb):
     data the clustered kernel and the one-block-row kernel agree exactly."""
     lay = _rand_layer(977, 10 * 64 - 9, 23 * 64 - 1, 64, np.float16, density=0.3, empty_rows=(5,), integer=True)
     x = np.random.default_rng(3).integers(-2, 3, (128, lay.N)).astype(np.float16)
-    L = pb.Layer.from_synth(lay)
     try:
+        pb.pp_set_tuning(12, 3)                       # the persistent kernel's plan is built when the layer is created
+        L = pb.Layer.from_synth(lay)
+        assert L.launch_info(128)["kernel"] == "tile_persist"
         pb.pp_set_tuning(12, 2)
         y1 = pb.pp_forward(L, _dev(x), 0).cpu().numpy()
         y1b = pb.pp_forward(L, _dev(x), 0).cpu().numpy()

@@ -58,12 +58,12 @@ def test_persistent_kernel_x_wait_runs_out(pb, one_poll):
 def test_tile_kernels_stage_wait_runs_out(pb, one_poll, tile_kernel):
     wl = synth.config5(k=128, batch=40, scale=0.125)      # 1024 x 1024, every tile kept
     lay = wl.layers[0]
-    L = pb.Layer.from_synth(lay)
     x = torch.from_numpy(wl.x).cuda()
     y_ref, _, a = po.layer_forward(lay, wl.x.astype(np.float64))
-    pb.pp_set_tuning(12, tile_kernel)
+    pb.pp_set_tuning(12, tile_kernel)                 # before the layer exists: the persistent kernel's plan is built at creation
     try:
-        assert L.launch_info(40)["kernel"] in ("tile", "tile_cluster", "tile_persist")
+        L = pb.Layer.from_synth(lay)
+        assert L.launch_info(40)["kernel"] == {0: "tile", 2: "tile_cluster", 3: "tile_persist"}[tile_kernel]
         one_poll(1)
         pb.pp_forward(L, x, lay.act)
         assert L.status() == PP_ERR_TIMEOUT
