@@ -226,8 +226,10 @@ pp_status_t pp_forward(pp_layer_t* layer, const void* x, void* y, int batch,
  * back, all on the given stream, and returns after the stream has drained, so y_host is valid on
  * return.  Unlike the calls above this one synchronises, and its first call on a layer (or a call
  * with a larger batch than any before) allocates the layer's two staging buffers.
- * x_host  host, [batch][N] row-major, element type = the layer's wdtype (pinned memory makes the
- *         copies asynchronous to the host, pageable memory works)
+ * x_host  host, [batch][N] row-major, element type = the layer's wdtype.  Pageable memory works (copy-engine
+ *         transfers).  When both buffers are page-locked and mapped into the device's address space
+ *         (cudaHostAlloc, cudaHostRegister) the library moves them with two small kernels of its own instead,
+ *         which takes less time per call than setting up two transfers.
  * y_host  host, float [batch][M]
  * Errors: as pp_forward, plus PP_ERR_ALLOC. */
 pp_status_t pp_forward_host(pp_layer_t* layer, const void* x_host, float* y_host, int batch,
@@ -464,7 +466,9 @@ pp_status_t pp_selftest_host(void);
  *         and at every pp_chain_forward), 0 (default) one launch per layer
  * key 15: polls after which the bounded device-side waits of the persistent kernel (copy of x) and of the chain
  *         kernel (layer boundaries) give up; 0 (default) = the kernels' own limits (seconds).  Small values exist
- *         so that tests can see a wait give up: the kernel then raises its status word and still ends by itself */
+ *         so that tests can see a wait give up: the kernel then raises its status word and still ends by itself
+ * key 16: 1 (default) pp_forward_host moves page-locked host buffers that the device can address with small
+ *         kernels, 0 always uses cudaMemcpyAsync */
 pp_status_t pp_set_tuning(int key, int value);
 
 #ifdef __cplusplus

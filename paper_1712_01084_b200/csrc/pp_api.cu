@@ -610,6 +610,51 @@ pp_status_t pp_forward(pp_layer_t* L, const void* x, void* y, int batch, pp_act_
     return forward_impl(L, x, y, batch, act, static_cast<cudaStream_t>(cuda_stream), false);
 }
 
+namespace {
+
+// Copies between the layer's staging buffers and page-locked host memory that the device can address: a few CTAs
+// move 16-byte words (bytes where a pointer or the length is not a multiple of 16), which costs one trip over the
+// host link instead of the set-up of a copy engine transfer.  The kernel lets the next launch start at once and
+// waits for the previous one itself (programmatic stream serialization; both are no-ops in a plain launch).
+__global__ void __launch_bounds__(1024) host_link_copy_kernel(unsigned char* __restrict__ dst,
+                                                              const unsigned char* __restrict__ src, size_t bytes) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x, nthr = (size_t)gridDim.x * blockDim.x;
+    if (((reinterpret_cast<uintptr_t>(dst) | reinterpret_cast<uintptr_t>(src)) & 15) == 0) {
+        const size_t words = bytes / 16;
+        for (size_t i = tid; i < words; i += nthr)
+            reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(src)[i];
+        for (size_t i = words * 16 + tid; i < bytes; i += nthr) dst[i] = src[i];
+    } else {
+        for (size_t i = tid; i < bytes; i += nthr) dst[i] = src[i];
+    }
+}
+
+// Device address of a host pointer if it lies in page-locked memory mapped into the device's address space
+// (cudaHostAlloc, cudaHostRegister), nullptr otherwise (pageable memory, or the query failed).
+void* device_view_of_host(const void* host) {
+    cudaPointerAttributes attr{};
+    if (cudaPointerGetAttributes(&attr, host) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return attr.type == cudaMemoryTypeHost ? attr.devicePointer : nullptr;
+}
+
+cudaError_t launch_host_link_copy(void* dst, const void* src, size_t bytes, bool dependent, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)std::min<size_t>(64, (bytes + 16383) / 16384));
+    cfg.blockDim = dim3(1024);
+    cfg.stream = stream;
+    cudaLaunchAttribute at{};
+    at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &at;
+    cfg.numAttrs = dependent ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, host_link_copy_kernel, static_cast<unsigned char*>(dst),
+                              static_cast<const unsigned char*>(src), bytes);
+}
+
+}  // namespace
+
 pp_status_t pp_forward_host(pp_layer_t* L, const void* x_host, float* y_host, int batch, pp_act_t act, void* cuda_stream) {
     if (!L || !x_host || !y_host || batch < 1) return PP_ERR_INVALID_ARG;
     if (act != PP_ACT_IDENTITY && act != PP_ACT_RELU) return PP_ERR_INVALID_ARG;
@@ -627,11 +672,25 @@ pp_status_t pp_forward_host(pp_layer_t* L, const void* x_host, float* y_host, in
         L->host_batch = batch;
     }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    if (cudaMemcpyAsync(L->d_host_x, x_host, (size_t)batch * pk->N * esz, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    const size_t xbytes = (size_t)batch * pk->N * esz, ybytes = (size_t)batch * pk->M * 4;
+    // Page-locked buffers the device can address are moved by small kernels (no copy-engine set-up, and the layer
+    // kernel's prologue runs under the inbound copy); anything else goes through cudaMemcpyAsync.
+    void* xv = pp::g_host_link_kernels ? device_view_of_host(x_host) : nullptr;
+    void* yv = xv ? device_view_of_host(y_host) : nullptr;
+    if (xv && yv) {
+        if (launch_host_link_copy(L->d_host_x, xv, xbytes, false, stream) != cudaSuccess) return PP_ERR_CUDA;
+        const pp_status_t st = forward_impl(L, L->d_host_x, L->d_host_y, batch, act, stream, false);
+        if (st != PP_OK) return st;
+        if (launch_host_link_copy(yv, L->d_host_y, ybytes, pp::g_stream_pdl != 0, stream) != cudaSuccess ||
+            cudaStreamSynchronize(stream) != cudaSuccess)
+            return PP_ERR_CUDA;
+        return PP_OK;
+    }
+    if (cudaMemcpyAsync(L->d_host_x, x_host, xbytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
         return PP_ERR_CUDA;
     const pp_status_t st = forward_impl(L, L->d_host_x, L->d_host_y, batch, act, stream, false);
     if (st != PP_OK) return st;
-    if (cudaMemcpyAsync(y_host, L->d_host_y, (size_t)batch * pk->M * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+    if (cudaMemcpyAsync(y_host, L->d_host_y, ybytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
         cudaStreamSynchronize(stream) != cudaSuccess)
         return PP_ERR_CUDA;
     return PP_OK;

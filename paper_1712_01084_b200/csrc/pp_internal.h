@@ -62,6 +62,7 @@ extern int g_tile_min_batch;  // fp16 B = 64 layers take the tensor-core tile pa
 extern int g_prepass;         // 1: permute multi-column inputs in a pre-pass when the kernel cannot do it in shared memory
 extern int g_link_identity;  // 1: chain links whose folded map is the identity store pivoted rows directly (Section 4.2.3)
 extern int g_lstm_persist;  // 1: recurrent cells run all steps in one cooperative kernel when the gate weights fit shared memory
+extern int g_host_link_kernels;   // 1: pp_forward_host moves page-locked, device-addressable host buffers with kernels instead of copy-engine transfers
 extern int g_chain_fused;    // 1: chains of fp16 layers run as one cooperative kernel when they qualify
 extern int g_stage_direct;   // batch 1: read x through the index array instead of permuting it first
 

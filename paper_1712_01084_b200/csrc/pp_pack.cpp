@@ -17,6 +17,7 @@ int g_lstm_persist = 1;
 int g_tile_cluster = 1;
 int g_tile_persist_auto = 0;
 int g_link_identity = 1;
+int g_host_link_kernels = 1;   // pp_forward_host: page-locked, device-addressable host buffers are moved by kernels
 int g_chain_fused = 0;      // measured: one launch per layer (programmatic dependent launch) is the faster way through a chain
 extern int g_stream_wait_polls;   // poll limit of the bounded device-side waits (pp_stream.cu)
 int g_stage_direct = 2;    // 0: always materialise the pivoted x in shared memory; 1: one input vector is read through the
@@ -409,6 +410,7 @@ pp_status_t pp_set_tuning(int key, int value) {
     if (key == 13 && (value == 0 || value == 1)) { pp::g_link_identity = value; return PP_OK; }
     if (key == 14 && (value == 0 || value == 1)) { pp::g_chain_fused = value; return PP_OK; }
     if (key == 15 && value >= 0) { pp::g_stream_wait_polls = value; return PP_OK; }
+    if (key == 16 && (value == 0 || value == 1)) { pp::g_host_link_kernels = value; return PP_OK; }
     return PP_ERR_INVALID_ARG;
 }
 

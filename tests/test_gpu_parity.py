@@ -595,18 +595,32 @@ def test_chain_identity_link_with_padding_rows(pb):
 
 def test_forward_host_matches_device_call(pb):
     """pp_forward_host (host buffers in, host buffers out) gives the bits of pp_forward, also when a second
-    call brings a larger batch (the staging buffers grow) and for pageable as well as pinned memory."""
+    call brings a larger batch (the staging buffers grow); pageable buffers (copy-engine transfers), page-locked
+    ones (moved by the library's own kernels, with lengths and addresses that are no multiples of 16 bytes) and
+    page-locked ones with tuning key 16 = 0."""
     lay = _rand_layer(4242, 300, 500, 32, np.float16, density=0.4)
     L = pb.Layer.from_synth(lay)
-    for batch, pin in ((1, True), (5, False), (3, True)):
-        x = np.random.default_rng(batch).uniform(-1, 1, (batch, lay.N)).astype(np.float16)
-        xh = torch.from_numpy(x)
-        xh = xh.pin_memory() if pin else xh
-        yh = pb.pp_forward_host(L, xh, 1)
-        yd = pb.pp_forward(L, _dev(x), 1).cpu()
-        assert torch.equal(yh, yd)
-        y_ref, _, a = po.layer_forward(lay, x.astype(np.float64), act=1, threads=4)
-        _check(yh.numpy(), y_ref, a, np.float16, f"host call batch {batch}")
+    try:
+        for batch, pin, key16, offset in ((1, True, 1, 0), (5, False, 1, 0), (3, True, 1, 0), (40, True, 1, 0),
+                                          (2, True, 0, 0), (1, True, 1, 1), (7, True, 1, 3)):
+            pb.pp_set_tuning(16, key16)
+            x = np.random.default_rng(batch).uniform(-1, 1, (batch, lay.N)).astype(np.float16)
+            if pin:                         # views into page-locked buffers, optionally off the 16-byte grid
+                xbuf = torch.empty(batch * lay.N + 8, dtype=torch.float16).pin_memory()
+                ybuf = torch.full((batch * lay.M + 8,), float("nan"), dtype=torch.float32).pin_memory()
+                xh = xbuf[offset:offset + batch * lay.N].view(batch, lay.N)
+                xh.copy_(torch.from_numpy(x))
+                out = ybuf[offset:offset + batch * lay.M].view(batch, lay.M)
+                yh = pb.pp_forward_host(L, xh, 1, out=out)
+                assert torch.isnan(ybuf[:offset]).all() and torch.isnan(ybuf[offset + batch * lay.M:]).all()
+            else:
+                yh = pb.pp_forward_host(L, torch.from_numpy(x), 1)
+            yd = pb.pp_forward(L, _dev(x), 1).cpu()
+            assert torch.equal(yh, yd), (batch, pin, key16, offset)
+            y_ref, _, a = po.layer_forward(lay, x.astype(np.float64), act=1, threads=4)
+            _check(yh.numpy(), y_ref, a, np.float16, f"host call batch {batch}")
+    finally:
+        pb.pp_set_tuning(16, 1)
     L.close()
 
 
@@ -631,3 +645,37 @@ def test_several_vectors_through_the_index_array(pb, B, batch, key7):
                     assert np.array_equal(y.astype(np.float64), y_ref)
     finally:
         pb.pp_set_tuning(7, 2)
+
+
+@pytest.mark.parametrize("tile_kernel,pdl", [(1, 1), (0, 1), (2, 0), (3, 1)])
+def test_interleaved_calls_of_several_layers_without_synchronising(pb, tile_kernel, pdl):
+    """Calls of different layers, batches and kernel families are enqueued back to back (each launch may begin
+    while the previous one is still running: dependent launches) and only checked at the end."""
+    rng = np.random.default_rng(100 + tile_kernel)
+    specs = [(700, 900, 64, np.float16, 1.0), (333, 200, 16, np.float32, 0.3), (2100, 1500, 64, np.float16, 0.5),
+             (650, 480, 32, np.float16, 0.2)]
+    pb.pp_set_tuning(12, tile_kernel)
+    pb.pp_set_tuning(8, pdl)
+    try:
+        lays = [_rand_layer(50 + i, M, N, B, dt, density=d) for i, (M, N, B, dt, d) in enumerate(specs)]
+        Ls = [pb.Layer.from_synth(l) for l in lays]
+        plan = []
+        for batch in (1, 130, 9, 1, 40, 2, 128, 16, 1, 31, 8, 64):
+            for i in rng.permutation(len(lays))[:3]:
+                x = rng.uniform(-1, 1, (batch, lays[i].N)).astype(lays[i].tile_values.dtype)
+                plan.append((int(i), x, int(rng.integers(0, 2))))
+        xs = [_dev(x) for _, x, _ in plan]
+        torch.cuda.synchronize()
+        outs = [pb.pp_forward(Ls[i], xd, act) for (i, _, act), xd in zip(plan, xs)]
+        torch.cuda.synchronize()
+        kernels = {Ls[i].launch_info(x.shape[0])["kernel"] for i, x, _ in plan}
+        assert {"stream", "gemv"} <= kernels and any(k.startswith("tile") for k in kernels)
+        for (i, x, act), yd in zip(plan, outs):
+            y_ref, _, a = po.layer_forward(lays[i], x.astype(np.float64), act=act, threads=8)
+            _check(yd.cpu().numpy(), y_ref, a, lays[i].tile_values.dtype, f"layer {i} batch {x.shape[0]}")
+        for L in Ls:
+            assert L.status() == 0
+            L.close()
+    finally:
+        pb.pp_set_tuning(12, 1)
+        pb.pp_set_tuning(8, 1)
