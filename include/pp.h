@@ -452,13 +452,14 @@ pp_status_t pp_selftest_host(void);
  *        the device (fragment order for the matrix-vector kernels, 8 KiB shared-memory images for the tile
  *        kernels: 2 x T x 8 KiB); a layer created while this key is 0 skips the second copy and never takes the
  *        tile path, whatever the key says later
- * key 12: tensor-core kernel of batched fp16 B = 64 layers: 0 one block-row per CTA; 2 the clustered kernel (4
- *         block-rows per cluster of 4 CTAs share every X block); 3 the persistent kernel (one CTA per SM over an
- *         equal share of the layer's steps, two accumulator sets in tensor memory, groups split between CTAs
- *         summed through partial-sum slots in global memory in a fixed order; measured slower than the other
- *         two, kept as an option: the key must be 3 when the layer is created, because the plan and its
- *         slots, 128 KiB per unit, are only allocated then; other layers fall back to one block-row per CTA); 1 (default) the clustered kernel when the groups' tile-columns carry at
- *         least 3.5 of 4 possible tiles on average, else one block-row per CTA
+ * key 12: tensor-core kernel of batched fp16 B = 64 layers: 0 or 1 (default) one block-row per CTA, its tiles
+ *         dealt round robin to four warps that issue the tensor-core instructions into accumulators of their own
+ *         (measured the fastest at every density and batch); 2 the clustered kernel (4 block-rows per cluster of
+ *         4 CTAs share every X block); 3 the persistent kernel (one CTA per SM over an equal share of the layer's
+ *         steps, two accumulator sets in tensor memory, groups split between CTAs summed through partial-sum
+ *         slots in global memory in a fixed order: the key must be 3 when the layer is created, because the plan
+ *         and its slots, 128 KiB per unit, are only allocated then; other layers fall back to one block-row per
+ *         CTA).  2 and 3 are kept as options
  * key 13: 1 (default) chain links whose folded map is the identity store pivoted rows without an index array,
  *         0 sends them through the map like any other link
  * key 11: 1 (default) lets pp_lstm_forward run all steps in one cooperative kernel when the layer qualifies, 0 never

@@ -32,8 +32,14 @@ namespace {
 constexpr int kProducers = 4;      // producer warps (one lane each issues bulk copies; the stage count is a multiple of it)
 constexpr int kXBytes = kTileBatch * 64 * 2;     // 128 x 64 fp16 = 16 KiB
 constexpr int kWBytes = 64 * 64 * 2;             // 64 x 64 fp16 = 8 KiB
-constexpr int kTmemCols = 64;
-constexpr int kThreads = 32 * (kProducers + 1 + 4);    // producers, MMA issuer, 4 epilogue warps
+// One-block-row kernel: the thread that issues the tensor-core instructions spends about 0.16 us per tile on the
+// hand-shake alone (wait for the stage, fence, commit) plus 0.03 us per instruction, whatever the instruction's
+// shape and whether any data moves at all (measured with the copies and the instructions taken out in turn), while
+// the copies of a tile take 0.17 us.  So kIssuers warps share the tiles of the block-row round robin, each with an
+// accumulator of its own in tensor memory; the epilogue adds the accumulators in a fixed order.
+constexpr int kIssuers = 4;
+constexpr int kTmemCols = 64 * kIssuers;
+constexpr int kThreads = 32 * (kProducers + kIssuers + 4);    // producers, MMA issuers, 4 epilogue warps
 constexpr int kPollLimit = 1 << 22;
 constexpr int kIdxCap = 512;       // tiles of a block-row whose indices are staged in shared memory
 
@@ -115,6 +121,18 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
                  :: "r"(smem_u32(bar)) : "memory");
 }
 
+#ifdef PP_TRACE
+__device__ __forceinline__ void tile_stamp(const TileArgs& a, int slot) {
+    if (a.trace) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t) :: "memory");
+        a.trace[(size_t)blockIdx.x * 8 + slot] = t;
+    }
+}
+#else
+__device__ __forceinline__ void tile_stamp(const TileArgs&, int) {}
+#endif
+
 // STAGES stages of (XB bytes of the X block + one tile).  A stage is re-used once per STAGES tiles and a
 // copy takes 1.5-2 us to land, so small batches (which need only the first 8-row groups of the X block)
 // trade the unused part of the X region for more stages in flight.
@@ -147,6 +165,7 @@ tile_f16_kernel(const TileArgs a) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int br = blockIdx.x;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next call's gather kernel may fetch its index entries meanwhile
+    if (threadIdx.x == 0 && blockIdx.x < 148) tile_stamp(a, 0);
     const int t0 = __ldg(a.row_ptr + br), k = __ldg(a.row_ptr + br + 1) - t0;
 
     // The block-row's tile list goes to shared memory once, by the whole CTA, while tensor memory is set
@@ -161,7 +180,7 @@ tile_f16_kernel(const TileArgs a) {
     }
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&sm->full[s], 1); mbar_init(&sm->empty[s], 1); }
-        mbar_init(&sm->acc_full, 1);
+        mbar_init(&sm->acc_full, kIssuers);
         sm->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -210,27 +229,31 @@ tile_f16_kernel(const TileArgs a) {
                     for (int i = 0; i < kPollLimit && !mbar_try_wait(&sm->full[t % kStages], (t / kStages) & 1); ++i) {}
             }
         }
-    } else if (warp == kProducers) {
-        // ---------------- MMA issuer (one lane)
+    } else if (warp < kProducers + kIssuers) {
+        // ---------------- MMA issuers (one lane each): issuer i takes tiles i, i + kIssuers, ... into accumulator i
         if (lane == 0) {
+            const int me = warp - kProducers;
+            const uint32_t acc = tmem + (uint32_t)(me * 64);
             bool ok = true, issued = false;
             const uint64_t desc0 = smem_desc_sw128(smem_u32(stages));
-            for (int t = 0; t < k && ok; ++t) {
+            for (int t = me; t < k && ok; t += kIssuers) {
                 const int s = t % kStages;
                 ok = mbar_wait(&sm->full[s], (t / kStages) & 1, abort_flag, a.polls);
                 if (!ok) break;
+                if (t == 0 && blockIdx.x < 148) tile_stamp(a, 1);
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint64_t xd = desc_advance(desc0, (uint32_t)(s * kStageBytes)), wd = desc_advance(xd, XB);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk)
-                    umma_f16(tmem, desc_advance(xd, kk * 32), desc_advance(wd, kk * 32), t > 0 || kk > 0);
+                    umma_f16(acc, desc_advance(xd, kk * 32), desc_advance(wd, kk * 32), issued || kk > 0);
                 issued = true;
                 umma_commit(&sm->empty[s]);          // frees the stage once these MMAs have read it
             }
-            // accumulator complete; when giving up after some tiles, the epilogue (and the release of tensor
-            // memory behind it) still waits for the instructions already issued
+            // this issuer's accumulator is complete; when giving up after some tiles, the epilogue (and the release
+            // of tensor memory behind it) still waits for the instructions already issued
             if (issued) umma_commit(&sm->acc_full);
             else mbar_arrive(&sm->acc_full);               // nothing was issued: nothing to wait for
+            if (me == 0 && blockIdx.x < 148) tile_stamp(a, 2);
         }
     } else {
         // ---------------- epilogue: 4 warps, warp (w % 4) owns tensor-memory lanes 32 (w % 4) ..
@@ -246,40 +269,47 @@ tile_f16_kernel(const TileArgs a) {
         // the tensor-memory loads below are warp-wide instructions: the whole warp takes one decision
         const bool ok = __all_sync(0xffffffffu, mbar_wait(&sm->acc_full, 0, abort_flag, 0) && !*abort_flag);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (threadIdx.x == 32 * (kProducers + kIssuers) && blockIdx.x < 148) tile_stamp(a, 3);
         if (ok && q * 32 < a.batch) {
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t r[32];
-                if (k > 0) {
-                    asm volatile(
-                        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-                        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-                        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-                          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-                          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                        : "r"(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0));
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                } else {
+                // the sum of the accumulators that received tiles (issuer i did iff k > i), in issuer order
+                float v[32];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) r[j] = 0u;
+                for (int j = 0; j < 32; ++j) v[j] = 0.0f;
+#pragma unroll
+                for (int i = 0; i < kIssuers; ++i) {
+                    if (i < k) {                 // the same decision in every lane: the load is a warp-wide instruction
+                        uint32_t r[32];
+                        asm volatile(
+                            "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                            "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                            "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                            : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                              "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                              "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                              "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                            : "r"(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(i * 64 + c0)));
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] += __uint_as_float(r[j]);
+                    }
                 }
                 // Transpose the 32 x 32 block through shared memory (the stages are idle by now), so that the
                 // lanes of a store run over output rows: 32 scattered words of ONE row of y.  With lanes over
                 // batch rows the words of a store lie a whole row pitch apart and crowd a few L2 slices.
                 float* xpose = reinterpret_cast<float*>(stages) + q * (32 * 33);
 #pragma unroll
-                for (int j = 0; j < 32; ++j) xpose[lane * 33 + j] = __uint_as_float(r[j]);
+                for (int j = 0; j < 32; ++j) xpose[lane * 33 + j] = v[j];
                 __syncwarp();
                 const float bias = sm->bias[c0 + lane];
                 const int dst = sm->dst[c0 + lane];
 #pragma unroll 8
                 for (int rr = 0; rr < 32; ++rr) {
                     const int bb = q * 32 + rr;
-                    float v = xpose[rr * 33 + lane] + bias;
-                    if (a.act == PP_ACT_RELU) v = fmaxf(v, 0.0f);
-                    if (dst >= 0 && bb < a.batch) a.y[(size_t)bb * a.ldy + dst] = v;
+                    float o = xpose[rr * 33 + lane] + bias;
+                    if (a.act == PP_ACT_RELU) o = fmaxf(o, 0.0f);
+                    if (dst >= 0 && bb < a.batch) a.y[(size_t)bb * a.ldy + dst] = o;
                 }
                 __syncwarp();
             }
@@ -287,6 +317,7 @@ tile_f16_kernel(const TileArgs a) {
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (threadIdx.x == 0 && blockIdx.x < 148) tile_stamp(a, 4);
     if (threadIdx.x == 0 && sm->abort_flag) *a.status = 1;
     if (warp == kProducers) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kTmemCols) : "memory");
@@ -619,17 +650,6 @@ __device__ __forceinline__ TileUnit load_unit(const TileUnit* p) {
     return u;
 }
 
-#ifdef PP_TRACE
-__device__ __forceinline__ void tile_stamp(const TileArgs& a, int slot) {
-    if (a.trace) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        a.trace[(size_t)blockIdx.x * 8 + slot] = t;
-    }
-}
-#else
-__device__ __forceinline__ void tile_stamp(const TileArgs&, int) {}
-#endif
 
 // Which unit of a group finishes chunk q of the group's rows.
 __device__ __forceinline__ int chunk_owner(int q, int n_parts) { return n_parts <= kPChunks ? q % n_parts : q; }
