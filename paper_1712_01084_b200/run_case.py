@@ -5,6 +5,7 @@
     python -m paper_1712_01084_b200.run_case cfg3 --batch 8 --calls 4 [--one-kernel]
     python -m paper_1712_01084_b200.run_case cfg4 --steps 64 --calls 2
     python -m paper_1712_01084_b200.run_case cfg5 --k 32 --batch 20 --no-tile      # chunked matrix-vector kernel
+    python -m paper_1712_01084_b200.run_case cfg5 --k 128 --batch 128 --tile-kernel 2     # clustered tile kernel
 
 Calls rotate over `--copies` independent copies of the layer(s) (default: enough to exceed twice the L2, at
 most 4) so that a profiled launch does not find its weights in L2.  Plain launches on the current stream, one
@@ -29,6 +30,8 @@ def main():
     ap.add_argument("--one-kernel", action="store_true", help="cfg3: the whole chain as one cooperative kernel")
     ap.add_argument("--no-tile", action="store_true", help="keep fp16 B=64 layers off the tensor-core tile path")
     ap.add_argument("--no-pdl", action="store_true", help="launch without programmatic stream serialization")
+    ap.add_argument("--tile-kernel", type=int, default=1, choices=[0, 1, 2, 3],
+                    help="tensor-core tile kernel (tuning key 12): 1 automatic, 0 one block-row per CTA, 2 clustered, 3 persistent")
     args = ap.parse_args()
 
     import torch
@@ -42,6 +45,7 @@ def main():
         pb.pp_set_tuning(8, 0)
     if args.one_kernel:
         pb.pp_set_tuning(14, 1)
+    pb.pp_set_tuning(12, args.tile_kernel)      # before any layer exists: the persistent kernel's plan is built at creation
     l2 = 126 * 2 ** 20
 
     def copies_for(weight_bytes):
