@@ -12,12 +12,14 @@
 //     with two bulk asynchronous copies per tile (cp.async.bulk, one request each, every CTA fetching for itself),
 //     signalling mbarriers (2-D tensor-map loads of 128-byte rows were request-rate bound: 60 us vs
 //     the same data as two contiguous copies);
-//   * warp 4 issues tcgen05.mma (kind::f16, accumulator in tensor memory) from shared-memory matrix
-//     descriptors and frees each stage with tcgen05.commit;
-//   * warps 5..8 read the accumulator with tcgen05.ld and run the fused epilogue: bias, activation,
-//     store through the row index array (Listing 1's last step).
-// A second kernel (further down) lets a cluster of four CTAs share the X blocks of four block-rows;
-// it wins when most tile-columns of a group carry tiles in all four block-rows.
+//   * warps 4..7 (one lane each) issue tcgen05.mma (kind::f16, accumulators in tensor memory) from
+//     shared-memory matrix descriptors and free each stage with tcgen05.commit; the tiles go round robin to
+//     the four warps, each with an accumulator of its own, because one thread cannot issue faster than
+//     a tile per 0.28 us;
+//   * warps 8..11 read the accumulators with tcgen05.ld, add them and run the fused epilogue: bias,
+//     activation, store through the row index array (Listing 1's last step).
+// A second kernel (further down) lets a cluster of four CTAs share the X blocks of four block-rows, a third
+// gives every SM an equal share of the work; both are slower (measured) and run only on request.
 // Every wait on an mbarrier is bounded; on a time-out the kernel raises the layer's status word,
 // stops issuing work, lets its outstanding copies land, frees its tensor memory and returns.
 #include <cuda_fp16.h>
