@@ -109,7 +109,7 @@ namespace {
 void lstm_plan_persistent(pp_lstm* R) {
     const pp_packed* pk = R->gates->pk;
     R->persist_grid = 0;
-    if (pk->wdtype != PP_F16 || R->H > 4 * 512 || pk->Npad % 8 != 0) return;
+    if (pk->wdtype != PP_F16 || R->H > 4 * 512 || pk->Npad % 8 != 0 || pk->Mpad >= 65536 || pk->Npad >= 65536) return;
     const int S = (int)pk->strip_start.size() - 1;
     int dev = 0, sms = 0, coop = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
