@@ -469,7 +469,14 @@ pp_status_t pp_selftest_host(void);
  *         kernel (layer boundaries) give up; 0 (default) = the kernels' own limits (seconds).  Small values exist
  *         so that tests can see a wait give up: the kernel then raises its status word and still ends by itself
  * key 16: 1 (default) pp_forward_host moves page-locked host buffers that the device can address with small
- *         kernels, 0 always uses cudaMemcpyAsync */
+ *         kernels, 0 always uses cudaMemcpyAsync
+ * key 17: 1 is the caller's promise, for the pp_forward / pp_forward_pivoted calls made while it is set, that x was
+ *         complete before any kernel still in flight in the stream was enqueued (independent requests whose inputs
+ *         were uploaded earlier; NOT a chain, where x is the previous call's y).  The persistent kernel (batch <= 8)
+ *         then fetches x before it waits for the previous kernel and waits only in front of its first write to y
+ *         or scratch, so consecutive calls overlap further; other kernels ignore the key.  0 (default): every read
+ *         of x waits for the previous kernel.  With the promise broken the call reads x too early: wrong values,
+ *         no fault */
 pp_status_t pp_set_tuning(int key, int value);
 
 #ifdef __cplusplus

@@ -338,12 +338,14 @@ pp::StreamArgs make_stream_args(const pp_layer* L, const int32_t* gather, const 
 // Enqueue one layer in groups of batch columns.
 // Persistent kernel for up to kStreamMaxBatch columns; PP_ERR_UNSUPPORTED when x does not fit shared memory.
 pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_len, int x_elt, void* y, int ldy,
-                       int out_mode, int batch, pp_act_t act, cudaStream_t stream, int x_limit, const int32_t* scatter) {
+                       int out_mode, int batch, pp_act_t act, cudaStream_t stream, int x_limit, const int32_t* scatter,
+                       bool x_ready = false) {
     const pp_packed* pk = L->pk;
     const bool rows_aligned = aligned16(x) && (batch == 1 || ((size_t)ldx * x_elt) % 16 == 0);
     const int stage_mode = pick_stage_mode(L, gather != nullptr, gather == L->d_gather, rows_aligned, x_len, batch);
     if (stage_mode < 0) return PP_ERR_UNSUPPORTED;
-    const pp::StreamArgs s = make_stream_args(L, gather, x, ldx, x_len, y, ldy, out_mode, batch, act, x_limit, scatter, stage_mode);
+    pp::StreamArgs s = make_stream_args(L, gather, x, ldx, x_len, y, ldy, out_mode, batch, act, x_limit, scatter, stage_mode);
+    s.x_ready = x_ready ? 1 : 0;
     return pp::launch_stream(pk->wdtype, pk->B, s, pk->cta_desc.data(), L->stream_grid, stream) == cudaSuccess
                ? PP_OK : PP_ERR_CUDA;
 }
@@ -355,7 +357,7 @@ pp_status_t run_stream(pp_layer* L, const int32_t* gather, const void* x, int ld
 // per SM and measured 60 us per pass against 85 us for one chunked pass over 16 columns).
 pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx, int x_len, int x_elt, void* y, int ldy,
                       int out_mode, int batch, pp_act_t act, cudaStream_t stream, int x_limit = -1,
-                      const int32_t* scatter = nullptr) {
+                      const int32_t* scatter = nullptr, bool x_ready = false) {
     const pp_packed* pk = L->pk;
     if (x_limit < 0) x_limit = pk->N;      // without a gather map: columns at or beyond x_limit read 0
     if (!scatter) scatter = L->d_scatter;  // a chain passes the map into its consumer's column order instead
@@ -396,7 +398,7 @@ pp_status_t run_layer(pp_layer* L, const int32_t* gather, const void* x, int ldx
             const int nb = batch - b0 < pp::kStreamMaxBatch ? batch - b0 : pp::kStreamMaxBatch;
             const pp_status_t st = run_stream(L, gather, static_cast<const char*>(x) + (size_t)b0 * ldx * x_elt, ldx, x_len,
                                               x_elt, static_cast<char*>(y) + (size_t)b0 * ldy * y_elt, ldy, out_mode, nb, act,
-                                              stream, x_limit, scatter);
+                                              stream, x_limit, scatter, x_ready);
             if (st == PP_ERR_UNSUPPORTED && b0 == 0) { done = false; break; }   // x too large to stage: chunked kernel
             if (st != PP_OK) return st;
         }
@@ -576,7 +578,10 @@ pp_status_t pp_layer_destroy(pp_layer_t* layer) {
 }
 
 // One layer forward; pivoted: y is float[batch][M_pad] in pivoted row order (no output index array).
-static pp_status_t forward_impl(pp_layer* L, const void* x, void* y, int batch, pp_act_t act, cudaStream_t stream, bool pivoted) {
+// x_ready: the caller's promise of tuning key 17 (only the persistent kernels act on it; a pre-pass or the copy of
+// pp_forward_host produces x inside the stream, so those paths never pass it on).
+static pp_status_t forward_impl(pp_layer* L, const void* x, void* y, int batch, pp_act_t act, cudaStream_t stream, bool pivoted,
+                                bool x_ready = false) {
     const pp_packed* pk = L->pk;
     const int ldy = pivoted ? pk->Mpad : pk->M;
     if (L->tile_ok && pp::g_tile_min_batch > 0 && batch >= pp::g_tile_min_batch && (size_t)pk->N * 2 <= 48 * 1024) {
@@ -600,14 +605,14 @@ static pp_status_t forward_impl(pp_layer* L, const void* x, void* y, int batch, 
         return PP_OK;
     }
     return run_layer(L, L->d_gather, x, pk->N, pk->N, pk->wdtype == PP_F16 ? 2 : 4, y, ldy,
-                     pivoted ? pp::OUT_PIVOTED_F32 : pp::OUT_SCATTER_F32, batch, act, stream);
+                     pivoted ? pp::OUT_PIVOTED_F32 : pp::OUT_SCATTER_F32, batch, act, stream, -1, nullptr, x_ready);
 }
 
 pp_status_t pp_forward(pp_layer_t* L, const void* x, void* y, int batch, pp_act_t act, void* cuda_stream) {
     if (!L || !x || !y || batch < 1 || x == y) return PP_ERR_INVALID_ARG;
     if (act != PP_ACT_IDENTITY && act != PP_ACT_RELU) return PP_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(y)) return PP_ERR_INVALID_ARG;
-    return forward_impl(L, x, y, batch, act, static_cast<cudaStream_t>(cuda_stream), false);
+    return forward_impl(L, x, y, batch, act, static_cast<cudaStream_t>(cuda_stream), false, pp::g_stream_x_ready != 0);
 }
 
 namespace {
@@ -707,7 +712,7 @@ pp_status_t pp_forward_pivoted(pp_layer_t* L, const void* x, float* y_piv, int b
     if (!L || !x || !y_piv || batch < 1 || x == static_cast<const void*>(y_piv)) return PP_ERR_INVALID_ARG;
     if (act != PP_ACT_IDENTITY && act != PP_ACT_RELU) return PP_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(y_piv)) return PP_ERR_INVALID_ARG;
-    return forward_impl(L, x, y_piv, batch, act, static_cast<cudaStream_t>(cuda_stream), true);
+    return forward_impl(L, x, y_piv, batch, act, static_cast<cudaStream_t>(cuda_stream), true, pp::g_stream_x_ready != 0);
 }
 
 pp_status_t pp_chain_create(pp_chain_t** out, pp_layer_t* const* layers, const pp_act_t* acts, int n_layers,

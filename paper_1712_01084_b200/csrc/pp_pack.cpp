@@ -24,6 +24,7 @@ int g_stage_direct = 2;    // 0: always materialise the pivoted x in shared memo
                            // index array in the multiply loop; 2: so are 2..8 vectors of fp16 layers
 extern int g_stream_depth; // weight-ring slots per warp of the persistent kernel (pp_stream.cu)
 extern int g_stream_pdl;   // programmatic dependent launch of the persistent kernel (pp_stream.cu)
+extern int g_stream_x_ready;   // pp_forward fetches x before the dependency wait (pp_stream.cu)
 }
 
 namespace {
@@ -411,6 +412,7 @@ pp_status_t pp_set_tuning(int key, int value) {
     if (key == 14 && (value == 0 || value == 1)) { pp::g_chain_fused = value; return PP_OK; }
     if (key == 15 && value >= 0) { pp::g_stream_wait_polls = value; return PP_OK; }
     if (key == 16 && (value == 0 || value == 1)) { pp::g_host_link_kernels = value; return PP_OK; }
+    if (key == 17 && (value == 0 || value == 1)) { pp::g_stream_x_ready = value; return PP_OK; }
     return PP_ERR_INVALID_ARG;
 }
 

@@ -475,10 +475,15 @@ struct XoffWindow {
 // its own prologue.  wait(): called by all threads after a CTA barrier; on return everything the producer wrote
 // is visible; false when a bounded wait gave up (the CTA then leaves the kernel).
 struct LaunchDependency {      // the producer is the previous kernel in the stream (programmatic dependent launch)
+    bool x_ready;              // x does not come from a kernel still in flight: only the writes have to wait
     __device__ __forceinline__ void release() const { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
     __device__ __forceinline__ bool wait() const {
-        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (!x_ready) asm volatile("griddepcontrol.wait;" ::: "memory");
         return true;
+    }
+    // called right before the layer's first write to global memory (y, exchange slots, counters)
+    __device__ __forceinline__ void wait_before_writes() const {
+        if (x_ready) asm volatile("griddepcontrol.wait;" ::: "memory");
     }
 };
 
@@ -665,6 +670,7 @@ __device__ __forceinline__ bool stream_f16_layer(const StreamArgs& a, const CtaD
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     trace_stamp(a, 4);
+    dep.wait_before_writes();
     finalize<RG>(a, d, L);
     trace_stamp(a, 5);
     return true;
@@ -674,7 +680,7 @@ template <int U>
 __global__ void __launch_bounds__(kThreads, 2) stream_f16_kernel(const __grid_constant__ StreamLaunch P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     init_xbar(carve(smem_raw, 16, U, P.a, 2));
-    stream_f16_layer<U>(P.a, cta_range(P), smem_raw, 0u, LaunchDependency{});
+    stream_f16_layer<U>(P.a, cta_range(P), smem_raw, 0u, LaunchDependency{P.a.x_ready != 0});
 }
 
 // ------------------------------------------------------------------ a whole chain of fp16 layers in one kernel
@@ -690,6 +696,7 @@ struct GridCounterDependency {
     int* status;
     int polls;
     __device__ __forceinline__ void release() const {}
+    __device__ __forceinline__ void wait_before_writes() const {}
     __device__ __forceinline__ bool wait() const {
         __shared__ int ok_flag;
         if (threadIdx.x == 0) {
@@ -812,7 +819,7 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const __grid_co
     warm_translations(a);
     __syncthreads();
     trace_stamp(a, 1);
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!a.x_ready) asm volatile("griddepcontrol.wait;" ::: "memory");
     trace_stamp(a, 2);
     issue_x<float>(a, L);
     finish_stage<float, U>(a, L);
@@ -885,6 +892,7 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const __grid_co
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     trace_stamp(a, 4);
+    if (a.x_ready) asm volatile("griddepcontrol.wait;" ::: "memory");    // y and scratch may still be in use by the previous kernel
     finalize<RG>(a, d, L);
     trace_stamp(a, 5);
 }
@@ -940,6 +948,7 @@ constexpr int kTraceCtas = 320;
 int g_stream_wait_polls = 0;   // polls before a bounded device-side wait gives up; 0 = the kernels' defaults
 int g_stream_depth = 0;   // ring slots per warp: 4, 6 or 8; 0 = chosen per launch
 int g_stream_pdl = 1;     // launch with programmatic stream serialization (prologue overlaps the previous kernel)
+int g_stream_x_ready = 0; // launches fetch x before the dependency wait (the caller's promise, tuning key 17)
 
 namespace {
 size_t smem_bytes_at(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int depth);

@@ -22,6 +22,9 @@ struct StreamArgs {
     int* counters;               // [S], zero between launches
     int* status;                 // raised to 1 when the bounded wait for the copy of x gave up; may be NULL
     int wait_polls;              // polls before the bounded wait for the copy of x gives up (0: the kernel's default; set by the launcher)
+    int x_ready;                 // 1: the caller promises that x was complete before anything still in flight in the stream was
+                                 // enqueued, so x is fetched BEFORE the dependency wait, which moves in front of the first write
+                                 // to y or scratch (set by the launcher from tuning key 17)
     unsigned long long* trace;   // diagnostic builds (PP_TRACE): [grid][8] time stamps of the kernel's phases; else unused
     int ldx, ldy;
     int x_limit;                 // with gather_idx == NULL: columns >= x_limit read 0
@@ -72,6 +75,7 @@ int chain_resident_ctas(size_t smem, int depth);            // CTAs of the chain
 // smem: 2 * region_bytes; depth: weight copies each warp keeps in flight (4 or 8), the same for every layer
 cudaError_t launch_chain_f16(const ChainLaunch& P, int grid, size_t smem, int depth, cudaStream_t stream);
 extern int g_stream_wait_polls;
+extern int g_stream_x_ready;   // tuning key 17: value of StreamArgs::x_ready for launches through launch_stream
 
 // host_table: the plan's CTA ranges in host memory (grid entries); small plans travel to the
 // kernel inside its parameters so that no CTA starts with a dependent global load.

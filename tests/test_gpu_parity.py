@@ -679,3 +679,33 @@ def test_interleaved_calls_of_several_layers_without_synchronising(pb, tile_kern
     finally:
         pb.pp_set_tuning(12, 1)
         pb.pp_set_tuning(8, 1)
+
+
+@pytest.mark.parametrize("dtype,B", [(np.float16, 64), (np.float16, 16), (np.float32, 32)])
+def test_inputs_ready_before_the_stream(pb, dtype, B):
+    """Tuning key 17: inputs that were complete before the calls were enqueued are fetched ahead of the dependency
+    wait; only the writes wait for the previous kernel.  Many calls of the same layers back to back (so consecutive
+    kernels share exchange slots, counters and shared strips) must give the bits of the ordinary calls."""
+    rng = np.random.default_rng(1700 + B)
+    lays = [_rand_layer(170 + B, 1100, 1300, B, dtype, density=0.5, integer=True),
+            _rand_layer(171 + B, 260, 200, B, dtype, density=0.7, integer=True)]
+    Ls = [pb.Layer.from_synth(l) for l in lays]
+    plan = [(int(rng.integers(0, 2)), int(b)) for b in (1, 1, 3, 1, 8, 1, 2, 1, 1, 5, 1, 1) for _ in range(3)]
+    xs = [rng.integers(-3, 4, (b, lays[i].N)).astype(dtype) for i, b in plan]
+    xd = [_dev(x) for x in xs]
+    torch.cuda.synchronize()                         # every input is complete before the first call is enqueued
+    try:
+        pb.pp_set_tuning(17, 1)
+        outs = [pb.pp_forward(Ls[i], x, 1) for (i, _), x in zip(plan, xd)]
+        torch.cuda.synchronize()
+    finally:
+        pb.pp_set_tuning(17, 0)
+    assert all(Ls[i].launch_info(b)["kernel"] == "stream" for i, b in plan)
+    for (i, b), x, yd in zip(plan, xs, outs):
+        y_ref, _, _ = po.layer_forward(lays[i], x.astype(np.float64), act=1, threads=8)
+        assert np.array_equal(yd.cpu().numpy().astype(np.float64), y_ref), f"layer {i} batch {b}"
+    for L in Ls:
+        assert L.status() == 0
+        L.close()
+    with pytest.raises(pb.PPError):
+        pb.pp_set_tuning(17, 2)
