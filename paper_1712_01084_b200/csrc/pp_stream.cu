@@ -90,7 +90,7 @@ __device__ __forceinline__ int x_index(const StreamArgs& a, int pj) {
 // Shared memory: fixed header, then the regions whose size depends on the launch.
 struct SmemLayout {
     int* sstart;     // [kStreamMaxStrips + 1] strip starts of this CTA's strips
-    int* wlohi;      // [kStreamMaxStrips] first | last << 8 warp that parked a partial for the strip
+    int* wlohi;      // [kStreamMaxStrips] bit w set: warp w parked a partial sum for the strip
     int* flags;      // [2]
     int* wb;         // [kStreamWarps + 1] fragment position where each warp's range starts
     uint64_t* xbar;  // mbarrier the bulk copies of x complete on
@@ -294,24 +294,60 @@ __device__ __forceinline__ void finish_stage(const StreamArgs& a, const SmemLayo
 }
 
 // Which warps will park a partial sum for each of this CTA's strips (their ranges intersect the strip
-// inside the CTA).  Runs right after the staging barrier, off the kernel's tail; the barrier that ends
-// the streaming phase publishes the result.
+// inside the CTA).  Runs right after the staging barrier; the barrier that ends the streaming phase
+// publishes the result.  Sixteen lanes share a strip: lane w tests where warp w's range starts against the
+// strip's first and last fragment inside the CTA, and since those starts ascend the highest lane that passes
+// names the warp (one thread per strip walking all warps held warp 0 back by 0.6 us, which is the whole
+// multiply phase of a small layer).
+static_assert(kStreamWarps == 16, "plan_parks gives half a warp to every strip");
 __device__ __forceinline__ void plan_parks(const CtaDesc& d, const SmemLayout& L) {
-    for (int ls = threadIdx.x; ls < d.s_count; ls += kThreads) {
-        const int lo = max(L.sstart[ls], d.p_begin), hi = min(L.sstart[ls + 1], d.p_end);
-        int w_lo = 1, w_hi = 0;
-        if (lo < hi) {
-            w_lo = w_hi = 0;
-            for (int w = 1; w < kStreamWarps; ++w) {
-                if (L.wb[w] <= lo) w_lo = w;
-                if (L.wb[w] <= hi - 1) w_hi = w;
-            }
+    const int w = threadIdx.x & 15, half = (threadIdx.x >> 4) & 1;
+    const int total = d.s_count * kStreamWarps;
+    for (int base = 0; base < total; base += kThreads) {
+        const int e = base + (int)threadIdx.x, ls = e >> 4;
+        const bool in = e < total;
+        int lo = 0, hi = 0;
+        bool at_lo = false, at_hi = false, live = false;
+        if (in) {
+            lo = max(L.sstart[ls], d.p_begin);
+            hi = min(L.sstart[ls + 1], d.p_end);
+            const int wbeg = L.wb[w];
+            at_lo = wbeg <= lo;
+            at_hi = wbeg <= hi - 1;
+            live = wbeg < L.wb[w + 1];                    // a warp with an empty range parks nothing
         }
-        L.wlohi[ls] = w_lo | (w_hi << 8);
+        const unsigned m_lo = (__ballot_sync(0xffffffffu, at_lo) >> (16 * half)) & 0xffffu;
+        const unsigned m_hi = (__ballot_sync(0xffffffffu, at_hi) >> (16 * half)) & 0xffffu;
+        const unsigned m_live = (__ballot_sync(0xffffffffu, live) >> (16 * half)) & 0xffffu;
+        if (in && w == 0) {
+            unsigned mask = 0u;                           // an empty intersection: no warp parks
+            if (lo < hi) {                                // warp 0 starts at the CTA's first fragment, so bit 0 is set in both
+                const int w_lo = 31 - __clz((int)m_lo), w_hi = 31 - __clz((int)m_hi);
+                mask = m_live & ((2u << w_hi) - 1u) & ~((1u << w_lo) - 1u);
+            }
+            L.wlohi[ls] = (int)mask;
+        }
     }
 }
 
 constexpr unsigned kEmptySlot = 0xffffffffu;   // exchange slots rest at this NaN pattern
+
+// Sum of the partial sums the warps parked for element `rem` (row * batch + column) of local strip `ls`, in warp
+// order.  All sixteen candidate loads are issued before the first addition (a loop that tested and loaded warp after
+// warp was a chain of sixteen shared-memory round trips on every call's tail).
+template <int RG>
+__device__ __forceinline__ float sum_parks_of(const SmemLayout& L, int ls, int rem, int per_strip) {
+    const unsigned m = (unsigned)L.wlohi[ls];
+    const float* base = L.segp + (size_t)ls * per_strip + rem;
+    float s[kStreamWarps];
+#pragma unroll
+    for (int w = 0; w < kStreamWarps; ++w) s[w] = (m >> w) & 1u ? base[w * per_strip] : 0.0f;
+    float v = 0.0f;
+#pragma unroll
+    for (int w = 0; w < kStreamWarps; ++w)
+        if ((m >> w) & 1u) v += s[w];
+    return v;
+}
 
 // Everything after the last barrier of the streaming phase: per-strip sums, cross-CTA reduction,
 // bias + activation + (scatter | pivoted store).  RG = rows per strip.
@@ -351,10 +387,7 @@ __device__ __forceinline__ void finalize(const StreamArgs& a, const CtaDesc& d, 
     if (single) {
         for (int e = tid; e < d.s_count * RG; e += kThreads) {
             const int ls = e / RG, r = e % RG;
-            const int wl = L.wlohi[ls] & 0xff, wh = L.wlohi[ls] >> 8;
-            float v = 0.0f;
-            for (int w = wl; w <= wh; ++w)
-                if (L.wb[w] < L.wb[w + 1]) v += L.segp[(ls + w) * RG + r];
+            float v = sum_parks_of<RG>(L, ls, r, per_strip);
             const int4 info = L.sinfo[ls];
             if (info.y == 2) {
                 unsigned* slot = reinterpret_cast<unsigned*>(a.partials + (size_t)info.z * (RG * kStreamMaxBatch) + r);
@@ -375,10 +408,7 @@ __device__ __forceinline__ void finalize(const StreamArgs& a, const CtaDesc& d, 
     for (int e = tid; e < n_out; e += kThreads) {
         const int ls = e / per_strip, rem = e - ls * per_strip;
         const int r = rem / batch, b = rem - r * batch;
-        const int wl = L.wlohi[ls] & 0xff, wh = L.wlohi[ls] >> 8;
-        float v = 0.0f;
-        for (int w = wl; w <= wh; ++w)      // warps with an empty range parked nothing
-            if (L.wb[w] < L.wb[w + 1]) v += L.segp[((ls + w) * RG + r) * batch + b];
+        const float v = sum_parks_of<RG>(L, ls, rem, per_strip);
         const int4 info = L.sinfo[ls];
         if (info.y == 1) {
             emit(ls, r, b, v);
@@ -452,19 +482,28 @@ struct WeightRing {
     }
 };
 
+// A read-only global load that is issued where it stands: the compiler may move an ordinary load down to the first
+// use of its value, which for a table fetched ahead of the dependency wait puts a trip to L2 or DRAM (0.7 us) back on
+// the critical path behind the wait.
+__device__ __forceinline__ int ld_nc_here(const int32_t* p) {
+    int v;
+    asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+
 // Column offsets of 32 consecutive fragments, one per lane, fetched one block ahead.
 struct XoffWindow {
     const int32_t* xoff;
     int cur, nxt, base;    // cur covers fragments [base, base + 32)
     __device__ __forceinline__ void init(const int32_t* table, int wbeg, int wend, int lane) {
         xoff = table; base = wbeg;
-        cur = wbeg + lane < wend ? __ldg(xoff + wbeg + lane) : 0;
-        nxt = wbeg + 32 + lane < wend ? __ldg(xoff + wbeg + 32 + lane) : 0;
+        cur = wbeg + lane < wend ? ld_nc_here(xoff + wbeg + lane) : 0;
+        nxt = wbeg + 32 + lane < wend ? ld_nc_here(xoff + wbeg + 32 + lane) : 0;
     }
     __device__ __forceinline__ int get(int p, int wend, int lane) {
         if (p - base == 32) {
             base += 32; cur = nxt;
-            nxt = base + 32 + lane < wend ? __ldg(xoff + base + 32 + lane) : 0;
+            nxt = base + 32 + lane < wend ? ld_nc_here(xoff + base + 32 + lane) : 0;
         }
         return __shfl_sync(0xffffffffu, cur, p - base);
     }
@@ -667,6 +706,7 @@ __device__ __forceinline__ bool stream_f16_layer(const StreamArgs& a, const CtaD
         }
         park(ls + warp);
     }
+    trace_stamp(a, 6);
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     trace_stamp(a, 4);
@@ -845,50 +885,102 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const __grid_co
         const float* xlane = xs + (lane / RG) * 4;
         const bool direct = a.stage_mode >= 3, idx16 = a.stage_mode == 4;
         const float* rawf = static_cast<const float*>(L.raw);
-        for (int base = wbeg; base < wend; base += U) {
+        // one fragment: 4 columns of RG rows (lane = row; with 16-row strips the upper half-warp takes the next 4 columns)
+        auto multiply = [&](const uint4 wa, int xoff) {
+            const float w0 = __uint_as_float(wa.x), w1 = __uint_as_float(wa.y);
+            const float w2 = __uint_as_float(wa.z), w3 = __uint_as_float(wa.w);
+            if (direct) {            // batch 1: read x through the index array (index -1 reads raw[-1] = 0)
+                int4 ii;
+                if (idx16) {
+                    const uint2 pp2 = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(L.idxs) + xoff + (lane / RG) * 4);
+                    ii = make_int4((int)(pp2.x & 0xffffu) - 1, (int)(pp2.x >> 16) - 1, (int)(pp2.y & 0xffffu) - 1, (int)(pp2.y >> 16) - 1);
+                } else {
+                    ii = *reinterpret_cast<const int4*>(L.idxs + xoff + (lane / RG) * 4);
+                }
+                acc[0][0] = fmaf(w0, rawf[ii.x], acc[0][0]);
+                acc[0][1] = fmaf(w1, rawf[ii.y], acc[0][1]);
+                acc[0][0] = fmaf(w2, rawf[ii.z], acc[0][0]);
+                acc[0][1] = fmaf(w3, rawf[ii.w], acc[0][1]);
+                return;
+            }
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int p = base + u;
-                if (p < wend) {
-                    if (p == seg_end) {
-                        park(ls + warp);
-                        do { ++ls; } while (L.sstart[ls + 1] <= p);
-                        seg_end = min(wend, L.sstart[ls + 1]);
-                    }
-                    const int xoff = xw.get(p, wend, lane);
-                    const uint4 wa = ring.take(u);
-                    ring.fill(u, p + U, wend);
-                    const float w0 = __uint_as_float(wa.x), w1 = __uint_as_float(wa.y);
-                    const float w2 = __uint_as_float(wa.z), w3 = __uint_as_float(wa.w);
-                    if (direct) {            // batch 1: read x through the index array (index -1 reads raw[-1] = 0)
-                        int4 ii;
+            for (int b = 0; b < NB; ++b) {
+                if (b < a.batch) {
+                    const float4 xv = *reinterpret_cast<const float4*>(xlane + b * a.xs_stride + xoff);
+                    acc[b][0] = fmaf(w0, xv.x, acc[b][0]);
+                    acc[b][1] = fmaf(w1, xv.y, acc[b][1]);
+                    acc[b][0] = fmaf(w2, xv.z, acc[b][0]);
+                    acc[b][1] = fmaf(w3, xv.w, acc[b][1]);
+                }
+            }
+        };
+        auto next_strip = [&](int p) {
+            park(ls + warp);
+            do { ++ls; } while (L.sstart[ls + 1] <= p);
+            seg_end = min(wend, L.sstart[ls + 1]);
+        };
+        if (wend - wbeg <= U) {
+            // A short range was requested whole by the prologue and finish_stage has waited for it: plain
+            // shared-memory loads, nothing to wait for and nothing to refill.
+            // One input vector: four fragments of one strip at a time, every load of the four issued before the first
+            // use (offset -> index entries -> x values is a chain of three shared-memory round trips, about 0.2 us
+            // when every fragment walks it alone).  The sums are added in the same order as one by one.
+#pragma unroll 1
+            for (int p = wbeg; p < wend;) {
+                if (p == seg_end) next_strip(p);
+                if (direct && p + 4 <= seg_end) {
+                    int xo[4];
+                    uint4 wa[4];
+                    int4 ii[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) xo[j] = xw.get(p + j, wend, lane);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) wa[j] = ring.slot[32 * (p + j - wbeg)];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
                         if (idx16) {
-                            const uint2 pp2 = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(L.idxs) + xoff + (lane / RG) * 4);
-                            ii = make_int4((int)(pp2.x & 0xffffu) - 1, (int)(pp2.x >> 16) - 1, (int)(pp2.y & 0xffffu) - 1, (int)(pp2.y >> 16) - 1);
+                            const uint2 pp2 = *reinterpret_cast<const uint2*>(reinterpret_cast<const uint16_t*>(L.idxs) + xo[j] + (lane / RG) * 4);
+                            ii[j] = make_int4((int)(pp2.x & 0xffffu) - 1, (int)(pp2.x >> 16) - 1, (int)(pp2.y & 0xffffu) - 1, (int)(pp2.y >> 16) - 1);
                         } else {
-                            ii = *reinterpret_cast<const int4*>(L.idxs + xoff + (lane / RG) * 4);
+                            ii[j] = *reinterpret_cast<const int4*>(L.idxs + xo[j] + (lane / RG) * 4);
                         }
-                        acc[0][0] = fmaf(w0, rawf[ii.x], acc[0][0]);
-                        acc[0][1] = fmaf(w1, rawf[ii.y], acc[0][1]);
-                        acc[0][0] = fmaf(w2, rawf[ii.z], acc[0][0]);
-                        acc[0][1] = fmaf(w3, rawf[ii.w], acc[0][1]);
-                        continue;
+                    }
+                    float xv[4][4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        xv[j][0] = rawf[ii[j].x]; xv[j][1] = rawf[ii[j].y]; xv[j][2] = rawf[ii[j].z]; xv[j][3] = rawf[ii[j].w];
                     }
 #pragma unroll
-                    for (int b = 0; b < NB; ++b) {
-                        if (b < a.batch) {
-                            const float4 xv = *reinterpret_cast<const float4*>(xlane + b * a.xs_stride + xoff);
-                            acc[b][0] = fmaf(w0, xv.x, acc[b][0]);
-                            acc[b][1] = fmaf(w1, xv.y, acc[b][1]);
-                            acc[b][0] = fmaf(w2, xv.z, acc[b][0]);
-                            acc[b][1] = fmaf(w3, xv.w, acc[b][1]);
-                        }
+                    for (int j = 0; j < 4; ++j) {
+                        acc[0][0] = fmaf(__uint_as_float(wa[j].x), xv[j][0], acc[0][0]);
+                        acc[0][1] = fmaf(__uint_as_float(wa[j].y), xv[j][1], acc[0][1]);
+                        acc[0][0] = fmaf(__uint_as_float(wa[j].z), xv[j][2], acc[0][0]);
+                        acc[0][1] = fmaf(__uint_as_float(wa[j].w), xv[j][3], acc[0][1]);
+                    }
+                    p += 4;
+                    continue;
+                }
+                multiply(ring.slot[32 * (p - wbeg)], xw.get(p, wend, lane));
+                ++p;
+            }
+        } else {
+            for (int base = wbeg; base < wend; base += U) {
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int p = base + u;
+                    if (p < wend) {
+                        if (p == seg_end) next_strip(p);
+                        const int xoff = xw.get(p, wend, lane);
+                        const uint4 wa = ring.take(u);
+                        ring.fill(u, p + U, wend);
+                        multiply(wa, xoff);
                     }
                 }
             }
         }
         park(ls + warp);
     }
+    trace_stamp(a, 6);
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     trace_stamp(a, 4);
