@@ -216,12 +216,50 @@ __device__ __forceinline__ void init_xbar(const SmemLayout& L) {
     }
 }
 
+// Which warps will park a partial sum for each of this CTA's strips (their ranges intersect the strip
+// inside the CTA).  Runs right after the staging barrier; the barrier that ends the streaming phase
+// publishes the result.  Sixteen lanes share a strip: lane w tests where warp w's range starts against the
+// strip's first and last fragment inside the CTA, and since those starts ascend the highest lane that passes
+// names the warp (one thread per strip walking all warps held warp 0 back by 0.6 us, which is the whole
+// multiply phase of a small layer).
+static_assert(kStreamWarps == 16, "plan_parks gives half a warp to every strip");
+__device__ __forceinline__ void plan_parks(const CtaDesc& d, const SmemLayout& L) {
+    const int w = threadIdx.x & 15, half = (threadIdx.x >> 4) & 1;
+    const int total = d.s_count * kStreamWarps;
+    for (int base = 0; base < total; base += kThreads) {
+        const int e = base + (int)threadIdx.x, ls = e >> 4;
+        const bool in = e < total;
+        int lo = 0, hi = 0;
+        bool at_lo = false, at_hi = false, live = false;
+        if (in) {
+            lo = max(L.sstart[ls], d.p_begin);
+            hi = min(L.sstart[ls + 1], d.p_end);
+            const int wbeg = L.wb[w];
+            at_lo = wbeg <= lo;
+            at_hi = wbeg <= hi - 1;
+            live = wbeg < L.wb[w + 1];                    // a warp with an empty range parks nothing
+        }
+        const unsigned m_lo = (__ballot_sync(0xffffffffu, at_lo) >> (16 * half)) & 0xffffu;
+        const unsigned m_hi = (__ballot_sync(0xffffffffu, at_hi) >> (16 * half)) & 0xffffu;
+        const unsigned m_live = (__ballot_sync(0xffffffffu, live) >> (16 * half)) & 0xffffu;
+        if (in && w == 0) {
+            unsigned mask = 0u;                           // an empty intersection: no warp parks
+            if (lo < hi) {                                // warp 0 starts at the CTA's first fragment, so bit 0 is set in both
+                const int w_lo = 31 - __clz((int)m_lo), w_hi = 31 - __clz((int)m_hi);
+                mask = m_live & ((2u << w_hi) - 1u) & ~((1u << w_lo) - 1u);
+            }
+            L.wlohi[ls] = (int)mask;
+        }
+    }
+}
+
 constexpr int kXWaitPolls = 1 << 22;   // default polls of the x barrier before the kernel gives up (seconds; a copy that lands never gets near it)
 
 // Phase 3: wait for the copies of phases 1 and 2, finish the staged pivoted x.  x_parity: phase of the x barrier
-// this use completes (0 for the first use in a kernel, alternating after that).
+// this use completes (0 for the first use in a kernel, alternating after that).  The park plan, which needs the
+// CTA's tables but not x, is made while the copy of x is still on its way.
 template <typename T, int U>
-__device__ __forceinline__ void finish_stage(const StreamArgs& a, const SmemLayout& L, uint32_t x_parity = 0u) {
+__device__ __forceinline__ void finish_stage(const StreamArgs& a, const CtaDesc& d, const SmemLayout& L, uint32_t x_parity = 0u) {
     constexpr int EPC = 16 / (int)sizeof(T);
     const int tid = threadIdx.x;
     const T* x = static_cast<const T*>(a.x);
@@ -240,6 +278,8 @@ __device__ __forceinline__ void finish_stage(const StreamArgs& a, const SmemLayo
                 dst[b * dst_stride + j] = j < n_src ? x[(size_t)b * a.ldx + j] : T(0.0f);
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");   // tables and first weight fragments have landed
+    __syncthreads();                                        // ... for every thread, and the stores above are visible
+    plan_parks(d, L);
     if (a.stage_mode != 0 && (a.stage_mode != 2 ? a.x_len : a.x_limit) >= EPC) {   // and so must x
         const uint32_t bar = (uint32_t)__cvta_generic_to_shared(L.xbar);
         uint32_t ok = 0u;
@@ -290,44 +330,9 @@ __device__ __forceinline__ void finish_stage(const StreamArgs& a, const SmemLayo
             }
         }
     }
-    __syncthreads();
-}
-
-// Which warps will park a partial sum for each of this CTA's strips (their ranges intersect the strip
-// inside the CTA).  Runs right after the staging barrier; the barrier that ends the streaming phase
-// publishes the result.  Sixteen lanes share a strip: lane w tests where warp w's range starts against the
-// strip's first and last fragment inside the CTA, and since those starts ascend the highest lane that passes
-// names the warp (one thread per strip walking all warps held warp 0 back by 0.6 us, which is the whole
-// multiply phase of a small layer).
-static_assert(kStreamWarps == 16, "plan_parks gives half a warp to every strip");
-__device__ __forceinline__ void plan_parks(const CtaDesc& d, const SmemLayout& L) {
-    const int w = threadIdx.x & 15, half = (threadIdx.x >> 4) & 1;
-    const int total = d.s_count * kStreamWarps;
-    for (int base = 0; base < total; base += kThreads) {
-        const int e = base + (int)threadIdx.x, ls = e >> 4;
-        const bool in = e < total;
-        int lo = 0, hi = 0;
-        bool at_lo = false, at_hi = false, live = false;
-        if (in) {
-            lo = max(L.sstart[ls], d.p_begin);
-            hi = min(L.sstart[ls + 1], d.p_end);
-            const int wbeg = L.wb[w];
-            at_lo = wbeg <= lo;
-            at_hi = wbeg <= hi - 1;
-            live = wbeg < L.wb[w + 1];                    // a warp with an empty range parks nothing
-        }
-        const unsigned m_lo = (__ballot_sync(0xffffffffu, at_lo) >> (16 * half)) & 0xffffu;
-        const unsigned m_hi = (__ballot_sync(0xffffffffu, at_hi) >> (16 * half)) & 0xffffu;
-        const unsigned m_live = (__ballot_sync(0xffffffffu, live) >> (16 * half)) & 0xffffu;
-        if (in && w == 0) {
-            unsigned mask = 0u;                           // an empty intersection: no warp parks
-            if (lo < hi) {                                // warp 0 starts at the CTA's first fragment, so bit 0 is set in both
-                const int w_lo = 31 - __clz((int)m_lo), w_hi = 31 - __clz((int)m_hi);
-                mask = m_live & ((2u << w_hi) - 1u) & ~((1u << w_lo) - 1u);
-            }
-            L.wlohi[ls] = (int)mask;
-        }
-    }
+    // modes 2..4 wrote nothing to shared memory since the barrier above (every thread has seen the x barrier
+    // complete itself); the permutation passes of modes 0 and 1 did
+    if (a.stage_mode < 2) __syncthreads();
 }
 
 constexpr unsigned kEmptySlot = 0xffffffffu;   // exchange slots rest at this NaN pattern
@@ -583,9 +588,8 @@ __device__ __forceinline__ bool stream_f16_layer(const StreamArgs& a, const CtaD
     issue_x<__half>(a, L);
 
     // 3. pivoted x in shared memory
-    finish_stage<__half, U>(a, L, x_parity);
+    finish_stage<__half, U>(a, d, L, x_parity);
     trace_stamp(a, 3);
-    plan_parks(d, L);
 
     // 4. stream this warp's share
     float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -862,9 +866,8 @@ __global__ void __launch_bounds__(kThreads, 2) stream_f32_kernel(const __grid_co
     if (!a.x_ready) asm volatile("griddepcontrol.wait;" ::: "memory");
     trace_stamp(a, 2);
     issue_x<float>(a, L);
-    finish_stage<float, U>(a, L);
+    finish_stage<float, U>(a, d, L);
     trace_stamp(a, 3);
-    plan_parks(d, L);
 
     float acc[NB][2];
 #pragma unroll
