@@ -24,7 +24,8 @@
  * current CUDA device.  All *_create calls copy what they are given; the caller
  * keeps ownership of its arrays.  Handles own their device memory until the
  * matching *_destroy.  The forward calls only ENQUEUE work on the given stream:
- * they never synchronise and never allocate.  Calls that use the same handle
+ * they never synchronise and never allocate (pp_forward_host, which works on
+ * host buffers, is the one exception and says so below).  Calls that use the same handle
  * must be ordered on one stream (a handle owns scratch memory that concurrent
  * calls would share).  Every failure is a return code; nothing aborts or traps.
  * There is no CPU fallback.
