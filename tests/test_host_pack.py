@@ -576,3 +576,16 @@ def test_layout_study_layouts(size, nb):
     assert np.array_equal(pb.pp_layout_pack(size, nb, pb.PP_LAYOUT_BRC, v), v.reshape(-1))
     assert np.array_equal(pb.pp_layout_pack(size, nb, pb.PP_LAYOUT_BCR, v), v.transpose(0, 2, 1).reshape(-1))
     assert np.array_equal(pb.pp_layout_pack(size, nb, pb.PP_LAYOUT_CBR, v), v.transpose(2, 0, 1).reshape(-1))
+
+
+def test_tuning_keys_reject_values_out_of_range():
+    """pp_set_tuning is host code: every key takes its documented values and refuses the others (no GPU needed)."""
+    from paper_1712_01084_b200 import binding as pb
+    good = {5: (0, 1), 6: (4, 6, 8, 0), 7: (0, 1, 2), 8: (0, 1), 12: (2, 3, 1), 13: (0, 1), 15: (7, 0), 16: (0, 1), 17: (1, 0)}
+    bad = {5: 2, 6: 5, 7: 3, 8: -1, 12: 4, 13: 2, 15: -1, 16: 2, 17: 2, 99: 0}
+    for key, values in good.items():
+        for v in values:                 # the last value of each tuple is the default, which stays set
+            pb.pp_set_tuning(key, v)
+    for key, v in bad.items():
+        with pytest.raises(pb.PPError):
+            pb.pp_set_tuning(key, v)
