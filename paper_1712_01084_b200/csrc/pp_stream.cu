@@ -677,6 +677,40 @@ __device__ __forceinline__ bool stream_f16_layer(const StreamArgs& a, const CtaD
                 }
                 continue;
             }
+            if (GRP == 8 && direct1) {
+                // One input vector, a group that ends the warp's range or crosses a strip boundary: the B operands
+                // of the (up to) eight fragments are built at once, then one pass per strip the group touches
+                // (nearly always one).  A fragment costs two tests, two shuffles, the ring slot and the tensor-core
+                // instruction: while the weights are in shared memory the SM is bound by instruction issue (eight
+                // warps per scheduler), and the per-fragment bookkeeping of the general loop below took three times
+                // as many instructions, which is most of the multiply phase of a sparse layer.
+                gather8(base);
+                const int gend = min(base + 8, wend);
+                int p = base;
+                while (true) {
+                    if (p == seg_end) {
+                        park(ls + warp);
+                        acc[0] = acc[1] = acc[2] = acc[3] = 0.0f;
+                        do { ++ls; } while (L.sstart[ls + 1] <= p);
+                        seg_end = min(wend, L.sstart[ls + 1]);
+                    }
+                    const int end = min(gend, seg_end);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int q = base + j;
+                        if (q >= p && q < end) {
+                            const uint32_t b0 = __shfl_sync(0xffffffffu, mb0, j * 4 + t);
+                            const uint32_t b1 = __shfl_sync(0xffffffffu, mb1, j * 4 + t);
+                            const uint4 wa = ring.take(j % U);
+                            ring.fill(j % U, q + U, wend);
+                            mma_16x8x16(acc, wa, b0, b1);
+                        }
+                    }
+                    p = end;
+                    if (p >= gend) break;
+                }
+                continue;
+            }
 #pragma unroll
             for (int j = 0; j < GRP; ++j) {
                 const int p = base + j;
