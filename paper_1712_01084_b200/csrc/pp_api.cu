@@ -566,7 +566,8 @@ pp_status_t pp_layer_launch_info(const pp_layer_t* L, int batch, int32_t out[6])
     const bool stream_path = stage >= 0 && (batch + pp::kStreamMaxBatch - 1) / pp::kStreamMaxBatch <= (batch + chunk_group - 1) / chunk_group;
     if (!stream_path) { out[0] = 0; out[1] = L->n_items; return PP_OK; }
     out[0] = 1; out[1] = L->stream_grid; out[4] = stage;
-    out[2] = pp::stream_pick_depth(pk->wdtype, pk->B, pk->Npad, pk->N, L->stream_max_rows, nb, stage, L->stream_grid);
+    out[2] = pp::stream_pick_depth(pk->wdtype, pk->B, pk->Npad, pk->N, L->stream_max_rows, nb, stage, L->stream_grid,
+                                   pp::stream_frags_per_warp(pk->cta_desc.data(), L->stream_grid));
     out[3] = (int32_t)pp::stream_launch_smem(pk->wdtype, pk->B, pk->Npad, pk->N, L->stream_max_rows, nb, stage, out[2]);
     out[5] = pp::g_stream_pdl;
     return PP_OK;

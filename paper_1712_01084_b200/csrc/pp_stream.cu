@@ -1083,13 +1083,31 @@ namespace {
 size_t smem_bytes_at(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int depth);
 }
 
+// Fragments a warp of the plan streams on average (the ring depth is chosen by it).
+int stream_frags_per_warp(const CtaDesc* host_table, int grid) {
+    if (!host_table || grid <= 0) return 0;
+    long long frags = 0;
+    for (int c = 0; c < grid; ++c) frags += host_table[c].p_end - host_table[c].p_begin;
+    return (int)(frags / ((long long)grid * kStreamWarps));
+}
+
+constexpr int kDeepRingFrags = 17;   // between 13.8 (density 0.25, 4 copies faster) and 20.8 (0.375, 8 copies faster) on 8192 x 8192
+
 // Weight copies each warp keeps in flight.  Two CTAs share an SM when the grid is larger than the SM
 // count and a CTA needs at most half of the SM's shared memory: then 4 per warp (64 KiB in flight per
 // SM).  A CTA that has the SM to itself takes the deepest ring that still fits.
-int stream_pick_depth(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int grid) {
+int stream_pick_depth(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int grid,
+                      int frags_per_warp) {
     if (g_stream_depth) return g_stream_depth;
     if (grid > 148 && smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, 4) <= 113 * 1024) {
-        return 4;                 // two CTAs per SM: deeper rings measured no faster
+        // Two CTAs per SM.  Long ranges of fp16 fragments stream faster with 8 copies per warp in flight when two
+        // such CTAs still fit an SM (8192 x 8192 at density 1 / 0.5 / 0.375: 23.2 / 12.8 / 10.3 us with 4 copies,
+        // 22.7 / 12.3 / 9.8 us with 8); short ranges are slower that way (density 0.25 and below: a call is one burst
+        // of requests, and the deeper prologue only queues the copy of x behind more weight traffic).
+        if (dt == PP_F16 && frags_per_warp >= kDeepRingFrags &&
+            smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, 8) <= 113 * 1024)
+            return 8;
+        return 4;
     }
     for (int d : {8, 6})
         if (smem_bytes_at(dt, B, n_pad, x_len, max_rows, batch, stage_mode, d) <= kStreamSmemLimit) return d;
@@ -1203,7 +1221,8 @@ cudaError_t launch_stream(pp_dtype_t dt, int B, const StreamArgs& a_in, const Ct
 #endif
     if (grid <= kParamCtas)
         for (int c = 0; c < grid; ++c) P.table[c] = host_table[c];
-    const int depth = stream_pick_depth(dt, B, a.n_pad, a.x_len, a.max_rows, a.batch, a.stage_mode, grid);
+    const int depth = stream_pick_depth(dt, B, a.n_pad, a.x_len, a.max_rows, a.batch, a.stage_mode, grid,
+                                        stream_frags_per_warp(host_table, grid));
     const size_t smem = smem_bytes_at(dt, B, a.n_pad, a.x_len, a.max_rows, a.batch, a.stage_mode, depth);
     if (dt == PP_F16) {
         if (depth == 8) return launch_one<stream_f16_kernel<8>>(P, grid, smem, stream);

@@ -48,7 +48,9 @@ struct StreamArgs {
 // chunked kernel when it exceeds kStreamSmemLimit.
 size_t stream_smem_bytes(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode);
 // Ring depth a launch picks, and the dynamic shared memory of a launch with that depth (max_rows as in the plan).
-int stream_pick_depth(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int grid);
+int stream_pick_depth(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int grid,
+                      int frags_per_warp);
+int stream_frags_per_warp(const CtaDesc* host_table, int grid);   // average over the plan's CTAs
 size_t stream_launch_smem(pp_dtype_t dt, int B, int n_pad, int x_len, int max_rows, int batch, int stage_mode, int depth);
 extern int g_stream_depth;   // weight-ring slots per warp: 4, 6 or 8; 0 = chosen per launch
 extern int g_stream_pdl;     // 1: launch with programmatic stream serialization
