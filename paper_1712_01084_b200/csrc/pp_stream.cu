@@ -677,14 +677,16 @@ __device__ __forceinline__ bool stream_f16_layer(const StreamArgs& a, const CtaD
                 }
                 continue;
             }
-            if (GRP == 8 && direct1) {
-                // One input vector, a group that ends the warp's range or crosses a strip boundary: the B operands
-                // of the (up to) eight fragments are built at once, then one pass per strip the group touches
+            if (GRP == 8 && direct) {
+                // A group that ends the warp's range or crosses a strip boundary.  One input vector: the B operands
+                // of the (up to) eight fragments are built at once (several vectors: every lane fetches its own entries
+                // per fragment, as in the full groups above), then one pass per strip the group touches
                 // (nearly always one).  A fragment costs two tests, two shuffles, the ring slot and the tensor-core
                 // instruction: while the weights are in shared memory the SM is bound by instruction issue (eight
                 // warps per scheduler), and the per-fragment bookkeeping of the general loop below took three times
                 // as many instructions, which is most of the multiply phase of a sparse layer.
-                gather8(base);
+                if (direct1) gather8(base);
+                else (void)xw.get(base, wend, lane);              // moves the window when needed
                 const int gend = min(base + 8, wend);
                 int p = base;
                 while (true) {
@@ -699,8 +701,13 @@ __device__ __forceinline__ bool stream_f16_layer(const StreamArgs& a, const CtaD
                     for (int j = 0; j < 8; ++j) {
                         const int q = base + j;
                         if (q >= p && q < end) {
-                            const uint32_t b0 = __shfl_sync(0xffffffffu, mb0, j * 4 + t);
-                            const uint32_t b1 = __shfl_sync(0xffffffffu, mb1, j * 4 + t);
+                            uint32_t b0 = 0u, b1 = 0u;
+                            if (direct1) {
+                                b0 = __shfl_sync(0xffffffffu, mb0, j * 4 + t);
+                                b1 = __shfl_sync(0xffffffffu, mb1, j * 4 + t);
+                            } else {
+                                gather_row(__shfl_sync(0xffffffffu, xw.cur, q - xw.base), b0, b1);
+                            }
                             const uint4 wa = ring.take(j % U);
                             ring.fill(j % U, q + U, wend);
                             mma_16x8x16(acc, wa, b0, b1);
