@@ -718,6 +718,40 @@ __device__ __forceinline__ bool stream_f16_layer(const StreamArgs& a, const CtaD
                 }
                 continue;
             }
+            if (GRP == 8) {
+                // The same pass per strip for an input staged in pivoted order (a chain's inner layers): a lane reads its
+                // operand words straight from the staged row.
+                (void)xw.get(base, wend, lane);              // moves the window when needed
+                const int gend = min(base + 8, wend);
+                int p = base;
+                while (true) {
+                    if (p == seg_end) {
+                        park(ls + warp);
+                        acc[0] = acc[1] = acc[2] = acc[3] = 0.0f;
+                        do { ++ls; } while (L.sstart[ls + 1] <= p);
+                        seg_end = min(wend, L.sstart[ls + 1]);
+                    }
+                    const int end = min(gend, seg_end);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int q = base + j;
+                        if (q >= p && q < end) {
+                            const int xoff = __shfl_sync(0xffffffffu, xw.cur, q - xw.base);
+                            uint32_t b0 = 0u, b1 = 0u;
+                            if (has_x) {
+                                b0 = *reinterpret_cast<const uint32_t*>(xrow + xoff);
+                                b1 = *reinterpret_cast<const uint32_t*>(xrow + xoff + 8);
+                            }
+                            const uint4 wa = ring.take(j % U);
+                            ring.fill(j % U, q + U, wend);
+                            mma_16x8x16(acc, wa, b0, b1);
+                        }
+                    }
+                    p = end;
+                    if (p >= gend) break;
+                }
+                continue;
+            }
 #pragma unroll
             for (int j = 0; j < GRP; ++j) {
                 const int p = base + j;
