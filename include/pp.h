@@ -441,7 +441,8 @@ pp_status_t pp_selftest_host(void);
  *        closer to it than this percentage of a CTA's share
  * key 5: 0 = never use the persistent kernel, 1 = use it when batch <= 8 and x fits shared memory (default 1)
  * key 6: asynchronous 512-byte weight copies each warp of the persistent kernel keeps in flight: 4, 6 or 8;
- *        0 (default) = 4 when two CTAs fit an SM, else the deepest ring that fits
+ *        0 (default) = with two CTAs per SM 4, or 8 for fp16 layers whose warps stream 17 fragments or more while
+ *        two such CTAs still fit an SM; with one CTA per SM the deepest ring that fits
  * key 7: how the persistent kernel applies the column permutation: 2 (default) reads x through the index
  *        array inside the multiply loop for one input vector and, in fp16 layers, for 2..8 vectors; 1 does so
  *        for one vector only; 0 always permutes x into pivoted order in shared memory first
