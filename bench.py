@@ -43,7 +43,7 @@ NOMINAL_HBM_GBS = 8000.0
 MIN_TIMED_CALLS = 2500          # the paper's latency figures average 2,500 calls (Section 5)
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the headline kernel (ncu, profiles/
 # stream_f16_cfg5_k128_batch1.md), valid for the kernel source with this SHA-256 prefix only
-STREAM_TRAFFIC = {"bytes": 139.66e6, "source": "paper_1712_01084_b200/csrc/pp_stream.cu", "sha256_16": "146896e2462268d9"}
+STREAM_TRAFFIC = {"bytes": 139.76e6, "source": "paper_1712_01084_b200/csrc/pp_stream.cu", "sha256_16": "b0612e7a227b1eb7"}
 
 
 def measured_peaks():

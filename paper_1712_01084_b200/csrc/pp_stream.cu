@@ -752,6 +752,7 @@ __device__ __forceinline__ bool stream_f16_layer(const StreamArgs& a, const CtaD
                 }
                 continue;
             }
+            if constexpr (GRP != 8) {            // rings of 6: fragment by fragment
 #pragma unroll
             for (int j = 0; j < GRP; ++j) {
                 const int p = base + j;
@@ -781,6 +782,7 @@ __device__ __forceinline__ bool stream_f16_layer(const StreamArgs& a, const CtaD
                     ring.fill(j % U, p + U, wend);
                     mma_16x8x16(acc, wa, b0, b1);
                 }
+            }
             }
         }
         park(ls + warp);
