@@ -709,3 +709,28 @@ def test_inputs_ready_before_the_stream(pb, dtype, B):
         L.close()
     with pytest.raises(pb.PPError):
         pb.pp_set_tuning(17, 2)
+
+
+@pytest.mark.parametrize("k", [128, 16])
+def test_inputs_ready_full_size(pb, k):
+    """Tuning key 17 on the full-size layer, the launch configuration the bench times: three calls back to back on one
+    layer (shared exchange slots and counters), each against the fp64 product."""
+    wl = synth.config5(k=k, batch=1)
+    lay = wl.layers[0]
+    rng = np.random.default_rng(171 + k)
+    xs = [wl.x] + [rng.uniform(-1, 1, wl.x.shape).astype(wl.x.dtype) for _ in range(2)]
+    xd = [_dev(x) for x in xs]
+    L = pb.Layer.from_synth(lay)
+    torch.cuda.synchronize()
+    try:
+        pb.pp_set_tuning(17, 1)
+        outs = [pb.pp_forward(L, x, lay.act) for x in xd]
+        torch.cuda.synchronize()
+    finally:
+        pb.pp_set_tuning(17, 0)
+    assert L.launch_info(1)["kernel"] == "stream"
+    for i, (x, yd) in enumerate(zip(xs, outs)):
+        y_ref, _, a = po.layer_forward(lay, x.astype(np.float64), act=lay.act, threads=8)
+        _check(yd.cpu().numpy(), y_ref, a, lay.tile_values.dtype, f"k={k} call {i}")
+    assert L.status() == 0
+    L.close()
